@@ -1,0 +1,195 @@
+/*
+ * abs.h -- C ABI of the adaptive-batch-size test and the fused local-optimiser
+ * kernels for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-round batch-size test of the adaptive local
+ * batch size method for local gradient methods and the parameter updates around
+ * it, for M simulated workers held as replicas on ONE GPU:
+ *
+ *   abs_test_stats     mean gradient, norm-test variance, inner-product and
+ *                      orthogonality variances of per-sample gradients
+ *                      (Eq. batch_grad, Eq. def_var, Eq. approx_norm_local)
+ *   abs_next_batch     the ceilings T^m, max{T, b}, the maximum over workers and
+ *                      the cap (Eq. norm_test, Eq. test_stat, Algorithm 1)
+ *   local_sgd_step     x^m <- x^m - alpha g^m           (Eq. local_sgd_alt, line 1)
+ *   local_adamw_step   AdamW inner optimiser             (Section 4.2, Appendix C.2)
+ *   local_shb_step     momentum-SGD inner optimiser      (Section 6.1)
+ *   replica_average    x^m <- (1/M) sum_m x^m            (Eq. local_sgd_alt, line 2)
+ *
+ * Conventions
+ *   - Every function returns an int: ABS_OK (0) or a negative ABS_ERR_* code.
+ *     Nothing throws across this boundary.  abs_last_error() gives a message.
+ *   - Unless a parameter says "host", every tensor pointer is a DEVICE pointer
+ *     owned by the caller, on the device the context was created for.
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL
+ *     is the legacy default stream).  They do not synchronise; results are
+ *     valid in stream order.  The *_host variants are the exception: they copy,
+ *     run and synchronise before returning.
+ *   - A context owns a workspace for per-CTA partial sums.  Calls that use the
+ *     same context must be issued in stream order on one stream at a time.
+ *   - Data-dependent conditions (non-finite input, zero mean gradient, a
+ *     copy that never completed) are reported in abs_stats.status on the
+ *     device; they never trap.
+ *   - Strides are in ELEMENTS of the tensor's type.  All index arithmetic is
+ *     64-bit.
+ */
+#ifndef ABS_H_
+#define ABS_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- error codes ---------------------------------------------------------- */
+#define ABS_OK                0
+#define ABS_ERR_INVALID_ARG  -1   /* null pointer, b < 2, d < 1, stride < extent, ...        */
+#define ABS_ERR_UNSUPPORTED  -2   /* shape outside what the kernels cover (stated per call)  */
+#define ABS_ERR_WORKSPACE    -3   /* the context's workspace is too small for this call      */
+#define ABS_ERR_CUDA         -4   /* a CUDA runtime / driver call failed                     */
+#define ABS_ERR_NO_DEVICE    -5   /* no usable sm_100 device; there is no CPU fallback       */
+
+/* ---- status bits written to abs_stats.status ------------------------------ */
+#define ABS_STATUS_NONFINITE  1u  /* an input or an accumulator was not finite (or overflowed) */
+#define ABS_STATUS_ZERO_MEAN  2u  /* ||gbar||^2 == 0: the test ratios are undefined            */
+#define ABS_STATUS_TIMEOUT    4u  /* an asynchronous tile copy did not arrive in time; the
+                                     numbers in this record are not valid                      */
+
+typedef struct abs_ctx abs_ctx;   /* opaque */
+
+/* Creates a context bound to CUDA device `device` (must be compute capability
+ * 10.x; otherwise ABS_ERR_NO_DEVICE).  workspace_bytes = 0 selects the default
+ * (64 MiB), enough for b <= 4096 rows and M <= 64 workers.  The context owns
+ * its device allocations until abs_destroy. */
+int abs_create(abs_ctx** out, int device, size_t workspace_bytes);
+int abs_destroy(abs_ctx* ctx);
+
+/* Message of the last failing call on this context (host string, owned by the
+ * context, valid until the next call).  ctx may be NULL: then the message of the
+ * last failing abs_create on this thread. */
+const char* abs_last_error(const abs_ctx* ctx);
+
+/* Optional tuning of the tiled statistics kernel; 0 restores the automatic
+ * choice.  key: "stats_stages" (2..8 tile buffers), "stats_ctas_per_worker",
+ * "stats_force_generic" (1 = always use the alignment-free kernel),
+ * "stats_flush_every" (tiles between fp64 flushes of the per-row sums).
+ * Unknown key or out-of-range value: ABS_ERR_INVALID_ARG. */
+int abs_set_tuning(abs_ctx* ctx, const char* key, long long value);
+
+typedef enum { ABS_F32 = 0, ABS_BF16 = 1 } abs_dtype;
+
+/* One record per worker, written by abs_test_stats.  With rows g_1..g_b of one
+ * worker, gbar = (1/b) sum_i g_i (Eq. batch_grad), N = ||gbar||^2,
+ * c_i = <g_i, gbar>:                                                           */
+typedef struct {
+  double gbar_sq;     /* N                                                       */
+  double var_norm;    /* 1/(b-1) sum_i ||g_i - gbar||^2          (Eq. def_var)   */
+  double var_ip;      /* 1/(b-1) sum_i (c_i - mean_i c_i)^2      (Eq. def_var of c_i) */
+  double var_orth;    /* 1/(b-1) sum_i ||o_i - mean o||^2, o_i = g_i - (c_i/N) gbar;
+                         evaluated as var_norm - var_ip / N (equal by orthogonality);
+                         equals var_norm when N == 0                              */
+  double sum_sq;      /* sum_i ||g_i||^2 = (b-1) var_norm + b N                  */
+  long long rows;     /* b                                                       */
+  unsigned status;    /* ABS_STATUS_* bits                                       */
+  unsigned reserved;  /* zero                                                    */
+} abs_stats;          /* 56 bytes */
+
+/* Batch-size test statistics of M workers (Eq. def_var applied per worker,
+ * Eq. approx_norm_local; Algorithm 1, "compute Var").
+ *   G            [M][b][d] per-sample (or per-micro-batch) gradients, dtype fp32
+ *                or bf16; element (m,i,j) at G[m*worker_stride + i*row_stride + j]
+ *   M >= 1, b >= 2 (the variance divides by b-1), d >= 1,
+ *   row_stride >= d, worker_stride >= (b-1)*row_stride + d (ignored if M == 1)
+ *   gbar_out     optional [M][d] fp32 (contiguous, worker m at gbar_out + m*d):
+ *                receives the batch gradients; may be NULL
+ *   stats_out    [M] records
+ * G is read exactly once from HBM when its base address and both strides are
+ * multiples of 16 bytes and b <= 4096; otherwise an alignment-free kernel that
+ * reads it twice is used.  The result does not depend on which kernel ran beyond
+ * floating-point rounding.  Accumulation: fp32 within a tile, fp64 across tiles;
+ * the reduction order is fixed, so repeated calls give bit-identical records.
+ * Errors: ABS_ERR_INVALID_ARG, ABS_ERR_WORKSPACE, ABS_ERR_CUDA.               */
+int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long long b, long long d,
+                   long long row_stride, long long worker_stride,
+                   float* gbar_out, abs_stats* stats_out, void* stream);
+
+/* Same computation for HOST buffers: G_host is copied to a device buffer owned
+ * by the context (grown on demand), the statistics are computed and copied back
+ * to stats_host [M] and, if not NULL, gbar_host [M][d]; the call returns after
+ * everything has completed.  G_host is contiguous ([M][b][d], row_stride = d).
+ * Pinned host memory makes the copies faster but is not required.             */
+int abs_test_stats_host(abs_ctx* ctx, const void* G_host, abs_dtype dtype, int M, long long b,
+                        long long d, float* gbar_host, abs_stats* stats_host, void* stream);
+
+typedef enum { ABS_TEST_NORM = 0, ABS_TEST_AUG_INNER_PRODUCT = 1 } abs_test_kind;
+
+typedef struct {
+  int kind;             /* abs_test_kind                                              */
+  int reserved;         /* zero                                                       */
+  double eta;           /* norm test constant (Eq. approx_norm)                       */
+  double theta;         /* inner-product test constant                                */
+  double nu;            /* orthogonality test constant                                */
+  long long b_max;      /* maximum local batch size (cap), >= 1                       */
+  double row_weight;    /* samples one row stands for: 1 for per-sample gradients, the
+                           micro-batch size for micro-batch gradients, the local batch
+                           size when rows are workers' batch gradients (Section 4.3)   */
+  double divisor;       /* 1, or M for Eq. test_stat_actual / Algorithm 2              */
+} abs_test_cfg;
+
+/* Next local batch size (Eq. norm_test, Eq. test_stat, Algorithm 1: b <- max{T, b};
+ * display below Eq. test_stat: maximum over workers).  Per worker m, in fp64,
+ *   norm test        T^m = ceil( s/D * var_norm / (eta^2 N) )
+ *   augmented ip     T^m = max( ceil( s/D * var_ip / (theta^2 N^2) ),
+ *                               ceil( s/D * var_orth / (nu^2 N) ) )
+ * with s = row_weight, D = divisor; 0/x counts as 0 (also 0/0), x/0 as +infinity;
+ * ceilings saturate at 2^62; a record flagged NONFINITE or TIMEOUT gives T^m = 0.
+ *   b_next = min( b_max, max( b_cur, max_m T^m ) ).
+ *   stats   [M] device records;  cfg  HOST pointer (copied by value at the call)
+ *   b_cur   device, 1 value;  T_out device [M] or NULL;  b_next device, 1 value
+ *           (may alias b_cur).  M <= 1024.                                          */
+int abs_next_batch(abs_ctx* ctx, const abs_stats* stats, int M, const abs_test_cfg* cfg,
+                   const long long* b_cur, long long* T_out, long long* b_next, void* stream);
+
+/* Local SGD step for all replicas (Eq. local_sgd_alt): X[m] <- X[m] - lr * Gb[m],
+ * m < M, in fp32.  X, Gb: [M][d] fp32 with replica m at + m*replica_stride
+ * (>= d).  average_after != 0 fuses the model averaging of the round's last step:
+ * every replica receives (1/M) sum_m (X[m] - lr*Gb[m]) at no extra memory traffic.
+ * X is updated in place.                                                        */
+int local_sgd_step(abs_ctx* ctx, float* X, const float* Gb, int M, long long d,
+                   long long replica_stride, float lr, int average_after, void* stream);
+
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;
+  int reserved;       /* zero */
+  long long step;     /* t >= 1, shared by all replicas, keeps counting across rounds */
+} abs_adamw_cfg;
+
+/* Local AdamW step for all replicas (inner optimiser of Section 4.2 / Appendix
+ * C.2; rule of the cited optimiser, decoupled weight decay):
+ *   m <- beta1 m + (1-beta1) g ;  v <- beta2 v + (1-beta2) g^2
+ *   x <- x (1 - lr wd) - lr (m / (1-beta1^t)) / ( sqrt(v / (1-beta2^t)) + eps )
+ * X, Mom1, Mom2, Gb: [M][d] fp32, same replica_stride; all but Gb updated in place.
+ * average_after != 0: X[m] <- mean over replicas of the updated X; the moments
+ * stay local.  cfg is a HOST pointer.                                           */
+int local_adamw_step(abs_ctx* ctx, float* X, float* Mom1, float* Mom2, const float* Gb, int M,
+                     long long d, long long replica_stride, const abs_adamw_cfg* cfg,
+                     int average_after, void* stream);
+
+/* Local stochastic-heavy-ball (momentum SGD) step, the inner optimiser of the
+ * paper's image experiments (Section 6.1):
+ *   g <- g + wd x ;  u <- momentum u + g ;  x <- x - lr u
+ * X, Buf (the momentum buffer u), Gb: [M][d] fp32.                              */
+int local_shb_step(abs_ctx* ctx, float* X, float* Buf, const float* Gb, int M, long long d,
+                   long long replica_stride, float lr, float momentum, float weight_decay,
+                   int average_after, void* stream);
+
+/* Model averaging (Eq. local_sgd_alt, second line; Algorithm 1 "update the
+ * global model"): every replica receives (1/M) sum_m X[m], in place.            */
+int replica_average(abs_ctx* ctx, float* X, int M, long long d, long long replica_stride,
+                    void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* ABS_H_ */
