@@ -1,0 +1,79 @@
+// Internal declarations shared by the translation units of the library.
+// Nothing here is part of the public C ABI (see include/abs.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "abs.h"
+
+namespace absk {
+
+constexpr int kSmCountFallback = 148;
+constexpr size_t kDefaultWorkspace = 64ull << 20;
+constexpr int kMaxFastRows = 4096;          // largest b the tiled statistics kernel covers
+
+struct Tuning {
+  long long stats_stages = 0;
+  long long stats_ctas_per_worker = 0;
+  long long stats_force_generic = 0;
+  long long stats_flush_every = 0;
+  long long stats_stage_kb = 0;
+};
+
+}  // namespace absk
+
+// The context: device, workspace for per-CTA partial sums, a device staging area
+// for the *_host entry points, tuning knobs and the last error message.
+struct abs_ctx {
+  int device = 0;
+  int sm_count = absk::kSmCountFallback;
+  size_t smem_optin = 0;
+  void* workspace = nullptr;       // device
+  size_t workspace_bytes = 0;
+  unsigned* flags = nullptr;       // device, 64 words: [0] async-copy timeout flag
+  void* staging = nullptr;         // device buffer for *_host calls, grown on demand
+  size_t staging_bytes = 0;
+  void* staging_out = nullptr;     // device buffer for stats / gbar of *_host calls
+  size_t staging_out_bytes = 0;
+  absk::Tuning tuning;
+  char err[512] = {0};
+};
+
+namespace absk {
+
+int set_error(abs_ctx* ctx, int code, const char* fmt, ...);
+
+#define ABS_CUDA_TRY(ctx, expr)                                                          \
+  do {                                                                                   \
+    cudaError_t e__ = (expr);                                                            \
+    if (e__ != cudaSuccess)                                                              \
+      return absk::set_error((ctx), ABS_ERR_CUDA, "%s failed: %s", #expr,                \
+                             cudaGetErrorString(e__));                                   \
+  } while (0)
+
+// ---- statistics kernels (abs_stats_tiled.cu, abs_stats_generic.cu) ---------------------
+// Layout of the partial-sum workspace written by both statistics kernels:
+//   ws[(m * P + p) * (b + 2) + r]      r < b : sum over the CTA's columns of (g_rj - gbar_j) gbar_j
+//   ws[(m * P + p) * (b + 2) + b]              sum over the CTA's columns of sum_r (g_rj - gbar_j)^2
+//   ws[(m * P + p) * (b + 2) + b + 1]          sum over the CTA's columns of gbar_j^2
+struct StatsLaunch {
+  const void* G;
+  abs_dtype dtype;
+  int M;
+  long long b, d, row_stride, worker_stride;
+  float* gbar_out;
+  abs_stats* stats_out;
+  cudaStream_t stream;
+};
+
+// Returns ABS_OK, or ABS_ERR_UNSUPPORTED when the tiled kernel cannot take the call
+// (alignment, b too large); *P_out receives the number of partial records per worker.
+int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
+int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
+int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P);
+
+}  // namespace absk

@@ -1,0 +1,226 @@
+// Alignment-free statistics kernel and the fp64 finalisation of the batch-size test.
+//
+// The generic kernel takes any base address, any strides and any b.  A CTA owns a
+// strip of 256 columns at a time: sweep A sums the strip's columns over all rows
+// (Eq. batch_grad), sweep B re-reads the strip (from L2 when it is still there) and
+// forms the centred sums of Eq. def_var.  Loads are scalar and coalesced across a
+// warp.  It reads G twice and is the fallback of the tiled kernel, not the fast path.
+#include <cuda_bf16.h>
+
+#include "abs_internal.cuh"
+
+namespace absk {
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kStrip = 256;
+
+__device__ __forceinline__ float load_elt(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float load_elt(const __nv_bfloat16* p) {
+  return __uint_as_float(static_cast<unsigned>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+}
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long long row_stride,
+                         long long worker_stride, long long n_strips, int P, double* __restrict__ ws,
+                         float* __restrict__ gbar_out) {
+  __shared__ float colpart[kWarps][kStrip];
+  __shared__ float gbar_s[kStrip];
+  __shared__ double red[2 * kWarps];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m = blockIdx.y, p = blockIdx.x;
+  const T* Gm = G + static_cast<long long>(m) * worker_stride;
+  double* out = ws + (static_cast<size_t>(m) * P + p) * (static_cast<size_t>(b) + 2);
+  const float inv_b = 1.0f / static_cast<float>(b);
+
+  for (long long r = tid; r < b; r += kThreads) out[r] = 0.0;
+  __syncthreads();
+
+  double vacc = 0.0, nacc = 0.0;
+  for (long long it = p; it < n_strips; it += P) {
+    const long long j0 = it * kStrip;
+    // sweep A: column sums, rows split over the warps
+    float cs[kStrip / 32];
+#pragma unroll
+    for (int c = 0; c < kStrip / 32; ++c) cs[c] = 0.f;
+    for (long long r = warp; r < b; r += kWarps) {
+      const T* row = Gm + r * row_stride + j0;
+#pragma unroll
+      for (int c = 0; c < kStrip / 32; ++c) {
+        const long long col = j0 + c * 32 + lane;
+        if (col < d) cs[c] += load_elt(row + c * 32 + lane);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < kStrip / 32; ++c) colpart[warp][c * 32 + lane] = cs[c];
+    __syncthreads();
+    {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) s += colpart[w][tid];
+      const float g = s * inv_b;
+      gbar_s[tid] = g;
+      if (j0 + tid < d) {
+        nacc += static_cast<double>(g * g);
+        if (gbar_out != nullptr) gbar_out[static_cast<long long>(m) * d + j0 + tid] = g;
+      }
+    }
+    __syncthreads();
+    // sweep B: centred sums; one warp owns a row, so e_r has a single writer
+    float gl[kStrip / 32];
+#pragma unroll
+    for (int c = 0; c < kStrip / 32; ++c) gl[c] = gbar_s[c * 32 + lane];
+    float vl = 0.f;
+    for (long long r = warp; r < b; r += kWarps) {
+      const T* row = Gm + r * row_stride + j0;
+      float el = 0.f;
+#pragma unroll
+      for (int c = 0; c < kStrip / 32; ++c) {
+        const long long col = j0 + c * 32 + lane;
+        if (col < d) {
+          const float dlt = load_elt(row + c * 32 + lane) - gl[c];
+          vl = fmaf(dlt, dlt, vl);
+          el = fmaf(dlt, gl[c], el);
+        }
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) el += __shfl_xor_sync(0xffffffffu, el, off);
+      if (lane == 0) out[r] += static_cast<double>(el);
+    }
+    vacc += static_cast<double>(vl);
+    __syncthreads();
+  }
+
+  vacc = warp_sum_d(vacc);
+  nacc = warp_sum_d(nacc);
+  if (lane == 0) {
+    red[warp] = vacc;
+    red[kWarps + warp] = nacc;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double vs = 0.0, ns = 0.0;
+    for (int w = 0; w < kWarps; ++w) {
+      vs += red[w];
+      ns += red[kWarps + w];
+    }
+    out[b] = vs;
+    out[b + 1] = ns;
+  }
+}
+
+// One CTA per worker folds the P partial records in a fixed order and writes abs_stats.
+constexpr int kFinalThreads = 1024;
+
+__global__ void __launch_bounds__(kFinalThreads)
+abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, const unsigned* __restrict__ flags,
+                          abs_stats* __restrict__ stats_out) {
+  __shared__ double red[4][kFinalThreads / 32];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m = blockIdx.x;
+  const size_t rec = static_cast<size_t>(b) + 2;
+  const double* base = ws + static_cast<size_t>(m) * P * rec;
+
+  double se = 0.0, see = 0.0;
+  for (long long r = tid; r < b; r += kFinalThreads) {
+    double e = 0.0;
+    for (int p = 0; p < P; ++p) e += base[p * rec + r];
+    se += e;
+    see += e * e;
+  }
+  // V and N: thread t takes the records p = t, t + 1024, ...
+  double vn = 0.0, nn = 0.0;
+  for (int p = tid; p < P; p += kFinalThreads) {
+    vn += base[p * rec + b];
+    nn += base[p * rec + b + 1];
+  }
+  const double a0 = warp_sum_d(se), a1 = warp_sum_d(see), a2 = warp_sum_d(vn), a3 = warp_sum_d(nn);
+  if (lane == 0) {
+    red[0][warp] = a0;
+    red[1][warp] = a1;
+    red[2][warp] = a2;
+    red[3][warp] = a3;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double s_e = 0.0, s_ee = 0.0, V = 0.0, N = 0.0;
+    for (int w = 0; w < kFinalThreads / 32; ++w) {
+      s_e += red[0][w];
+      s_ee += red[1][w];
+      V += red[2][w];
+      N += red[3][w];
+    }
+    const double bd = static_cast<double>(b);
+    const double var_norm = V / (bd - 1.0);
+    double ss = s_ee - s_e * s_e / bd;     // sum_i (e_i - mean e)^2; mean e is rounding noise only
+    if (ss < 0.0) ss = 0.0;
+    const double var_ip = ss / (bd - 1.0);
+    double var_orth = var_norm;
+    if (N > 0.0) {
+      var_orth = var_norm - var_ip / N;
+      if (var_orth < 0.0) var_orth = 0.0;
+    }
+    unsigned status = 0u;
+    if (!(isfinite(V) && isfinite(N) && isfinite(s_ee))) status |= ABS_STATUS_NONFINITE;
+    if (N == 0.0) status |= ABS_STATUS_ZERO_MEAN;
+    if (flags[0] != 0u) status |= ABS_STATUS_TIMEOUT;
+    abs_stats s;
+    s.gbar_sq = N;
+    s.var_norm = var_norm;
+    s.var_ip = var_ip;
+    s.var_orth = var_orth;
+    s.sum_sq = V + bd * N;
+    s.rows = b;
+    s.status = status;
+    s.reserved = 0u;
+    stats_out[m] = s;
+  }
+}
+
+}  // namespace
+
+int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
+  const long long n_strips = (a.d + kStrip - 1) / kStrip;
+  long long P = (static_cast<long long>(ctx->sm_count) * 4) / a.M;
+  if (P < 1) P = 1;
+  if (P > n_strips) P = n_strips;
+  if (P > 65535) P = 65535;
+  if (a.M > 65535) return set_error(ctx, ABS_ERR_UNSUPPORTED, "M = %d exceeds 65535", a.M);
+  // fit the workspace: fewer CTAs per worker if b is very large
+  const size_t rec = (static_cast<size_t>(a.b) + 2) * sizeof(double);
+  while (P > 1 && static_cast<size_t>(a.M) * P * rec > ctx->workspace_bytes) P = (P + 1) / 2;
+  if (static_cast<size_t>(a.M) * P * rec > ctx->workspace_bytes)
+    return set_error(ctx, ABS_ERR_WORKSPACE, "abs_test_stats needs %zu workspace bytes, context has %zu",
+                     static_cast<size_t>(a.M) * P * rec, ctx->workspace_bytes);
+  const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
+  double* ws = static_cast<double*>(ctx->workspace);
+  if (a.dtype == ABS_F32)
+    abs_stats_generic_kernel<float><<<grid, kThreads, 0, a.stream>>>(
+        static_cast<const float*>(a.G), a.b, a.d, a.row_stride, a.worker_stride, n_strips, static_cast<int>(P), ws,
+        a.gbar_out);
+  else
+    abs_stats_generic_kernel<__nv_bfloat16><<<grid, kThreads, 0, a.stream>>>(
+        static_cast<const __nv_bfloat16*>(a.G), a.b, a.d, a.row_stride, a.worker_stride, n_strips,
+        static_cast<int>(P), ws, a.gbar_out);
+  ABS_CUDA_TRY(ctx, cudaGetLastError());
+  *P_out = static_cast<int>(P);
+  return ABS_OK;
+}
+
+int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P) {
+  abs_stats_finalize_kernel<<<a.M, kFinalThreads, 0, a.stream>>>(static_cast<const double*>(ctx->workspace), a.b, P,
+                                                               ctx->flags, a.stats_out);
+  ABS_CUDA_TRY(ctx, cudaGetLastError());
+  return ABS_OK;
+}
+
+}  // namespace absk
