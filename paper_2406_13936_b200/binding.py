@@ -1,0 +1,240 @@
+"""Thin ctypes binding of the C ABI in include/abs.h.
+
+Argument marshalling only: every function takes torch tensors (device memory) or
+plain numbers, passes raw pointers and sizes to the library and raises AbsError on a
+non-zero return code.  Nothing is computed here, and there is no fallback: if the
+shared library is missing or cannot be loaded the import of a function fails loudly.
+"""
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+ABS_F32, ABS_BF16 = 0, 1
+ABS_TEST_NORM, ABS_TEST_AUG_INNER_PRODUCT = 0, 1
+STATUS_NONFINITE, STATUS_ZERO_MEAN, STATUS_TIMEOUT = 1, 2, 4
+STATS_RECORD_BYTES = 56
+
+
+class AbsError(RuntimeError):
+    pass
+
+
+class TestCfg(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("reserved", ctypes.c_int), ("eta", ctypes.c_double),
+                ("theta", ctypes.c_double), ("nu", ctypes.c_double), ("b_max", ctypes.c_longlong),
+                ("row_weight", ctypes.c_double), ("divisor", ctypes.c_double)]
+
+
+class AdamWCfg(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
+                ("eps", ctypes.c_float), ("weight_decay", ctypes.c_float), ("reserved", ctypes.c_int),
+                ("step", ctypes.c_longlong)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("gbar_sq", ctypes.c_double), ("var_norm", ctypes.c_double), ("var_ip", ctypes.c_double),
+                ("var_orth", ctypes.c_double), ("sum_sq", ctypes.c_double), ("rows", ctypes.c_longlong),
+                ("status", ctypes.c_uint), ("reserved", ctypes.c_uint)]
+
+
+EXPORTS = {
+    "abs_create": [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_size_t],
+    "abs_destroy": [ctypes.c_void_p],
+    "abs_set_tuning": [ctypes.c_void_p, ctypes.c_char_p, ctypes.c_longlong],
+    "abs_test_stats": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
+                       ctypes.c_longlong, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_void_p,
+                       ctypes.c_void_p, ctypes.c_void_p],
+    "abs_test_stats_host": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
+                            ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_next_batch": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(TestCfg),
+                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "local_sgd_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
+                       ctypes.c_longlong, ctypes.c_float, ctypes.c_int, ctypes.c_void_p],
+    "local_adamw_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                         ctypes.c_int, ctypes.c_longlong, ctypes.c_longlong, ctypes.POINTER(AdamWCfg),
+                         ctypes.c_int, ctypes.c_void_p],
+    "local_shb_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                       ctypes.c_longlong, ctypes.c_longlong, ctypes.c_float, ctypes.c_float, ctypes.c_float,
+                       ctypes.c_int, ctypes.c_void_p],
+    "replica_average": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_longlong,
+                        ctypes.c_void_p],
+}
+
+_lib = None
+
+
+def library_path():
+    return _build.LIB_PATH
+
+
+def load_library():
+    """dlopen the CUDA library; raises AbsError if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise AbsError("CUDA library %s is missing: run paper_2406_13936_b200.build.build() "
+                       "(there is no CPU fallback)" % path)
+    lib = ctypes.CDLL(path)
+    for name, argtypes in EXPORTS.items():
+        fn = getattr(lib, name)
+        fn.argtypes = argtypes
+        fn.restype = ctypes.c_int
+    lib.abs_last_error.argtypes = [ctypes.c_void_p]
+    lib.abs_last_error.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else ctypes.c_void_p(0)
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dtype_code(t):
+    if t.dtype == torch.float32:
+        return ABS_F32
+    if t.dtype == torch.bfloat16:
+        return ABS_BF16
+    raise AbsError("G must be float32 or bfloat16, got %s" % t.dtype)
+
+
+class Context:
+    """Owns an abs_ctx.  One context per device; calls are issued in stream order."""
+
+    def __init__(self, device=0, workspace_bytes=0):
+        self._lib = load_library()
+        handle = ctypes.c_void_p()
+        rc = self._lib.abs_create(ctypes.byref(handle), int(device), int(workspace_bytes))
+        if rc != 0:
+            raise AbsError("abs_create failed (%d): %s" % (rc, self._lib.abs_last_error(None).decode()))
+        self._h = handle
+        self.device = int(device)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.abs_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc, what):
+        if rc != 0:
+            raise AbsError("%s failed (%d): %s" % (what, rc, self._lib.abs_last_error(self._h).decode()))
+
+    def set_tuning(self, key, value):
+        self._check(self._lib.abs_set_tuning(self._h, key.encode(), int(value)), "abs_set_tuning")
+
+    # ---- statistics --------------------------------------------------------------------
+    def new_stats(self, M):
+        """Device buffer for M abs_stats records (M x 7 float64 words)."""
+        return torch.zeros((M, 7), dtype=torch.float64, device="cuda:%d" % self.device)
+
+    def abs_test_stats(self, G, stats_out, gbar_out=None, stream=None):
+        """G: [M, b, d] or [b, d] device tensor (last dim contiguous); stats_out from new_stats."""
+        if G.dim() == 2:
+            G = G.unsqueeze(0)
+        if G.stride(2) != 1:
+            raise AbsError("the last dimension of G must be contiguous")
+        M, b, d = G.shape
+        rc = self._lib.abs_test_stats(self._h, _ptr(G), _dtype_code(G), M, b, d, G.stride(1), G.stride(0),
+                                      _ptr(gbar_out), _ptr(stats_out), _stream(stream))
+        self._check(rc, "abs_test_stats")
+        return stats_out
+
+    def abs_test_stats_host(self, G_host, want_gbar=False, stream=None):
+        """G_host: contiguous CPU tensor [M, b, d]; returns (list of stats dicts, gbar or None)."""
+        if G_host.dim() == 2:
+            G_host = G_host.unsqueeze(0)
+        G_host = G_host.contiguous()
+        M, b, d = G_host.shape
+        recs = (Stats * M)()
+        gbar = torch.empty((M, d), dtype=torch.float32) if want_gbar else None
+        rc = self._lib.abs_test_stats_host(self._h, _ptr(G_host), _dtype_code(G_host), M, b, d, _ptr(gbar),
+                                           ctypes.cast(recs, ctypes.c_void_p), _stream(stream))
+        self._check(rc, "abs_test_stats_host")
+        return [_record_to_dict(r) for r in recs], gbar
+
+    def abs_next_batch(self, stats, cfg, b_cur, b_next, T_out=None, stream=None):
+        """stats: device records; cfg: TestCfg; b_cur / b_next: int64 device tensors of one element."""
+        M = stats.shape[0]
+        rc = self._lib.abs_next_batch(self._h, _ptr(stats), M, ctypes.byref(cfg), _ptr(b_cur), _ptr(T_out),
+                                      _ptr(b_next), _stream(stream))
+        self._check(rc, "abs_next_batch")
+        return b_next
+
+    # ---- local updates -------------------------------------------------------------------
+    @staticmethod
+    def _replicas(X):
+        if X.dim() == 1:
+            X = X.unsqueeze(0)
+        if X.stride(1) != 1:
+            raise AbsError("replica tensors must be contiguous in the last dimension")
+        return X, X.shape[0], X.shape[1], X.stride(0)
+
+    def local_sgd_step(self, X, Gb, lr, average_after=False, stream=None):
+        X2, M, d, stride = self._replicas(X)
+        Gb2, _, _, gstride = self._replicas(Gb)
+        if gstride != stride and M > 1:
+            raise AbsError("X and Gb must share the replica stride")
+        self._check(self._lib.local_sgd_step(self._h, _ptr(X2), _ptr(Gb2), M, d, stride, float(lr),
+                                             int(bool(average_after)), _stream(stream)), "local_sgd_step")
+
+    def local_adamw_step(self, X, Mom1, Mom2, Gb, cfg, average_after=False, stream=None):
+        X2, M, d, stride = self._replicas(X)
+        for t in (Mom1, Mom2, Gb):
+            if self._replicas(t)[3] != stride and M > 1:
+                raise AbsError("all replica tensors must share the replica stride")
+        self._check(self._lib.local_adamw_step(self._h, _ptr(X2), _ptr(Mom1), _ptr(Mom2), _ptr(Gb), M, d, stride,
+                                               ctypes.byref(cfg), int(bool(average_after)), _stream(stream)),
+                    "local_adamw_step")
+
+    def local_shb_step(self, X, Buf, Gb, lr, momentum, weight_decay, average_after=False, stream=None):
+        X2, M, d, stride = self._replicas(X)
+        for t in (Buf, Gb):
+            if self._replicas(t)[3] != stride and M > 1:
+                raise AbsError("all replica tensors must share the replica stride")
+        self._check(self._lib.local_shb_step(self._h, _ptr(X2), _ptr(Buf), _ptr(Gb), M, d, stride, float(lr),
+                                             float(momentum), float(weight_decay), int(bool(average_after)),
+                                             _stream(stream)), "local_shb_step")
+
+    def replica_average(self, X, stream=None):
+        X2, M, d, stride = self._replicas(X)
+        self._check(self._lib.replica_average(self._h, _ptr(X2), M, d, stride, _stream(stream)), "replica_average")
+
+
+def _record_to_dict(r):
+    return dict(gbar_sq=r.gbar_sq, var_norm=r.var_norm, var_ip=r.var_ip, var_orth=r.var_orth, sum_sq=r.sum_sq,
+                rows=r.rows, status=r.status)
+
+
+def stats_to_dicts(stats):
+    """Copy device abs_stats records (tensor from Context.new_stats) to a list of dicts."""
+    host = stats.detach().cpu().contiguous()
+    raw = host.numpy().tobytes()
+    out = []
+    for m in range(host.shape[0]):
+        out.append(_record_to_dict(Stats.from_buffer_copy(raw[m * STATS_RECORD_BYTES:(m + 1) * STATS_RECORD_BYTES])))
+    return out
+
+
+def make_test_cfg(kind, b_max, eta=0.0, theta=0.0, nu=0.0, row_weight=1.0, divisor=1.0):
+    code = {"norm": ABS_TEST_NORM, "aug_ip": ABS_TEST_AUG_INNER_PRODUCT}[kind]
+    return TestCfg(code, 0, float(eta), float(theta), float(nu), int(b_max), float(row_weight), float(divisor))
+
+
+def make_adamw_cfg(lr, beta1, beta2, eps, weight_decay, step):
+    return AdamWCfg(float(lr), float(beta1), float(beta2), float(eps), float(weight_decay), 0, int(step))

@@ -1,0 +1,186 @@
+// Context management, argument validation and dispatch for the statistics entry points.
+#include <stdarg.h>
+#include <new>
+
+#include "abs_internal.cuh"
+
+namespace absk {
+
+static thread_local char g_create_error[512] = {0};
+
+int set_error(abs_ctx* ctx, int code, const char* fmt, ...) {
+  char* dst = ctx != nullptr ? ctx->err : g_create_error;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(dst, 512, fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+namespace {
+
+struct DeviceScope {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceScope(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    if (prev == dev) prev = -1;
+  }
+  ~DeviceScope() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int validate_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long long b, long long d,
+                   long long row_stride, long long worker_stride, const abs_stats* stats_out) {
+  if (G == nullptr || stats_out == nullptr) return set_error(ctx, ABS_ERR_INVALID_ARG, "G or stats_out is null");
+  if (dtype != ABS_F32 && dtype != ABS_BF16) return set_error(ctx, ABS_ERR_INVALID_ARG, "unknown dtype %d", (int)dtype);
+  if (M < 1) return set_error(ctx, ABS_ERR_INVALID_ARG, "M must be >= 1, got %d", M);
+  if (b < 2) return set_error(ctx, ABS_ERR_INVALID_ARG, "b must be >= 2 (the variance divides by b-1), got %lld", b);
+  if (d < 1) return set_error(ctx, ABS_ERR_INVALID_ARG, "d must be >= 1, got %lld", d);
+  if (b > (1ll << 24)) return set_error(ctx, ABS_ERR_UNSUPPORTED, "b = %lld exceeds 2^24 rows", b);
+  if (row_stride < d) return set_error(ctx, ABS_ERR_INVALID_ARG, "row_stride %lld < d %lld", row_stride, d);
+  if (M > 1 && worker_stride < (b - 1) * row_stride + d)
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "worker_stride %lld overlaps the previous worker", worker_stride);
+  return ABS_OK;
+}
+
+int run_stats(abs_ctx* ctx, const StatsLaunch& a) {
+  ABS_CUDA_TRY(ctx, cudaMemsetAsync(ctx->flags, 0, sizeof(unsigned), a.stream));
+  int P = 0;
+  int rc = ABS_ERR_UNSUPPORTED;
+  if (!ctx->tuning.stats_force_generic) rc = launch_stats_tiled(ctx, a, &P);
+  if (rc == ABS_ERR_UNSUPPORTED) rc = launch_stats_generic(ctx, a, &P);
+  if (rc != ABS_OK) return rc;
+  return launch_stats_finalize(ctx, a, P);
+}
+
+int grow(abs_ctx* ctx, void** buf, size_t* have, size_t need) {
+  if (*have >= need) return ABS_OK;
+  if (*buf != nullptr) {
+    ABS_CUDA_TRY(ctx, cudaFree(*buf));
+    *buf = nullptr;
+    *have = 0;
+  }
+  ABS_CUDA_TRY(ctx, cudaMalloc(buf, need));
+  *have = need;
+  return ABS_OK;
+}
+
+}  // namespace
+}  // namespace absk
+
+using namespace absk;
+
+extern "C" int abs_create(abs_ctx** out, int device, size_t workspace_bytes) {
+  if (out == nullptr) return set_error(nullptr, ABS_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || count < 1) {
+    cudaGetLastError();
+    return set_error(nullptr, ABS_ERR_NO_DEVICE, "no CUDA device is visible; this library has no CPU fallback");
+  }
+  if (device < 0 || device >= count) return set_error(nullptr, ABS_ERR_INVALID_ARG, "device %d out of range", device);
+  int major = 0, sms = 0, optin = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess)
+    return set_error(nullptr, ABS_ERR_CUDA, "cannot query device %d", device);
+  if (major != 10)
+    return set_error(nullptr, ABS_ERR_NO_DEVICE, "device %d has compute capability %d.x; the kernels are built for 10.x only",
+                     device, major);
+  abs_ctx* ctx = new (std::nothrow) abs_ctx();
+  if (ctx == nullptr) return set_error(nullptr, ABS_ERR_CUDA, "out of host memory");
+  ctx->device = device;
+  ctx->sm_count = sms;
+  ctx->smem_optin = static_cast<size_t>(optin);
+  ctx->workspace_bytes = workspace_bytes ? workspace_bytes : kDefaultWorkspace;
+  DeviceScope scope(device);
+  cudaError_t e = scope.ok ? cudaMalloc(&ctx->workspace, ctx->workspace_bytes) : cudaErrorInvalidDevice;
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->flags), 64 * sizeof(unsigned));
+  if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, 64 * sizeof(unsigned));
+  if (e != cudaSuccess) {
+    set_error(nullptr, ABS_ERR_CUDA, "allocating the context failed: %s", cudaGetErrorString(e));
+    if (ctx->workspace) cudaFree(ctx->workspace);
+    if (ctx->flags) cudaFree(ctx->flags);
+    delete ctx;
+    return ABS_ERR_CUDA;
+  }
+  *out = ctx;
+  return ABS_OK;
+}
+
+extern "C" int abs_destroy(abs_ctx* ctx) {
+  if (ctx == nullptr) return ABS_OK;
+  DeviceScope scope(ctx->device);
+  if (ctx->workspace) cudaFree(ctx->workspace);
+  if (ctx->flags) cudaFree(ctx->flags);
+  if (ctx->staging) cudaFree(ctx->staging);
+  if (ctx->staging_out) cudaFree(ctx->staging_out);
+  delete ctx;
+  return ABS_OK;
+}
+
+extern "C" const char* abs_last_error(const abs_ctx* ctx) { return ctx != nullptr ? ctx->err : g_create_error; }
+
+extern "C" int abs_set_tuning(abs_ctx* ctx, const char* key, long long value) {
+  if (ctx == nullptr || key == nullptr) return ABS_ERR_INVALID_ARG;
+  if (value < 0) return set_error(ctx, ABS_ERR_INVALID_ARG, "tuning values are >= 0");
+  if (strcmp(key, "stats_stages") == 0) {
+    if (value != 0 && (value < 2 || value > 8)) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_stages must be 0 or 2..8");
+    ctx->tuning.stats_stages = value;
+  } else if (strcmp(key, "stats_ctas_per_worker") == 0) {
+    if (value > 65535) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_ctas_per_worker must be <= 65535");
+    ctx->tuning.stats_ctas_per_worker = value;
+  } else if (strcmp(key, "stats_force_generic") == 0) {
+    ctx->tuning.stats_force_generic = value ? 1 : 0;
+  } else if (strcmp(key, "stats_flush_every") == 0) {
+    if (value > 4096) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_flush_every must be <= 4096");
+    ctx->tuning.stats_flush_every = value;
+  } else if (strcmp(key, "stats_stage_kb") == 0) {
+    if (value != 0 && (value < 4 || value > 200)) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_stage_kb must be 0 or 4..200");
+    ctx->tuning.stats_stage_kb = value;
+  } else {
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "unknown tuning key '%s'", key);
+  }
+  return ABS_OK;
+}
+
+extern "C" int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long long b, long long d,
+                              long long row_stride, long long worker_stride, float* gbar_out, abs_stats* stats_out,
+                              void* stream) {
+  if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
+  int rc = validate_stats(ctx, G, dtype, M, b, d, row_stride, worker_stride, stats_out);
+  if (rc != ABS_OK) return rc;
+  DeviceScope scope(ctx->device);
+  if (!scope.ok) return set_error(ctx, ABS_ERR_CUDA, "cannot select device %d", ctx->device);
+  StatsLaunch a{G, dtype, M, b, d, row_stride, worker_stride, gbar_out, stats_out, static_cast<cudaStream_t>(stream)};
+  return run_stats(ctx, a);
+}
+
+extern "C" int abs_test_stats_host(abs_ctx* ctx, const void* G_host, abs_dtype dtype, int M, long long b, long long d,
+                                   float* gbar_host, abs_stats* stats_host, void* stream) {
+  if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
+  int rc = validate_stats(ctx, G_host, dtype, M, b, d, d, b * d, stats_host);
+  if (rc != ABS_OK) return rc;
+  DeviceScope scope(ctx->device);
+  if (!scope.ok) return set_error(ctx, ABS_ERR_CUDA, "cannot select device %d", ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t es = dtype == ABS_F32 ? 4 : 2;
+  const size_t g_bytes = static_cast<size_t>(M) * b * d * es;
+  const size_t stats_bytes = (static_cast<size_t>(M) * sizeof(abs_stats) + 255) / 256 * 256;
+  const size_t gbar_bytes = gbar_host != nullptr ? static_cast<size_t>(M) * d * sizeof(float) : 0;
+  rc = grow(ctx, &ctx->staging, &ctx->staging_bytes, g_bytes);
+  if (rc != ABS_OK) return rc;
+  rc = grow(ctx, &ctx->staging_out, &ctx->staging_out_bytes, stats_bytes + gbar_bytes);
+  if (rc != ABS_OK) return rc;
+  abs_stats* d_stats = static_cast<abs_stats*>(ctx->staging_out);
+  float* d_gbar = gbar_host != nullptr ? reinterpret_cast<float*>(static_cast<char*>(ctx->staging_out) + stats_bytes) : nullptr;
+  ABS_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->staging, G_host, g_bytes, cudaMemcpyHostToDevice, st));
+  StatsLaunch a{ctx->staging, dtype, M, b, d, d, b * d, d_gbar, d_stats, st};
+  rc = run_stats(ctx, a);
+  if (rc != ABS_OK) return rc;
+  ABS_CUDA_TRY(ctx, cudaMemcpyAsync(stats_host, d_stats, static_cast<size_t>(M) * sizeof(abs_stats), cudaMemcpyDeviceToHost, st));
+  if (gbar_host != nullptr) ABS_CUDA_TRY(ctx, cudaMemcpyAsync(gbar_host, d_gbar, gbar_bytes, cudaMemcpyDeviceToHost, st));
+  ABS_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  return ABS_OK;
+}
