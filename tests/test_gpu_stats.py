@@ -134,7 +134,7 @@ def test_tiled_and_generic_kernels_agree_and_are_deterministic(ctx):
     for ra, rg in zip(a, g):
         for key in ("gbar_sq", "var_norm", "var_ip", "var_orth", "sum_sq"):
             assert ra[key] == pytest.approx(rg[key], rel=1e-6)
-    np.testing.assert_allclose(ga.cpu().numpy(), gg.cpu().numpy(), rtol=1e-6, atol=1e-9)
+    np.testing.assert_allclose(ga.cpu().numpy(), gg.cpu().numpy(), rtol=1e-6, atol=1e-6 * ga.abs().max().item())
 
 
 @pytest.mark.parametrize("key,value", [("stats_stages", 2), ("stats_stages", 6), ("stats_stage_kb", 16),
