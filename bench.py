@@ -1,0 +1,361 @@
+"""Benchmark of the batch-size-test hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic per-sample gradients:
+  abs_test_stats (mean gradient, norm / inner-product / orthogonality variances)
+  -> abs_next_batch (ceilings, max over workers, cap)
+  -> local_adamw_step on the mean gradient with the model averaging fused in.
+The headline value is the bytes of G the step consumes divided by the step time (GB/s);
+rounds/s is its reciprocal.  Extra legs time the fused AdamW / SGD steps and the bf16
+statistics on their own workloads.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = dict(name="stats sweep centre: G fp32 [M=1, b=256, d=11.2M], sigma=1, eta=theta=nu=0.5",
+                M=1, b=256, d=11_200_000, sigma=1.0, seed=2)
+HP = dict(lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0]))
+                    mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_step(G_np, x, m, v, b, t):
+    """The whole step in the CPU oracle, as it stands."""
+    import oracle.abs_oracle as orc
+    s = orc.batch_test_stats(G_np)
+    orc.next_batch([s], b, 1 << 20, "aug_ip", theta=0.5, nu=0.5)
+    orc.next_batch([s], b, 1 << 20, "norm", eta=0.5)
+    x, m, v = orc.adamw_step(x, m, v, s["gbar"][None, :], t=t, **HP)
+    return orc.replica_average(x), m, v
+
+
+def cpu_sample(divisor=4):
+    import numpy as np
+    from paper_2406_13936_b200 import inputs
+    b, d = WORKLOAD["b"], WORKLOAD["d"] // divisor
+    G = inputs.gaussian_rows(WORKLOAD["seed"], 1, b, d, WORKLOAD["sigma"], device="cpu")[0].numpy()
+    x = np.zeros((1, d))
+    return G, x, "first %d of %d columns (1/%d of the workload), all %d rows" % (d, WORKLOAD["d"], divisor, b)
+
+
+def time_cpu_baseline():
+    import numpy as np
+    G, x, what = cpu_sample()
+    t0 = time.perf_counter()
+    oracle_step(G, x, np.zeros_like(x), np.zeros_like(x), WORKLOAD["b"], 1)
+    dt = time.perf_counter() - t0
+    return dict(value=G.nbytes / dt / 1e9, unit="GB/s", cores=1, kind="oracle", sample=what,
+                seconds=round(dt, 3))
+
+
+def run_reference(args):
+    """The oracle timed on the host cores on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    G, x, what = cpu_sample(divisor=16)
+    m, v = np.zeros_like(x), np.zeros_like(x)
+    for t in range(args.warmup):
+        oracle_step(G, x, m, v, WORKLOAD["b"], t + 1)
+    t0 = time.perf_counter()
+    for t in range(args.steps):
+        oracle_step(G, x, m, v, WORKLOAD["b"], t + 1)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = G.nbytes / dt / 1e9
+    line = dict(impl="reference", metric="batch_test_step_GBps", value=value, unit="GB/s", n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=dt * 1e3, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=WORKLOAD["name"], sample=what),
+                cpu_baseline=dict(value=value, unit="GB/s", cores=1, kind="oracle", sample=what),
+                e2e=dict(value=value, unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU legs
+def time_steps(torch, fn, steps, warmup):
+    """CUDA-event timing of `steps` calls of fn(i) after `warmup` untimed ones; returns seconds per call."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn(warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / 1e3 / steps
+
+
+def extra_legs(torch, pkg, inputs, ctx, peak):
+    """Fused optimiser steps and bf16 statistics on their own workloads (not the headline)."""
+    out = {}
+    free = torch.cuda.mem_get_info()[0]
+    # fused local AdamW + averaging: M=8 fp32 replicas of a GPT-2-small-sized model, H=16 steps per round
+    M, d, H = 8, 124_439_808, 16
+    if free > 40e9:
+        X, m1, m2, grads = inputs.adamw_problem(4, M, d, pool=2, device="cuda")
+        t = [0]
+
+        def adamw(i, avg=False):
+            t[0] += 1
+            ctx.local_adamw_step(X, m1, m2, grads[i % 2], pkg.make_adamw_cfg(step=t[0], **HP), average_after=avg)
+
+        sec = time_steps(torch, adamw, 8, 3)
+        sec_avg = time_steps(torch, lambda i: adamw(i, True), 8, 3)
+        gbs = 28.0 * M * d / sec / 1e9
+        out["adamw_step"] = dict(workload="M=8 d=124,439,808 fp32, 28 B/element", ms=sec * 1e3, GBps=gbs,
+                                 frac_of_peak=gbs / peak, ms_with_fused_average=sec_avg * 1e3,
+                                 GBps_with_fused_average=28.0 * M * d / sec_avg / 1e9)
+        round_s = (H - 1) * sec + sec_avg
+        out["adamw_round"] = dict(workload="H=16 local AdamW steps, averaging fused into the last",
+                                  rounds_per_s=1.0 / round_s, ms_per_round=round_s * 1e3)
+        sec = time_steps(torch, lambda i: ctx.local_sgd_step(X, grads[i % 2], 1e-3), 8, 3)
+        out["sgd_step"] = dict(workload="M=8 d=124,439,808 fp32, 12 B/element", ms=sec * 1e3,
+                               GBps=12.0 * M * d / sec / 1e9, frac_of_peak=12.0 * M * d / sec / 1e9 / peak)
+        sec = time_steps(torch, lambda i: ctx.replica_average(X), 8, 3)
+        out["replica_average"] = dict(workload="stand-alone, 8 B/element/replica", ms=sec * 1e3,
+                                      GBps=8.0 * M * d / sec / 1e9, frac_of_peak=8.0 * M * d / sec / 1e9 / peak)
+        del X, m1, m2, grads
+        torch.cuda.empty_cache()
+    # bf16 statistics: M=8 workers x 16 micro-batch gradients of a GPT-2-small-sized model
+    free = torch.cuda.mem_get_info()[0]
+    M, b = 8, 16
+    if free > 45e9:
+        G = inputs.student_t_rows(3, M, b, d, device="cuda")
+        stats = ctx.new_stats(M)
+        sec = time_steps(torch, lambda i: ctx.abs_test_stats(G, stats), 10, 3)
+        gbs = G.numel() * 2 / sec / 1e9
+        out["stats_bf16"] = dict(workload="G bf16 [8, 16, 124,439,808] Student-t rows", ms=sec * 1e3, GBps=gbs,
+                                 frac_of_peak=gbs / peak)
+        del G
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_ours(args):
+    import torch
+    import paper_2406_13936_b200 as pkg
+    from paper_2406_13936_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pkg.build.build()
+    ctx = pkg.Context(local)
+    peak, peak_kind = measured_peak()
+
+    M, b, d = WORKLOAD["M"], WORKLOAD["b"], WORKLOAD["d"]
+    G = inputs.gaussian_rows(WORKLOAD["seed"] + rank, M, b, d, WORKLOAD["sigma"], device="cuda")
+    X, m1, m2, _ = inputs.adamw_problem(4, M, d, pool=0, device="cuda")
+    gbar = torch.empty((M, d), device="cuda")
+    stats = ctx.new_stats(M)
+    b_cur = torch.tensor([b], dtype=torch.int64, device="cuda")
+    b_next = torch.zeros(1, dtype=torch.int64, device="cuda")
+    T_out = torch.zeros(M, dtype=torch.int64, device="cuda")
+    cfg = pkg.make_test_cfg("aug_ip", 1 << 20, theta=0.5, nu=0.5)
+    cfg_norm = pkg.make_test_cfg("norm", 1 << 20, eta=0.5)
+    g_bytes = G.numel() * G.element_size()
+    n_ev = args.steps
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
+
+    def step(i, timed=-1):
+        if timed >= 0:
+            ev[timed][0].record()
+        ctx.abs_test_stats(G, stats, gbar)
+        if timed >= 0:
+            ev[timed][1].record()
+        ctx.abs_next_batch(stats, cfg, b_cur, b_next, T_out)       # augmented inner-product test
+        ctx.abs_next_batch(stats, cfg_norm, b_cur, b_next, T_out)  # norm test
+        ctx.local_adamw_step(X, m1, m2, gbar, pkg.make_adamw_cfg(step=i + 1, **HP), average_after=True)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(args.steps):
+        step(args.warmup + i, timed=i)
+    t1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    sec = t0.elapsed_time(t1) / 1e3
+    stats_ms = sum(a.elapsed_time(z) for a, z in ev) / n_ev
+    if dist is not None:
+        tt = torch.tensor([sec], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        sec = tt.item()
+    ms_per_step = sec / args.steps * 1e3
+    value = world * g_bytes * args.steps / sec / 1e9
+    launches_per_step = 2 + 2 + 1      # tiled statistics + finalise, two next-batch kernels, fused AdamW
+    rec = pkg.stats_to_dicts(stats)[0]
+
+    # end to end: G starts in pinned host memory, results are read back every step
+    e2e = None
+    if rank == 0 or world > 1:
+        G_host = torch.empty((M, b, d), dtype=torch.float32, pin_memory=True)
+        G_host.copy_(G)
+        del G
+        torch.cuda.empty_cache()
+
+        def host_step(i):
+            ctx.abs_test_stats_host(G_host, gbar_dev=gbar, stats_dev=stats)
+            ctx.abs_next_batch(stats, cfg, b_cur, b_next, T_out)
+            ctx.abs_next_batch(stats, cfg_norm, b_cur, b_next, T_out)
+            ctx.local_adamw_step(X, m1, m2, gbar, pkg.make_adamw_cfg(step=i + 1, **HP), average_after=True)
+            return b_next.item()
+
+        host_step(0)
+        torch.cuda.synchronize()
+        n_e2e = 3
+        w0 = time.perf_counter()
+        for i in range(n_e2e):
+            host_step(1 + i)
+        torch.cuda.synchronize()
+        e2e_sec = (time.perf_counter() - w0) / n_e2e
+        if dist is not None:
+            tt = torch.tensor([e2e_sec], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_sec = tt.item()
+        e2e = dict(value=world * g_bytes / e2e_sec / 1e9, unit="GB/s", h2d_bytes_per_step=g_bytes,
+                   d2h_bytes_per_step=56 * M + 8, steps=n_e2e, ms_per_step=e2e_sec * 1e3)
+        del G_host
+
+    extra = None
+    if rank == 0 and world == 1 and not args.no_extra:
+        extra = extra_legs(torch, pkg, inputs, ctx, peak)
+    cpu = time_cpu_baseline() if (rank == 0 and world == 1) else None
+
+    if rank == 0:
+        achieved = g_bytes / (stats_ms / 1e3) / 1e9
+        line = dict(
+            metric="batch_test_step_GBps", value=value, unit="GB/s", n_gpus=world, steps=args.steps,
+            warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+            dtype="f32", data="synthetic",
+            config=dict(workload=WORKLOAD["name"], M=M, b=b, d=d, bytes_per_step=g_bytes,
+                        l2="inputs (11.5 GB) larger than L2, no flush needed",
+                        step="abs_test_stats + abs_next_batch (aug. inner-product and norm) + local_adamw_step "
+                             "with fused replica_average",
+                        shard="one independent problem per GPU, no collective"),
+            rounds_per_s=world * args.steps / sec,
+            roofline=dict(bound="hbm", kernel="abs_stats_tiled_kernel<float,16,keep> (+ finalise)",
+                          achieved=achieved, peak=peak, unit="GB/s", frac=achieved / peak, peak_kind=peak_kind,
+                          frac_of_nominal_8TBps=achieved / 8000.0, ms=stats_ms, traffic=None),
+            cpu_baseline=cpu, e2e=e2e, gpu_launches=launches_per_step * args.steps, clocks=clocks,
+            result=dict(b_next=int(b_next.item()), var_norm=rec["var_norm"], gbar_sq=rec["gbar_sq"],
+                        status=rec["status"]),
+            extra=extra)
+        print(json.dumps(line))
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

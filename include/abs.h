@@ -73,7 +73,8 @@ const char* abs_last_error(const abs_ctx* ctx);
 /* Optional tuning of the tiled statistics kernel; 0 restores the automatic
  * choice.  key: "stats_stages" (2..8 tile buffers), "stats_ctas_per_worker",
  * "stats_force_generic" (1 = always use the alignment-free kernel),
- * "stats_flush_every" (tiles between fp64 flushes of the per-row sums).
+ * "stats_flush_every" (tiles between fp64 flushes of the per-row sums),
+ * "stats_stage_kb" (upper bound on one tile buffer, 4..200 KiB).
  * Unknown key or out-of-range value: ABS_ERR_INVALID_ARG. */
 int abs_set_tuning(abs_ctx* ctx, const char* key, long long value);
 
@@ -118,9 +119,13 @@ int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long lon
  * by the context (grown on demand), the statistics are computed and copied back
  * to stats_host [M] and, if not NULL, gbar_host [M][d]; the call returns after
  * everything has completed.  G_host is contiguous ([M][b][d], row_stride = d).
- * Pinned host memory makes the copies faster but is not required.             */
+ * Pinned host memory makes the copies faster but is not required.
+ * stats_dev / gbar_dev are optional DEVICE buffers ([M] records, [M][d] fp32) that
+ * receive the same results on the device, for a following abs_next_batch /
+ * local_*_step that should not wait for another host-to-device copy.            */
 int abs_test_stats_host(abs_ctx* ctx, const void* G_host, abs_dtype dtype, int M, long long b,
-                        long long d, float* gbar_host, abs_stats* stats_host, void* stream);
+                        long long d, float* gbar_host, abs_stats* stats_host,
+                        float* gbar_dev, abs_stats* stats_dev, void* stream);
 
 typedef enum { ABS_TEST_NORM = 0, ABS_TEST_AUG_INNER_PRODUCT = 1 } abs_test_kind;
 

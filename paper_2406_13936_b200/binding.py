@@ -48,7 +48,8 @@ EXPORTS = {
                        ctypes.c_longlong, ctypes.c_longlong, ctypes.c_longlong, ctypes.c_void_p,
                        ctypes.c_void_p, ctypes.c_void_p],
     "abs_test_stats_host": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
-                            ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+                            ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                            ctypes.c_void_p],
     "abs_next_batch": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(TestCfg),
                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "local_sgd_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
@@ -155,8 +156,9 @@ class Context:
         self._check(rc, "abs_test_stats")
         return stats_out
 
-    def abs_test_stats_host(self, G_host, want_gbar=False, stream=None):
-        """G_host: contiguous CPU tensor [M, b, d]; returns (list of stats dicts, gbar or None)."""
+    def abs_test_stats_host(self, G_host, want_gbar=False, gbar_dev=None, stats_dev=None, stream=None):
+        """G_host: contiguous CPU tensor [M, b, d]; returns (list of stats dicts, gbar or None).
+        gbar_dev / stats_dev: optional device tensors that also receive the results."""
         if G_host.dim() == 2:
             G_host = G_host.unsqueeze(0)
         G_host = G_host.contiguous()
@@ -164,7 +166,8 @@ class Context:
         recs = (Stats * M)()
         gbar = torch.empty((M, d), dtype=torch.float32) if want_gbar else None
         rc = self._lib.abs_test_stats_host(self._h, _ptr(G_host), _dtype_code(G_host), M, b, d, _ptr(gbar),
-                                           ctypes.cast(recs, ctypes.c_void_p), _stream(stream))
+                                           ctypes.cast(recs, ctypes.c_void_p), _ptr(gbar_dev), _ptr(stats_dev),
+                                           _stream(stream))
         self._check(rc, "abs_test_stats_host")
         return [_record_to_dict(r) for r in recs], gbar
 

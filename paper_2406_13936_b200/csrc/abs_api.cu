@@ -158,7 +158,8 @@ extern "C" int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int 
 }
 
 extern "C" int abs_test_stats_host(abs_ctx* ctx, const void* G_host, abs_dtype dtype, int M, long long b, long long d,
-                                   float* gbar_host, abs_stats* stats_host, void* stream) {
+                                   float* gbar_host, abs_stats* stats_host, float* gbar_dev, abs_stats* stats_dev,
+                                   void* stream) {
   if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
   int rc = validate_stats(ctx, G_host, dtype, M, b, d, d, b * d, stats_host);
   if (rc != ABS_OK) return rc;
@@ -168,19 +169,23 @@ extern "C" int abs_test_stats_host(abs_ctx* ctx, const void* G_host, abs_dtype d
   const size_t es = dtype == ABS_F32 ? 4 : 2;
   const size_t g_bytes = static_cast<size_t>(M) * b * d * es;
   const size_t stats_bytes = (static_cast<size_t>(M) * sizeof(abs_stats) + 255) / 256 * 256;
-  const size_t gbar_bytes = gbar_host != nullptr ? static_cast<size_t>(M) * d * sizeof(float) : 0;
+  const bool own_gbar = gbar_host != nullptr && gbar_dev == nullptr;
+  const size_t gbar_bytes = static_cast<size_t>(M) * d * sizeof(float);
   rc = grow(ctx, &ctx->staging, &ctx->staging_bytes, g_bytes);
   if (rc != ABS_OK) return rc;
-  rc = grow(ctx, &ctx->staging_out, &ctx->staging_out_bytes, stats_bytes + gbar_bytes);
+  rc = grow(ctx, &ctx->staging_out, &ctx->staging_out_bytes, stats_bytes + (own_gbar ? gbar_bytes : 0));
   if (rc != ABS_OK) return rc;
-  abs_stats* d_stats = static_cast<abs_stats*>(ctx->staging_out);
-  float* d_gbar = gbar_host != nullptr ? reinterpret_cast<float*>(static_cast<char*>(ctx->staging_out) + stats_bytes) : nullptr;
+  abs_stats* d_stats = stats_dev != nullptr ? stats_dev : static_cast<abs_stats*>(ctx->staging_out);
+  float* d_gbar = gbar_dev;
+  if (own_gbar) d_gbar = reinterpret_cast<float*>(static_cast<char*>(ctx->staging_out) + stats_bytes);
   ABS_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->staging, G_host, g_bytes, cudaMemcpyHostToDevice, st));
   StatsLaunch a{ctx->staging, dtype, M, b, d, d, b * d, d_gbar, d_stats, st};
   rc = run_stats(ctx, a);
   if (rc != ABS_OK) return rc;
-  ABS_CUDA_TRY(ctx, cudaMemcpyAsync(stats_host, d_stats, static_cast<size_t>(M) * sizeof(abs_stats), cudaMemcpyDeviceToHost, st));
-  if (gbar_host != nullptr) ABS_CUDA_TRY(ctx, cudaMemcpyAsync(gbar_host, d_gbar, gbar_bytes, cudaMemcpyDeviceToHost, st));
+  ABS_CUDA_TRY(ctx, cudaMemcpyAsync(stats_host, d_stats, static_cast<size_t>(M) * sizeof(abs_stats),
+                                    cudaMemcpyDeviceToHost, st));
+  if (gbar_host != nullptr)
+    ABS_CUDA_TRY(ctx, cudaMemcpyAsync(gbar_host, d_gbar, gbar_bytes, cudaMemcpyDeviceToHost, st));
   ABS_CUDA_TRY(ctx, cudaStreamSynchronize(st));
   return ABS_OK;
 }
