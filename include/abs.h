@@ -127,6 +127,42 @@ int abs_test_stats_host(abs_ctx* ctx, const void* G_host, abs_dtype dtype, int M
                         long long d, float* gbar_host, abs_stats* stats_host,
                         float* gbar_dev, abs_stats* stats_dev, void* stream);
 
+/* Statistics without any allocation.  (The paper has no counterpart: this entry
+ * point exists for the sake of the calling program, not of the method.)
+ *
+ * abs_create allocates a device workspace, and cudaMalloc / cudaFree synchronise the
+ * device.  Some callers cannot accept that: programs whose device memory is handed
+ * out entirely by their own pool, plug-ins that run under a fixed memory budget,
+ * latency-critical sections that must not hit an implicit device synchronisation.
+ * For them this call computes exactly what abs_test_stats computes, takes no
+ * context, and keeps its scratch (per-CTA partial sums and a status word) in a
+ * fixed array of ABS_NOALLOC_SCRATCH_BYTES + 256 bytes that is part of the library
+ * image: every GPU on which the library is loaded holds that array until the
+ * process exits, used or not.
+ *   - Arguments and results as for abs_test_stats; the device used is the CURRENT
+ *     CUDA device of the calling thread, and all pointers must belong to it.
+ *   - Limits: b <= ABS_NOALLOC_MAX_ROWS and M <= ABS_NOALLOC_MAX_WORKERS; larger
+ *     problems are refused with ABS_ERR_UNSUPPORTED (message from
+ *     abs_noalloc_last_error) and need abs_test_stats with a context.
+ *   - The first call on each device looks up the device address of the array and a
+ *     few device attributes (no allocation by this library; a CUDA runtime that
+ *     loads modules lazily places the array on the GPU at this moment).  Make that
+ *     first call during start-up, outside any stream capture.
+ *   - All calls on one device share the one array.  It still holds the previous
+ *     call's partial sums; the call clears what has to start at zero itself.  Two
+ *     calls that can run on the GPU at the same time (different streams, different
+ *     host threads) would overwrite each other's partial sums: issue them in one
+ *     stream, or order them with events.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine.                    */
+#define ABS_NOALLOC_SCRATCH_BYTES (8u << 20)
+#define ABS_NOALLOC_MAX_ROWS      2048
+#define ABS_NOALLOC_MAX_WORKERS   64
+int abs_test_stats_noalloc(const void* G, abs_dtype dtype, int M, long long b, long long d,
+                           long long row_stride, long long worker_stride,
+                           float* gbar_out, abs_stats* stats_out, void* stream);
+/* Message of the last failing abs_test_stats_noalloc call on this thread. */
+const char* abs_noalloc_last_error(void);
+
 typedef enum { ABS_TEST_NORM = 0, ABS_TEST_AUG_INNER_PRODUCT = 1 } abs_test_kind;
 
 typedef struct {

@@ -50,6 +50,9 @@ EXPORTS = {
     "abs_test_stats_host": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
                             ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                             ctypes.c_void_p],
+    "abs_test_stats_noalloc": [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_longlong, ctypes.c_longlong,
+                               ctypes.c_longlong, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p,
+                               ctypes.c_void_p],
     "abs_next_batch": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(TestCfg),
                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "local_sgd_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
@@ -87,6 +90,8 @@ def load_library():
         fn.restype = ctypes.c_int
     lib.abs_last_error.argtypes = [ctypes.c_void_p]
     lib.abs_last_error.restype = ctypes.c_char_p
+    lib.abs_noalloc_last_error.argtypes = []
+    lib.abs_noalloc_last_error.restype = ctypes.c_char_p
     _lib = lib
     return lib
 
@@ -217,6 +222,26 @@ class Context:
     def replica_average(self, X, stream=None):
         X2, M, d, stride = self._replicas(X)
         self._check(self._lib.replica_average(self._h, _ptr(X2), M, d, stride, _stream(stream)), "replica_average")
+
+
+def abs_test_stats_noalloc(G, stats_out, gbar_out=None, stream=None):
+    """Context-free statistics that allocate nothing (scratch is a fixed array inside the library).
+
+    For callers that may not call cudaMalloc: same arguments and results as
+    Context.abs_test_stats, limited to b <= 2048 rows and M <= 64 workers, on the current
+    CUDA device.  Calls that may overlap on the GPU must be ordered by the caller.
+    """
+    lib = load_library()
+    if G.dim() == 2:
+        G = G.unsqueeze(0)
+    if G.stride(2) != 1:
+        raise AbsError("the last dimension of G must be contiguous")
+    M, b, d = G.shape
+    rc = lib.abs_test_stats_noalloc(_ptr(G), _dtype_code(G), M, b, d, G.stride(1), G.stride(0), _ptr(gbar_out),
+                                    _ptr(stats_out), _stream(stream))
+    if rc != 0:
+        raise AbsError("abs_test_stats_noalloc failed (%d): %s" % (rc, lib.abs_noalloc_last_error().decode()))
+    return stats_out
 
 
 def _record_to_dict(r):
