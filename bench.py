@@ -208,6 +208,54 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
     return out
 
 
+PROFILE_CASES = {
+    # small cases of the same kernels for profiler captures: larger than L2, about 1 GB on the device
+    "stats_f32_b256": dict(kind="stats", M=1, b=256, d=1_000_000, dtype="f32"),
+    "stats_f32_b64": dict(kind="stats", M=1, b=64, d=4_000_000, dtype="f32"),
+    "stats_f32_b1024": dict(kind="stats", M=1, b=1024, d=256_000, dtype="f32"),
+    "stats_bf16_b16": dict(kind="stats", M=8, b=16, d=4_000_000, dtype="bf16"),
+    "adamw": dict(kind="adamw", M=8, d=8_000_000),
+    # full-size cases of the sweep, for timing only (not for multi-pass captures)
+    "stats_f32_b64_d11m": dict(kind="stats", M=1, b=64, d=11_200_000, dtype="f32"),
+    "stats_f32_b256_d11m": dict(kind="stats", M=1, b=256, d=11_200_000, dtype="f32"),
+    "stats_f32_b1024_d11m": dict(kind="stats", M=1, b=1024, d=11_200_000, dtype="f32"),
+    "stats_bf16_b16_d124m": dict(kind="stats", M=8, b=16, d=124_439_808, dtype="bf16"),
+}
+
+
+def run_profile_case(args):
+    """A few launches of one kernel on a small case (for ncu); prints its CUDA-event time."""
+    import torch
+    import paper_2406_13936_b200 as pkg
+    from paper_2406_13936_b200 import inputs
+    case = PROFILE_CASES[args.case]
+    pkg.build.build()
+    ctx = pkg.Context(0)
+    for kv in args.tune:
+        key, val = kv.split("=")
+        ctx.set_tuning(key, int(val))
+    peak, _ = measured_peak()
+    if case["kind"] == "stats":
+        M, b, d = case["M"], case["b"], case["d"]
+        if case["dtype"] == "f32":
+            G = inputs.gaussian_rows(2, M, b, d, 1.0, device="cuda")
+        else:
+            G = inputs.gaussian_rows(2, M, b, d, 1.0, device="cuda", dtype=torch.bfloat16)
+        stats = ctx.new_stats(M)
+        nbytes = G.numel() * G.element_size()
+        sec = time_steps(torch, lambda i: ctx.abs_test_stats(G, stats), args.steps, args.warmup)
+    else:
+        M, d = case["M"], case["d"]
+        X, m1, m2, grads = inputs.adamw_problem(4, M, d, pool=1, device="cuda")
+        nbytes = 28 * M * d
+        sec = time_steps(torch, lambda i: ctx.local_adamw_step(X, m1, m2, grads[0],
+                                                               pkg.make_adamw_cfg(step=i + 1, **HP)),
+                         args.steps, args.warmup)
+    print(json.dumps(dict(case=args.case, tune=args.tune, ms=sec * 1e3, GBps=nbytes / sec / 1e9,
+                          frac_of_peak=nbytes / sec / 1e9 / peak, bytes=nbytes)))
+    ctx.close()
+
+
 def run_ours(args):
     import torch
     import paper_2406_13936_b200 as pkg
@@ -349,9 +397,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true")
+    ap.add_argument("--case", default=None, choices=sorted(PROFILE_CASES),
+                    help="run only a few launches of one kernel on a small case (for profiler captures)")
+    ap.add_argument("--tune", action="append", default=[], help="key=value passed to abs_set_tuning (with --case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
-    if args.impl == "reference":
+    if args.case:
+        run_profile_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

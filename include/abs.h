@@ -74,7 +74,10 @@ const char* abs_last_error(const abs_ctx* ctx);
  * choice.  key: "stats_stages" (2..8 tile buffers), "stats_ctas_per_worker",
  * "stats_force_generic" (1 = always use the alignment-free kernel),
  * "stats_flush_every" (tiles between fp64 flushes of the per-row sums),
- * "stats_stage_kb" (upper bound on one tile buffer, 4..200 KiB).
+ * "stats_stage_kb" (upper bound on one tile buffer, 4..200 KiB),
+ * "stats_no_gram" (1 = do not use the tensor-core Gram kernel for bf16, b <= 32),
+ * "stats_ctas_per_sm" (1: one CTA per SM, 64 KiB buffers, up to 16 rows per
+ * thread; 2: two CTAs per SM, 32 KiB buffers, up to 8 rows per thread).
  * Unknown key or out-of-range value: ABS_ERR_INVALID_ARG. */
 int abs_set_tuning(abs_ctx* ctx, const char* key, long long value);
 
@@ -106,8 +109,9 @@ typedef struct {
  *                receives the batch gradients; may be NULL
  *   stats_out    [M] records
  * G is read exactly once from HBM when its base address and both strides are
- * multiples of 16 bytes and b <= 4096; otherwise an alignment-free kernel that
- * reads it twice is used.  The result does not depend on which kernel ran beyond
+ * multiples of 16 bytes and b <= 4096 (bf16 input with b <= 32 goes through a
+ * tensor-core Gram-matrix kernel, everything else through the tiled kernel);
+ * otherwise an alignment-free kernel that reads it twice is used.  The result does not depend on which kernel ran beyond
  * floating-point rounding.  Accumulation: fp32 within a tile, fp64 across tiles;
  * the reduction order is fixed, so repeated calls give bit-identical records.
  * Errors: ABS_ERR_INVALID_ARG, ABS_ERR_WORKSPACE, ABS_ERR_CUDA.               */

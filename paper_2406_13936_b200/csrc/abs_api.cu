@@ -48,7 +48,8 @@ int run_stats(abs_ctx* ctx, const StatsLaunch& a) {
   ABS_CUDA_TRY(ctx, cudaMemsetAsync(ctx->flags, 0, sizeof(unsigned), a.stream));
   int P = 0;
   int rc = ABS_ERR_UNSUPPORTED;
-  if (!ctx->tuning.stats_force_generic) rc = launch_stats_tiled(ctx, a, &P);
+  if (!ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_gram) rc = launch_stats_gram(ctx, a, &P);
+  if (rc == ABS_ERR_UNSUPPORTED && !ctx->tuning.stats_force_generic) rc = launch_stats_tiled(ctx, a, &P);
   if (rc == ABS_ERR_UNSUPPORTED) rc = launch_stats_generic(ctx, a, &P);
   if (rc != ABS_OK) return rc;
   return launch_stats_finalize(ctx, a, P);
@@ -139,6 +140,11 @@ extern "C" int abs_set_tuning(abs_ctx* ctx, const char* key, long long value) {
   } else if (strcmp(key, "stats_stage_kb") == 0) {
     if (value != 0 && (value < 4 || value > 200)) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_stage_kb must be 0 or 4..200");
     ctx->tuning.stats_stage_kb = value;
+  } else if (strcmp(key, "stats_no_gram") == 0) {
+    ctx->tuning.stats_no_gram = value ? 1 : 0;
+  } else if (strcmp(key, "stats_ctas_per_sm") == 0) {
+    if (value > 2) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_ctas_per_sm must be 0, 1 or 2");
+    ctx->tuning.stats_ctas_per_sm = value;
   } else {
     return set_error(ctx, ABS_ERR_INVALID_ARG, "unknown tuning key '%s'", key);
   }

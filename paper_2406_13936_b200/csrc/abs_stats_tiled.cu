@@ -20,7 +20,7 @@
 // folded into per-thread fp64 every tile.  All reductions have a fixed order.
 #include <cuda_bf16.h>
 
-#include "abs_internal.cuh"
+#include "abs_pipeline.cuh"
 
 namespace absk {
 namespace {
@@ -47,63 +47,6 @@ struct TiledParams {
   unsigned* flags;
   long long timeout_cycles;
 };
-
-// ---- PTX wrappers ------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after `limit` clock cycles (or as soon as another thread of the
-// CTA gave up), raises the CTA's abort flag and returns false.  The caller carries on
-// with whatever is in shared memory; the record is flagged ABS_STATUS_TIMEOUT.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile unsigned* abort_flag,
-                                          long long limit) {
-  if (mbar_try_wait(bar, parity)) return true;
-  if (*abort_flag) return false;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (*abort_flag || clock64() - t0 > limit) {
-      *abort_flag = 1u;
-      return false;
-    }
-  }
-  return true;
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
-                                            uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-      "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ void named_bar_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
 
 // ---- element traits ------------------------------------------------------------------------
 template <typename T>
@@ -134,15 +77,12 @@ struct Vec<__nv_bfloat16> {
   }
 };
 
-__device__ __forceinline__ double warp_sum(double v) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  return v;
-}
-
 // ---- the kernel ----------------------------------------------------------------------------
-template <typename T, int RMAX, bool KEEP>
-__global__ void __launch_bounds__(kThreads, 1)
+// RMAX: upper bound on the rows a thread owns; KEEP: the rows stay in registers between the
+// sweeps; FULL: every thread owns exactly RMAX rows (no per-row predicates).  Variants with
+// at most 8 rows per thread are compiled for two CTAs per SM.
+template <typename T, int RMAX, bool KEEP, bool FULL>
+__global__ void __launch_bounds__(kThreads, (RMAX <= 8 ? 2 : 1))
 abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledParams prm) {
   constexpr int VE = Vec<T>::VE;
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -251,7 +191,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
       for (int j = 0; j < VE; ++j) cs[j] = 0.f;
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
-        if (k < n_rows_mine) {
+        if (FULL || k < n_rows_mine) {
           const uint4 u = lds128(base + static_cast<uint32_t>(k) * row_step);
           if (KEEP) v[k] = u;
           float x[VE];
@@ -310,24 +250,34 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
       }
 
       // sweep 2: centred sums
-      float vl = 0.f;
+      float vl[VE];     // one accumulator per column: VE independent dependency chains
+#pragma unroll
+      for (int j = 0; j < VE; ++j) vl[j] = 0.f;
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
-        if (k < n_rows_mine) {
+        if (FULL || k < n_rows_mine) {
           const uint4 u = KEEP ? v[k] : lds128(base + static_cast<uint32_t>(k) * row_step);
           float x[VE];
           Vec<T>::unpack(u, x);
-          float ek = e[k];
+          float ea = 0.f, eb = 0.f;
 #pragma unroll
-          for (int j = 0; j < VE; ++j) {
-            const float dlt = x[j] - g[j];
-            vl = fmaf(dlt, dlt, vl);
-            ek = fmaf(dlt, g[j], ek);
+          for (int j = 0; j < VE; j += 2) {
+            const float d0 = x[j] - g[j];
+            const float d1 = x[j + 1] - g[j + 1];
+            vl[j] = fmaf(d0, d0, vl[j]);
+            vl[j + 1] = fmaf(d1, d1, vl[j + 1]);
+            ea = fmaf(d0, g[j], ea);
+            eb = fmaf(d1, g[j + 1], eb);
           }
-          e[k] = ek;
+          e[k] += ea + eb;
         }
       }
-      vacc += static_cast<double>(vl);
+      {
+        float vs = 0.f;
+#pragma unroll
+        for (int j = 0; j < VE; ++j) vs += vl[j];
+        vacc += static_cast<double>(vs);
+      }
       if (!KEEP) {
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_u32 + 8u * s);
@@ -339,7 +289,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
         for (int k = 0; k < RMAX; ++k) {
           float ek = e[k];
           for (int off = 1; off < lpr; off <<= 1) ek += __shfl_xor_sync(0xffffffffu, ek, off);
-          if (cv == 0 && k < n_rows_mine) e_mine[rg + k * RG] += static_cast<double>(ek);
+          if (cv == 0 && (FULL || k < n_rows_mine)) e_mine[rg + k * RG] += static_cast<double>(ek);
           e[k] = 0.f;
         }
       }
@@ -373,25 +323,9 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
 }
 
 // ---- host side -----------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(sym);
-  }
-  return fn;
-}
-
 struct TileChoice {
   int lpr_log2, rs_log2, bx, stages, box_rows, n_row_boxes, rmax;
-  bool keep;
+  bool keep, full;
   unsigned box_bytes, stage_bytes;
   size_t smem_bytes;
 };
@@ -403,10 +337,13 @@ size_t extras_bytes(int lpr, int ve, int bx, long long b, int stages) {
 
 // Picks the widest box rows that leave every thread at most 16 rows (so the tile can stay in
 // registers between the sweeps) and whose stage fits the per-stage budget.
-bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, size_t stage_max, TileChoice* c) {
+bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, size_t stage_max, int keep_rows,
+                 TileChoice* c) {
   const int n_row_boxes = static_cast<int>((b + 255) / 256);
+  // with at most 8 rows per thread the kernel is compiled for two CTAs per SM: leave room for both
+  const size_t smem_budget = keep_rows <= 8 ? (smem_optin - 2048) / 2 : smem_optin;
   for (int pass = 0; pass < 2; ++pass) {            // pass 0: tile kept in registers; pass 1: re-read
-    const int rows_per_thread = pass == 0 ? 16 : 32;
+    const int rows_per_thread = pass == 0 ? keep_rows : 32;
     for (int lpr_log2 = 5; lpr_log2 >= 0; --lpr_log2) {
       const int lpr = 1 << lpr_log2;
       const int subs = 32 / lpr;
@@ -426,8 +363,8 @@ bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, 
       const size_t stage = static_cast<size_t>(bx) * rows_pad * lpr * 16;
       if (stage > stage_max) continue;
       int stages = static_cast<int>(want_stages > 0 ? want_stages : 3);
-      while (stages > 2 && stages * stage + extras_bytes(lpr, ve, bx, b, stages) + 128 > smem_optin) --stages;
-      if (stages * stage + extras_bytes(lpr, ve, bx, b, stages) + 128 > smem_optin) continue;
+      while (stages > 2 && stages * stage + extras_bytes(lpr, ve, bx, b, stages) + 128 > smem_budget) --stages;
+      if (stages * stage + extras_bytes(lpr, ve, bx, b, stages) + 128 > smem_budget) continue;
       const long long RG = static_cast<long long>(subs) << rs_log2;
       const long long R = (b + RG - 1) / RG;
       c->lpr_log2 = lpr_log2;
@@ -438,6 +375,7 @@ bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, 
       c->n_row_boxes = n_row_boxes;
       c->keep = (pass == 0);
       c->rmax = pass == 0 ? (R <= 4 ? 4 : (R <= 8 ? 8 : 16)) : 32;
+      c->full = (b % RG == 0) && (R == c->rmax);
       c->box_bytes = static_cast<unsigned>(rows_pad * lpr * 16);
       c->stage_bytes = static_cast<unsigned>(stage);
       c->smem_bytes = stages * stage + extras_bytes(lpr, ve, bx, b, stages) + 128;
@@ -447,25 +385,32 @@ bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, 
   return false;
 }
 
-template <typename T, int RMAX, bool KEEP>
+template <typename T, int RMAX, bool KEEP, bool FULL>
 int launch_variant(abs_ctx* ctx, const CUtensorMap& tmap, const TiledParams& prm, dim3 grid, size_t smem,
                    cudaStream_t stream) {
-  auto kern = abs_stats_tiled_kernel<T, RMAX, KEEP>;
+  auto kern = abs_stats_tiled_kernel<T, RMAX, KEEP, FULL>;
   ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   kern<<<grid, kThreads, smem, stream>>>(tmap, prm);
   ABS_CUDA_TRY(ctx, cudaGetLastError());
   return ABS_OK;
 }
 
+template <typename T, bool FULL>
+int launch_full(abs_ctx* ctx, const TileChoice& c, const CUtensorMap& tmap, const TiledParams& prm, dim3 grid,
+                cudaStream_t stream) {
+  if (!c.keep) return launch_variant<T, 32, false, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
+  switch (c.rmax) {
+    case 4: return launch_variant<T, 4, true, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
+    case 8: return launch_variant<T, 8, true, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
+    default: return launch_variant<T, 16, true, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
+  }
+}
+
 template <typename T>
 int launch_typed(abs_ctx* ctx, const TileChoice& c, const CUtensorMap& tmap, const TiledParams& prm, dim3 grid,
                  cudaStream_t stream) {
-  if (!c.keep) return launch_variant<T, 32, false>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-  switch (c.rmax) {
-    case 4: return launch_variant<T, 4, true>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-    case 8: return launch_variant<T, 8, true>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-    default: return launch_variant<T, 16, true>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-  }
+  return c.full ? launch_full<T, true>(ctx, c, tmap, prm, grid, stream)
+                : launch_full<T, false>(ctx, c, tmap, prm, grid, stream);
 }
 
 }  // namespace
@@ -473,18 +418,17 @@ int launch_typed(abs_ctx* ctx, const TileChoice& c, const CUtensorMap& tmap, con
 int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   const int es = a.dtype == ABS_F32 ? 4 : 2;
   const int ve = 16 / es;
-  const unsigned long long row_b = static_cast<unsigned long long>(a.row_stride) * es;
-  const unsigned long long wrk_b = static_cast<unsigned long long>(a.M > 1 ? a.worker_stride : a.b * a.row_stride) * es;
-  if ((reinterpret_cast<uintptr_t>(a.G) & 15u) || (row_b & 15u) || (wrk_b & 15u)) return ABS_ERR_UNSUPPORTED;
-  if (a.b > kMaxFastRows || a.d > 0x7fff0000ll || a.M > 65535) return ABS_ERR_UNSUPPORTED;
-  if (row_b >= (1ull << 40) || wrk_b >= (1ull << 40)) return ABS_ERR_UNSUPPORTED;
-  EncodeTiledFn encode = encode_tiled_fn();
-  if (encode == nullptr) return ABS_ERR_UNSUPPORTED;
+  if (a.b > kMaxFastRows || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
 
   TileChoice c;
+  // two resident CTAs per SM with 32 KiB tile buffers and 8 rows per thread, or one CTA with 64 KiB
+  // buffers and 16 rows per thread
+  const int per_sm = ctx->tuning.stats_ctas_per_sm > 0 ? static_cast<int>(ctx->tuning.stats_ctas_per_sm) : 1;
   const size_t stage_max = ctx->tuning.stats_stage_kb > 0 ? static_cast<size_t>(ctx->tuning.stats_stage_kb) << 10
-                                                          : (64u << 10);
-  if (!choose_tile(a.b, ve, ctx->smem_optin, ctx->tuning.stats_stages, stage_max, &c)) return ABS_ERR_UNSUPPORTED;
+                                                          : (per_sm == 2 ? (32u << 10) : (64u << 10));
+  if (!choose_tile(a.b, ve, ctx->smem_optin, ctx->tuning.stats_stages, stage_max, per_sm == 2 ? 8 : 16, &c) &&
+      !choose_tile(a.b, ve, ctx->smem_optin, ctx->tuning.stats_stages, 64u << 10, 16, &c))
+    return ABS_ERR_UNSUPPORTED;
 
   const int lpr = 1 << c.lpr_log2;
   const long long box_cols = static_cast<long long>(lpr) * ve;
@@ -493,7 +437,7 @@ int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
 
   int ctas_per_sm = static_cast<int>(ctx->smem_optin / (c.smem_bytes + 1024));
   if (ctas_per_sm < 1) ctas_per_sm = 1;
-  if (ctas_per_sm > 2) ctas_per_sm = 2;
+  if (ctas_per_sm > 2 || (ctas_per_sm == 2 && c.rmax > 8)) ctas_per_sm = c.rmax > 8 ? 1 : 2;
   long long P = ctx->tuning.stats_ctas_per_worker > 0
                     ? ctx->tuning.stats_ctas_per_worker
                     : (static_cast<long long>(ctx->sm_count) * ctas_per_sm) / a.M;
@@ -506,16 +450,10 @@ int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
                      ctx->workspace_bytes);
 
   CUtensorMap tmap;
-  const cuuint64_t gdim[3] = {static_cast<cuuint64_t>(a.d), static_cast<cuuint64_t>(a.b), static_cast<cuuint64_t>(a.M)};
-  const cuuint64_t gstr[2] = {row_b, wrk_b};
-  const cuuint32_t box[3] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(c.box_rows), 1u};
-  const cuuint32_t estr[3] = {1u, 1u, 1u};
-  const CUresult r = encode(&tmap, a.dtype == ABS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                            3, const_cast<void*>(a.G), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS)
-    return set_error(ctx, ABS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r));
+  {
+    const int rc = encode_g_tensor_map(ctx, a, box_cols, c.box_rows, &tmap);
+    if (rc != ABS_OK) return rc;
+  }
 
   TiledParams prm;
   prm.b = a.b;
@@ -530,7 +468,7 @@ int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.stage_bytes = c.stage_bytes;
   prm.n_iters = n_iters;
   prm.P = static_cast<int>(P);
-  prm.flush_every = static_cast<int>(ctx->tuning.stats_flush_every > 0 ? ctx->tuning.stats_flush_every : 8);
+  prm.flush_every = static_cast<int>(ctx->tuning.stats_flush_every > 0 ? ctx->tuning.stats_flush_every : 64);
   prm.ws = static_cast<double*>(ctx->workspace);
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;

@@ -137,6 +137,29 @@ def test_tiled_and_generic_kernels_agree_and_are_deterministic(ctx):
     np.testing.assert_allclose(ga.cpu().numpy(), gg.cpu().numpy(), rtol=1e-6, atol=1e-6 * ga.abs().max().item())
 
 
+@pytest.mark.parametrize("M,b,d", [(1, 16, 9000), (2, 7, 3001), (3, 32, 5000), (1, 24, 700), (1, 2, 40)])
+def test_gram_and_tiled_kernels_agree_on_bf16(ctx, M, b, d):
+    """bf16 input with b <= 32 goes through the tensor-core Gram kernel; the tiled kernel must give
+    the same statistics (and both match the oracle) when the Gram kernel is switched off."""
+    G = make_G(70 + b, M, b, d + (-d) % 8, torch.bfloat16, sigma=2.0)
+    gram, gbar_g = run_gpu(ctx, G)
+    ctx.set_tuning("stats_no_gram", 1)
+    try:
+        tiled, gbar_t = run_gpu(ctx, G)
+    finally:
+        ctx.set_tuning("stats_no_gram", 0)
+    H = to_f64(G)
+    for m in range(M):
+        ref = orc.batch_test_stats(H[m])
+        check_record(gram[m], ref, 1e-3, b)
+        check_record(tiled[m], ref, 1e-3, b)
+        # the Gram kernel adds exact products: it is far inside the bf16 tolerance
+        for key in ("gbar_sq", "var_norm", "sum_sq"):
+            assert gram[m][key] == pytest.approx(ref[key], rel=1e-5)
+    np.testing.assert_allclose(gbar_g.cpu().numpy(), gbar_t.cpu().numpy(), rtol=1e-6,
+                               atol=1e-6 * gbar_t.abs().max().item())
+
+
 @pytest.mark.parametrize("key,value", [("stats_stages", 2), ("stats_stages", 6), ("stats_stage_kb", 16),
                                        ("stats_flush_every", 1), ("stats_ctas_per_worker", 3)])
 def test_tuning_knobs_do_not_change_the_result(ctx, key, value):
