@@ -75,6 +75,8 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_force_generic" (1 = always use the alignment-free kernel),
  * "stats_flush_every" (tiles between fp64 flushes of the per-row sums),
  * "stats_stage_kb" (upper bound on one tile buffer, 4..200 KiB),
+ * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
+ * cluster when b > 256),
  * "stats_no_gram" (1 = do not use the tensor-core Gram kernel for bf16, b <= 32),
  * "stats_ctas_per_sm" (1: one CTA per SM, 64 KiB buffers, up to 16 rows per
  * thread; 2: two CTAs per SM, 32 KiB buffers, up to 8 rows per thread).
@@ -110,7 +112,8 @@ typedef struct {
  *   stats_out    [M] records
  * G is read exactly once from HBM when its base address and both strides are
  * multiples of 16 bytes and b <= 4096 (bf16 input with b <= 32 goes through a
- * tensor-core Gram-matrix kernel, everything else through the tiled kernel);
+ * tensor-core Gram-matrix kernel, b > 256 through a kernel that splits the rows
+ * over a thread-block cluster, everything else through the tiled kernel);
  * otherwise an alignment-free kernel that reads it twice is used.  The result does not depend on which kernel ran beyond
  * floating-point rounding.  Accumulation: fp32 within a tile, fp64 across tiles;
  * the reduction order is fixed, so repeated calls give bit-identical records.

@@ -49,6 +49,8 @@ int run_stats(abs_ctx* ctx, const StatsLaunch& a) {
   int P = 0;
   int rc = ABS_ERR_UNSUPPORTED;
   if (!ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_gram) rc = launch_stats_gram(ctx, a, &P);
+  if (rc == ABS_ERR_UNSUPPORTED && !ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_cluster)
+    rc = launch_stats_cluster(ctx, a, &P);
   if (rc == ABS_ERR_UNSUPPORTED && !ctx->tuning.stats_force_generic) rc = launch_stats_tiled(ctx, a, &P);
   if (rc == ABS_ERR_UNSUPPORTED) rc = launch_stats_generic(ctx, a, &P);
   if (rc != ABS_OK) return rc;
@@ -140,6 +142,8 @@ extern "C" int abs_set_tuning(abs_ctx* ctx, const char* key, long long value) {
   } else if (strcmp(key, "stats_stage_kb") == 0) {
     if (value != 0 && (value < 4 || value > 200)) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_stage_kb must be 0 or 4..200");
     ctx->tuning.stats_stage_kb = value;
+  } else if (strcmp(key, "stats_no_cluster") == 0) {
+    ctx->tuning.stats_no_cluster = value ? 1 : 0;
   } else if (strcmp(key, "stats_no_gram") == 0) {
     ctx->tuning.stats_no_gram = value ? 1 : 0;
   } else if (strcmp(key, "stats_ctas_per_sm") == 0) {

@@ -24,6 +24,7 @@ struct Tuning {
   long long stats_stage_kb = 0;
   long long stats_ctas_per_sm = 0;
   long long stats_no_gram = 0;
+  long long stats_no_cluster = 0;
 };
 
 }  // namespace absk
@@ -75,7 +76,8 @@ struct StatsLaunch {
 // Returns ABS_OK, or ABS_ERR_UNSUPPORTED when the tiled kernel cannot take the call
 // (alignment, b too large); *P_out receives the number of partial records per worker.
 int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
-int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out);   // bf16, b <= 32
+int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // bf16, b <= 32
+int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out);   // 256 < b <= 4096
 int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
 int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P);
 

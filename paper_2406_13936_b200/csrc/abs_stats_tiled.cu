@@ -48,35 +48,6 @@ struct TiledParams {
   long long timeout_cycles;
 };
 
-// ---- element traits ------------------------------------------------------------------------
-template <typename T>
-struct Vec;
-template <>
-struct Vec<float> {
-  static constexpr int VE = 4;  // elements per 16-byte vector
-  static __device__ __forceinline__ void unpack(const uint4& v, float (&x)[4]) {
-    x[0] = __uint_as_float(v.x);
-    x[1] = __uint_as_float(v.y);
-    x[2] = __uint_as_float(v.z);
-    x[3] = __uint_as_float(v.w);
-  }
-};
-template <>
-struct Vec<__nv_bfloat16> {
-  static constexpr int VE = 8;
-  // a bfloat16 is the upper half of a binary32: widening is a shift / a mask
-  static __device__ __forceinline__ void unpack(const uint4& v, float (&x)[8]) {
-    x[0] = __uint_as_float(v.x << 16);
-    x[1] = __uint_as_float(v.x & 0xffff0000u);
-    x[2] = __uint_as_float(v.y << 16);
-    x[3] = __uint_as_float(v.y & 0xffff0000u);
-    x[4] = __uint_as_float(v.z << 16);
-    x[5] = __uint_as_float(v.z & 0xffff0000u);
-    x[6] = __uint_as_float(v.w << 16);
-    x[7] = __uint_as_float(v.w & 0xffff0000u);
-  }
-};
-
 // ---- the kernel ----------------------------------------------------------------------------
 // RMAX: upper bound on the rows a thread owns; KEEP: the rows stay in registers between the
 // sweeps; FULL: every thread owns exactly RMAX rows (no per-row predicates).  Variants with

@@ -160,6 +160,30 @@ def test_gram_and_tiled_kernels_agree_on_bf16(ctx, M, b, d):
                                atol=1e-6 * gbar_t.abs().max().item())
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("M,b,d", [(1, 512, 3000), (2, 700, 1300), (1, 1024, 2100), (1, 1500, 640), (1, 2048, 520),
+                                   (1, 3000, 200), (1, 4096, 264)])
+def test_cluster_and_tiled_kernels_agree(ctx, M, b, d, dtype):
+    """b > 256 splits the rows over a thread-block cluster; with that switched off the single-CTA
+    tiled kernel takes the call.  Both must match the oracle and each other."""
+    G = make_G(90 + b, M, b, d + (-d) % 8, dtype, sigma=1.5)
+    clus, gbar_c = run_gpu(ctx, G)
+    ctx.set_tuning("stats_no_cluster", 1)
+    try:
+        tiled, gbar_t = run_gpu(ctx, G)
+    finally:
+        ctx.set_tuning("stats_no_cluster", 0)
+    H = to_f64(G)
+    for m in range(M):
+        ref = orc.batch_test_stats(H[m])
+        check_record(clus[m], ref, TOL[dtype], b)
+        check_record(tiled[m], ref, TOL[dtype], b)
+    np.testing.assert_allclose(gbar_c.cpu().numpy(), gbar_t.cpu().numpy(), rtol=1e-6,
+                               atol=1e-6 * gbar_t.abs().max().item())
+    again, _ = run_gpu(ctx, G)
+    assert again == clus                                     # fixed reduction order
+
+
 @pytest.mark.parametrize("key,value", [("stats_stages", 2), ("stats_stages", 6), ("stats_stage_kb", 16),
                                        ("stats_flush_every", 1), ("stats_ctas_per_worker", 3)])
 def test_tuning_knobs_do_not_change_the_result(ctx, key, value):
