@@ -75,6 +75,7 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_force_generic" (1 = always use the alignment-free kernel),
  * "stats_flush_every" (tiles between fp64 flushes of the per-row sums),
  * "stats_stage_kb" (upper bound on one tile buffer, 4..200 KiB),
+ * "stats_cluster_rows" (target rows per CTA of the cluster kernel, 16..512),
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
  * cluster when b > 256),
  * "stats_no_gram" (1 = do not use the tensor-core Gram kernel for bf16, b <= 32),

@@ -25,6 +25,7 @@ struct Tuning {
   long long stats_ctas_per_sm = 0;
   long long stats_no_gram = 0;
   long long stats_no_cluster = 0;
+  long long stats_cluster_rows = 0;
 };
 
 }  // namespace absk

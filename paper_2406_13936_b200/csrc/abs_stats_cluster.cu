@@ -1,27 +1,29 @@
 // Cluster variant of the single-pass statistics kernel for large batches (256 < b <= 4096).
 //
 // A column strip with all b rows does not fit one SM's shared memory at a row width that the
-// memory system likes (>= 256 bytes), so the rows are split over a thread-block cluster of
-// C = 2, 4 or 8 CTAs: CTA `rank` holds rows [rank*RC, rank*RC + RC) of the strip, RC = ceil(b/C).
-// Each CTA sums its rows' columns, the per-CTA column sums (lpr*VE floats) are pushed into every
-// peer's shared memory (st.shared::cluster) and announced on the peer's mbarrier
-// (mbarrier.arrive.release.cluster); after that every CTA knows gbar for the strip and runs
-// the centred sweep on the rows it still holds in registers.  Eq. batch_grad / Eq. def_var as in
-// the tiled kernel; G is still read exactly once.
+// memory system likes (>= 256 bytes), and a CTA that touches a thousand far-apart rows per tile
+// runs into address-translation misses.  So the rows are split over a thread-block cluster of
+// C = 2, 4, 8 or 16 CTAs: CTA `rank` holds rows [rank*RC, rank*RC + RC) of the strip,
+// RC = ceil(b/C) <= 256.  Each CTA sums its rows' columns; the per-CTA column sums (lpr*VE
+// floats) are shipped to every peer with one bulk shared-to-shared copy that signals the peer's
+// mbarrier; after that every CTA knows gbar for the strip and runs the centred sweep on its rows
+// (Eq. batch_grad, Eq. def_var as in the tiled kernel).  G is still read exactly once.
 //
-// The mbarrier hand-shake, not the hardware cluster barrier, is used inside the loop because the
-// producer warp does not take part in it.  Waits are bounded like everywhere else.
-#include <cooperative_groups.h>
-
+// The loop is software pipelined: a step moves the rows of tile i from shared memory into
+// registers (so the tile buffer goes straight back to the loader), sends the column sums round
+// the cluster, and then finishes tile i-1 from a second register set, whose sums have had a
+// whole step to arrive.  Four exchange buffers / barriers are in flight.  There is no separate
+// loader warp: after the CTA-wide barrier that follows the register load, thread 0 re-arms the
+// buffer and issues the next TMA load into it.  All waits are bounded.
 #include "abs_pipeline.cuh"
 
 namespace absk {
 namespace {
 
-constexpr int kCW = 8;                         // consumer warps
-constexpr int kThreadsC = kCW * 32 + 32;
-constexpr int kMaxCluster = 8;
-constexpr int RMAXC = 16;                      // rows per thread kept in registers
+constexpr int kCW = 8;                         // warps
+constexpr int kThreadsC = kCW * 32;
+constexpr int kMaxCluster = 16;                // 16 needs the non-portable cluster size opt-in
+constexpr int kDepth = 4;                      // column-sum exchange buffers in flight (power of two)
 
 struct ClusterParams {
   long long b, d;
@@ -54,42 +56,23 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t ra
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
+// Copies `bytes` (a multiple of 16) from this CTA's shared memory into a peer's and adds them to
+// the transaction count of the peer's mbarrier.
+__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes,
+                                                  uint32_t mbar_cluster) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_cluster),
+      "r"(src_cta), "r"(bytes), "r"(mbar_cluster)
       : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile unsigned* abort_flag,
-                                                  long long limit) {
-  if (mbar_try_wait_cluster(bar, parity)) return true;
-  if (*abort_flag) return false;
-  const long long t0 = clock64();
-  while (!mbar_try_wait_cluster(bar, parity)) {
-    if (*abort_flag || clock64() - t0 > limit) {
-      *abort_flag = 1u;
-      return false;
-    }
-  }
-  return true;
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <typename T, bool FULL>
+// RMAX: rows per thread and register set (two sets alternate); FULL: every thread of every CTA
+// owns exactly RMAX rows, so the row loops need no predicates.
+template <typename T, int RMAX, bool FULL>
 __global__ void __launch_bounds__(kThreadsC, 1)
 abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const ClusterParams prm) {
   constexpr int VE = Vec<T>::VE;
@@ -107,137 +90,138 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
   const int S = prm.stages;
   const int lpr = 1 << prm.lpr_log2;
   const unsigned row_bytes = static_cast<unsigned>(lpr) * 16u;
-  const int cols = lpr * VE;                     // floats per strip row
+  const int cols = lpr * VE;                     // columns of a strip
 
   unsigned char* stage_mem = smem_raw;
   float* part = reinterpret_cast<float*>(stage_mem + static_cast<size_t>(S) * prm.stage_bytes);   // [2][8][cols]
-  float* xsum = part + 2 * kCW * cols;                                                             // [2][8][cols]
-  double* e_acc = reinterpret_cast<double*>(xsum + 2 * kMaxCluster * cols);                        // [RC]
+  float* xsum = part + 2 * kCW * cols;                                                             // [kDepth][16][cols]
+  double* e_acc = reinterpret_cast<double*>(xsum + kDepth * kMaxCluster * cols);                   // [RC]
   double* red = e_acc + RC;                                                                        // [16]
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(red + 2 * kCW);                 // full[S] empty[S] x[2]
-  volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + 2 * S + 2);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(red + 2 * kCW);                 // full[S] x[kDepth]
+  volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + S + kDepth);
 
   const uint32_t stage_u32 = smem_u32(stage_mem);
   const uint32_t full_u32 = smem_u32(bars);
-  const uint32_t empty_u32 = smem_u32(bars + S);
-  const uint32_t xbar_u32 = smem_u32(bars + 2 * S);
+  const uint32_t xbar_u32 = smem_u32(bars + S);
   const uint32_t xsum_u32 = smem_u32(xsum);
 
+  const long long n_mine = (prm.n_iters > cl) ? (prm.n_iters - cl + prm.n_clusters - 1) / prm.n_clusters : 0;
+
+  // Loads tile i of this cluster (rows of this CTA) into its ring buffer; thread 0 only.
+  auto issue_load = [&](long long i) {
+    const int s = static_cast<int>(i % S);
+    const uint32_t full = full_u32 + 8u * s;
+    mbar_expect_tx(full, prm.stage_bytes);
+    const long long x = (cl + i * prm.n_clusters) * cols;
+    const uint32_t dst0 = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes;
+    for (int rb = 0; rb < prm.n_row_boxes; ++rb)
+      tma_load_3d(dst0 + static_cast<uint32_t>(rb * prm.box_rows) * row_bytes, &tmap, static_cast<int>(x),
+                  row0 + rb * prm.box_rows, m, full);
+  };
+
   if (tid == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(full_u32 + 8u * s, 1);
-      mbar_init(empty_u32 + 8u * s, kCW);
-    }
-    mbar_init(xbar_u32, static_cast<uint32_t>(C * lpr));
-    mbar_init(xbar_u32 + 8u, static_cast<uint32_t>(C * lpr));
+    for (int s = 0; s < S; ++s) mbar_init(full_u32 + 8u * s, 1);
+    for (int q = 0; q < kDepth; ++q) mbar_init(xbar_u32 + 8u * q, 1);
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   for (int i = tid; i < RC; i += kThreadsC) e_acc[i] = 0.0;
   cluster_sync_all();      // every CTA's barriers exist before anybody signals them
+  if (tid == 0)
+    for (long long i = 0; i < S && i < n_mine; ++i) issue_load(i);
 
-  const long long n_mine = (prm.n_iters > cl) ? (prm.n_iters - cl + prm.n_clusters - 1) / prm.n_clusters : 0;
+  const int sub = lane >> prm.lpr_log2;          // sub-row-group within the warp
+  const int cv = lane & (lpr - 1);               // 16-byte column vector within the strip row
+  const int subs = 32 >> prm.lpr_log2;
+  const int RG = kCW * subs;                     // row groups
+  const int rg = warp * subs + sub;
+  const int n_rows_mine = (b_loc > rg) ? (b_loc - rg + RG - 1) / RG : 0;
+  const unsigned row_step = static_cast<unsigned>(RG) * row_bytes;
+  const uint32_t my_off = static_cast<uint32_t>(rg) * row_bytes + static_cast<uint32_t>(cv) * 16u;
+  const float inv_b = 1.0f / static_cast<float>(b);
+  const bool writes_mean = (rank == 0 && rg == 0);
+
   double vacc = 0.0, nacc = 0.0;
-
-  if (warp == kCW) {
-    if (lane == 0) {
-      for (long long i = 0; i < n_mine; ++i) {
-        const int s = static_cast<int>(i % S);
-        const long long use = i / S;
-        if (use > 0)
-          mbar_wait(empty_u32 + 8u * s, static_cast<uint32_t>((use - 1) & 1), abort_flag, prm.timeout_cycles);
-        const uint32_t full = full_u32 + 8u * s;
-        mbar_expect_tx(full, prm.stage_bytes);
-        const long long x = (cl + i * prm.n_clusters) * cols;
-        const uint32_t dst0 = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes;
-        for (int rb = 0; rb < prm.n_row_boxes; ++rb)
-          tma_load_3d(dst0 + static_cast<uint32_t>(rb * prm.box_rows) * row_bytes, &tmap, static_cast<int>(x),
-                      row0 + rb * prm.box_rows, m, full);
-      }
-      for (int s = 0; s < S && s < n_mine; ++s) {    // leave no copy in flight
-        const long long last_use = (n_mine - 1 - s) / S;
-        volatile unsigned ignore = 0u;
-        mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>(last_use & 1), &ignore, prm.timeout_cycles);
-      }
-    }
-  } else {
-    const int sub = lane >> prm.lpr_log2;
-    const int cv = lane & (lpr - 1);
-    const int subs = 32 >> prm.lpr_log2;
-    const int RG = kCW * subs;
-    const int rg = warp * subs + sub;
-    const int n_rows_mine = (b_loc > rg) ? (b_loc - rg + RG - 1) / RG : 0;
-    const unsigned row_step = static_cast<unsigned>(RG) * row_bytes;
-    const uint32_t my_off = static_cast<uint32_t>(rg) * row_bytes + static_cast<uint32_t>(cv) * 16u;
-    const float inv_b = 1.0f / static_cast<float>(b);
-    const bool writes_mean = (rank == 0 && rg == 0);
-
-    float e[RMAXC];
+  float e[RMAX];
 #pragma unroll
-    for (int k = 0; k < RMAXC; ++k) e[k] = 0.f;
-    int since_flush = 0;
+  for (int k = 0; k < RMAX; ++k) e[k] = 0.f;
+  int since_flush = 0;
 
-    for (long long i = 0; i < n_mine; ++i) {
+  uint4 va[RMAX], vb[RMAX];
+  auto step = [&](uint4 (&cur)[RMAX], uint4 (&prev)[RMAX], const long long i) {
+    if (i < n_mine) {
+      // ---- first half: tile i into registers, its column sums round the cluster ----
       const int s = static_cast<int>(i % S);
       mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>((i / S) & 1), abort_flag, prm.timeout_cycles);
       const uint32_t base = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + my_off;
-
-      uint4 v[RMAXC];
       float cs[VE];
 #pragma unroll
       for (int j = 0; j < VE; ++j) cs[j] = 0.f;
 #pragma unroll
-      for (int k = 0; k < RMAXC; ++k) {
+      for (int k = 0; k < RMAX; ++k) {
         if (FULL || k < n_rows_mine) {
-          v[k] = lds128(base + static_cast<uint32_t>(k) * row_step);
+          cur[k] = lds128(base + static_cast<uint32_t>(k) * row_step);
           float x[VE];
-          Vec<T>::unpack(v[k], x);
+          Vec<T>::unpack(cur[k], x);
 #pragma unroll
           for (int j = 0; j < VE; ++j) cs[j] += x[j];
         }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty_u32 + 8u * s);      // the tile is in registers now
       for (int off = lpr; off < 32; off <<= 1) {
 #pragma unroll
         for (int j = 0; j < VE; ++j) cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], off);
       }
-      const int par = static_cast<int>(i & 1);
-      float* buf = part + static_cast<size_t>(par) * (kCW * cols);
+      float* buf = part + static_cast<size_t>(i & 1) * (kCW * cols);
       if (sub == 0) {
 #pragma unroll
         for (int j = 0; j < VE; ++j) buf[warp * cols + cv * VE + j] = cs[j];
       }
-      named_bar_sync(1, kCW * 32);
-      // one thread per 16-byte column vector folds the 8 warps and tells every CTA of the cluster
-      if (tid < lpr) {
-        float tot[VE];
+      __syncthreads();     // partial sums visible; every thread has its rows in registers
+      if (tid == 0 && i + S < n_mine) issue_load(i + S);     // the buffer is free: refill it
+      // Warp 0 folds the 8 warps' sums (one lane per 16-byte column vector) into this CTA's own
+      // slot, arms its own barrier for the bytes the peers will send, and lane `peer` ships the
+      // slot to that peer with one bulk copy that signals the peer's barrier.
+      if (warp == 0) {
+        const int q = static_cast<int>(i & (kDepth - 1));
+        float* mine = xsum + (q * kMaxCluster + rank) * cols;
+        if (lane < lpr) {
+          float tot[VE];
 #pragma unroll
-        for (int j = 0; j < VE; ++j) tot[j] = 0.f;
-        for (int w = 0; w < kCW; ++w) {
+          for (int j = 0; j < VE; ++j) tot[j] = 0.f;
+          for (int w = 0; w < kCW; ++w) {
 #pragma unroll
-          for (int j = 0; j < VE; ++j) tot[j] += buf[w * cols + tid * VE + j];
+            for (int j = 0; j < VE; ++j) tot[j] += buf[w * cols + lane * VE + j];
+          }
+#pragma unroll
+          for (int j = 0; j < VE; ++j) mine[lane * VE + j] = tot[j];
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads what was just written
         }
-        const uint32_t slot = xsum_u32 + static_cast<uint32_t>(((par * kMaxCluster + rank) * cols + tid * VE) * 4);
-        for (int peer = 0; peer < C; ++peer) {
-          const uint32_t dst = map_to_rank(slot, static_cast<uint32_t>(peer));
-#pragma unroll
-          for (int j = 0; j < VE; j += 4) st_cluster_v4(dst + 4u * j, tot[j], tot[j + 1], tot[j + 2], tot[j + 3]);
-          mbar_arrive_remote(map_to_rank(xbar_u32 + 8u * par, static_cast<uint32_t>(peer)));
+        __syncwarp();
+        const uint32_t bytes = static_cast<uint32_t>(cols) * 4u;
+        if (lane == 0) mbar_expect_tx(xbar_u32 + 8u * q, static_cast<uint32_t>(C - 1) * bytes);
+        if (lane < C && lane != rank) {
+          const uint32_t slot = xsum_u32 + static_cast<uint32_t>((q * kMaxCluster + rank) * cols * 4);
+          bulk_copy_to_peer(map_to_rank(slot, static_cast<uint32_t>(lane)), slot, bytes,
+                            map_to_rank(xbar_u32 + 8u * q, static_cast<uint32_t>(lane)));
         }
       }
-      mbar_wait_cluster(xbar_u32 + 8u * par, static_cast<uint32_t>((i >> 1) & 1), abort_flag, prm.timeout_cycles);
-#pragma unroll
-      for (int j = 0; j < VE; ++j) cs[j] = 0.f;
-      for (int peer = 0; peer < C; ++peer) {
-        const float* src = xsum + (par * kMaxCluster + peer) * cols + cv * VE;
-#pragma unroll
-        for (int j = 0; j < VE; ++j) cs[j] += src[j];
-      }
+    }
+    if (i >= 1) {
+      // ---- second half: finish tile i-1 from the other register set ----
+      const long long t = i - 1;
+      const int q = static_cast<int>(t & (kDepth - 1));
+      mbar_wait(xbar_u32 + 8u * q, static_cast<uint32_t>((t / kDepth) & 1), abort_flag, prm.timeout_cycles);
       float g[VE];
 #pragma unroll
-      for (int j = 0; j < VE; ++j) g[j] = cs[j] * inv_b;
+      for (int j = 0; j < VE; ++j) g[j] = 0.f;
+      for (int peer = 0; peer < C; ++peer) {      // fixed order: the same mean in every CTA
+        const float* src = xsum + (q * kMaxCluster + peer) * cols + cv * VE;
+#pragma unroll
+        for (int j = 0; j < VE; ++j) g[j] += src[j];
+      }
+#pragma unroll
+      for (int j = 0; j < VE; ++j) g[j] *= inv_b;
 
       if (writes_mean) {
         float nl = 0.f;
@@ -245,7 +229,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
         for (int j = 0; j < VE; ++j) nl = fmaf(g[j], g[j], nl);
         nacc += static_cast<double>(nl);
         if (prm.gbar_out != nullptr) {
-          const long long col = ((cl + i * prm.n_clusters) * static_cast<long long>(lpr) + cv) * VE;
+          const long long col = ((cl + t * prm.n_clusters) * static_cast<long long>(lpr) + cv) * VE;
           float* dst = prm.gbar_out + static_cast<long long>(m) * prm.d + col;
           if (col + VE <= prm.d && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
 #pragma unroll
@@ -263,10 +247,10 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
 #pragma unroll
       for (int j = 0; j < VE; ++j) vl[j] = 0.f;
 #pragma unroll
-      for (int k = 0; k < RMAXC; ++k) {
+      for (int k = 0; k < RMAX; ++k) {
         if (FULL || k < n_rows_mine) {
           float x[VE];
-          Vec<T>::unpack(v[k], x);
+          Vec<T>::unpack(prev[k], x);
           float ea = 0.f, eb = 0.f;
 #pragma unroll
           for (int j = 0; j < VE; j += 2) {
@@ -286,10 +270,10 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
         for (int j = 0; j < VE; ++j) vs += vl[j];
         vacc += static_cast<double>(vs);
       }
-      if (++since_flush >= prm.flush_every || i + 1 == n_mine) {
+      if (++since_flush >= prm.flush_every || i == n_mine) {
         since_flush = 0;
 #pragma unroll
-        for (int k = 0; k < RMAXC; ++k) {
+        for (int k = 0; k < RMAX; ++k) {
           float ek = e[k];
           for (int off = 1; off < lpr; off <<= 1) ek += __shfl_xor_sync(0xffffffffu, ek, off);
           if (cv == 0 && (FULL || k < n_rows_mine)) e_acc[rg + k * RG] += static_cast<double>(ek);
@@ -297,12 +281,16 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
         }
       }
     }
+  };
+  for (long long i = 0; i <= n_mine; i += 2) {
+    step(va, vb, i);
+    if (i + 1 <= n_mine) step(vb, va, i + 1);
   }
 
   // ------------------------------ CTA epilogue ------------------------------
   vacc = warp_sum(vacc);
   nacc = warp_sum(nacc);
-  if (lane == 0 && warp < kCW) {
+  if (lane == 0) {
     red[warp] = vacc;
     red[kCW + warp] = nacc;
   }
@@ -325,11 +313,15 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
   cluster_sync_all();      // nobody leaves while a peer could still address its shared memory
 }
 
-template <typename T, bool FULL>
+template <typename T, int RMAX, bool FULL>
 int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams prm, const StatsLaunch& a, int C,
                            size_t smem, int* records_out) {
-  auto kern = abs_stats_cluster_kernel<T, FULL>;
+  auto kern = abs_stats_cluster_kernel<T, RMAX, FULL>;
   ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  if (C > 8 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    cudaGetLastError();
+    return ABS_ERR_UNSUPPORTED;
+  }
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -343,8 +335,13 @@ int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams 
   cfg.numAttrs = 1;
   cfg.gridDim = dim3(static_cast<unsigned>(C), 1, 1);
   int max_clusters = 0;
-  ABS_CUDA_TRY(ctx, cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg));
-  if (max_clusters < 1) return ABS_ERR_UNSUPPORTED;
+  const cudaError_t occ = cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg);
+  if (occ != cudaSuccess || max_clusters < 1) {
+    cudaGetLastError();
+    set_error(ctx, ABS_ERR_UNSUPPORTED, "a cluster of %d CTAs cannot be scheduled (%s, %d clusters)", C,
+              cudaGetErrorString(occ), max_clusters);
+    return ABS_ERR_UNSUPPORTED;
+  }
   long long n_clusters = ctx->tuning.stats_ctas_per_worker > 0 ? ctx->tuning.stats_ctas_per_worker
                                                                : static_cast<long long>(max_clusters) / a.M;
   if (n_clusters < 1) n_clusters = 1;
@@ -361,31 +358,28 @@ int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams 
   return ABS_OK;
 }
 
-}  // namespace
-
-// Takes the call when 256 < b <= 4096 and the tiled loads can address G.
-int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
-  if (a.b <= 256 || a.b > kMaxFastRows || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
+// One attempt with a given cluster size; ABS_ERR_UNSUPPORTED if that size cannot be used.
+int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   const int es = a.dtype == ABS_F32 ? 4 : 2;
   const int ve = 16 / es;
-  int C = 2;
-  while (C < kMaxCluster && (a.b + C - 1) / C > 256) C *= 2;
-  const int RC = static_cast<int>((a.b + C - 1) / C);             // <= 512
-  const int lpr_log2 = RC <= 256 ? 4 : 3;                          // 256-byte rows, 128-byte beyond 2048 rows
+  const int RC = static_cast<int>((a.b + C - 1) / C);
+  if (RC > 512) return ABS_ERR_UNSUPPORTED;
+  const int lpr_log2 = RC <= 256 ? 4 : 3;                          // 256-byte rows; 128-byte for 257..512 rows
   const int lpr = 1 << lpr_log2;
   const int subs = 32 / lpr;
   const int RG = kCW * subs;
-  if ((RC + RG - 1) / RG > RMAXC) return ABS_ERR_UNSUPPORTED;
+  const int R = (RC + RG - 1) / RG;                                // rows per thread, <= 16
+  const int rmax = R <= 8 ? 8 : 16;
   const int n_row_boxes = (RC + 255) / 256;
   const int box_rows = (RC + n_row_boxes - 1) / n_row_boxes;
   const int rows_pad = box_rows * n_row_boxes;
   const unsigned stage_bytes = static_cast<unsigned>(rows_pad) * lpr * 16u;
   const int cols = lpr * ve;
-  const size_t extras = static_cast<size_t>(2 * kCW * cols + 2 * kMaxCluster * cols) * 4 + static_cast<size_t>(RC) * 8 +
-                        2 * kCW * 8 + 16 + 128;
-  int stages = static_cast<int>(ctx->tuning.stats_stages > 0 ? ctx->tuning.stats_stages : 3);
-  while (stages > 2 && stages * static_cast<size_t>(stage_bytes) + extras + stages * 16 + 16 > ctx->smem_optin) --stages;
-  const size_t smem = stages * static_cast<size_t>(stage_bytes) + extras + stages * 16 + 16;
+  const size_t extras = static_cast<size_t>(2 * kCW * cols + kDepth * kMaxCluster * cols) * 4 +
+                        static_cast<size_t>(RC) * 8 + 2 * kCW * 8 + kDepth * 8 + 16 + 128;
+  int stages = static_cast<int>(ctx->tuning.stats_stages > 0 ? ctx->tuning.stats_stages : 4);
+  while (stages > 2 && stages * static_cast<size_t>(stage_bytes) + extras + stages * 8 > ctx->smem_optin) --stages;
+  const size_t smem = stages * static_cast<size_t>(stage_bytes) + extras + stages * 8;
   if (smem > ctx->smem_optin) return ABS_ERR_UNSUPPORTED;
 
   CUtensorMap tmap;
@@ -408,12 +402,32 @@ int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.timeout_cycles = 4000000000ll;
-  const bool full = (a.b % C == 0) && (RC % RG == 0) && (RC / RG == RMAXC);
-  if (a.dtype == ABS_F32)
-    return full ? launch_cluster_variant<float, true>(ctx, tmap, prm, a, C, smem, P_out)
-                : launch_cluster_variant<float, false>(ctx, tmap, prm, a, C, smem, P_out);
-  return full ? launch_cluster_variant<__nv_bfloat16, true>(ctx, tmap, prm, a, C, smem, P_out)
-              : launch_cluster_variant<__nv_bfloat16, false>(ctx, tmap, prm, a, C, smem, P_out);
+  const bool full = (a.b % C == 0) && (RC % RG == 0) && (RC / RG == rmax);
+#define ABS_CLUSTER_DISPATCH(T)                                                                          \
+  (rmax == 8 ? (full ? launch_cluster_variant<T, 8, true>(ctx, tmap, prm, a, C, smem, P_out)             \
+                     : launch_cluster_variant<T, 8, false>(ctx, tmap, prm, a, C, smem, P_out))           \
+             : (full ? launch_cluster_variant<T, 16, true>(ctx, tmap, prm, a, C, smem, P_out)            \
+                     : launch_cluster_variant<T, 16, false>(ctx, tmap, prm, a, C, smem, P_out)))
+  if (a.dtype == ABS_F32) return ABS_CLUSTER_DISPATCH(float);
+  return ABS_CLUSTER_DISPATCH(__nv_bfloat16);
+#undef ABS_CLUSTER_DISPATCH
+}
+
+}  // namespace
+
+// Takes the call when 256 < b <= 4096 and the tiled loads can address G.  Prefers the cluster
+// size that leaves each CTA at most 256 rows (64 KiB tiles of 256-byte rows); falls back to
+// smaller clusters when the larger one cannot be scheduled.
+int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
+  if (a.b <= 256 || a.b > kMaxFastRows || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
+  int C = 2;
+  const int want_rows = ctx->tuning.stats_cluster_rows > 0 ? static_cast<int>(ctx->tuning.stats_cluster_rows) : 256;
+  while (C < kMaxCluster && (a.b + C - 1) / C > want_rows) C *= 2;
+  for (; C >= 2; C /= 2) {
+    const int rc = try_cluster_size(ctx, a, C, P_out);
+    if (rc != ABS_ERR_UNSUPPORTED) return rc;
+  }
+  return ABS_ERR_UNSUPPORTED;
 }
 
 }  // namespace absk
