@@ -238,6 +238,31 @@ int local_shb_step(abs_ctx* ctx, float* X, float* Buf, const float* Gb, int M, l
 int replica_average(abs_ctx* ctx, float* X, int M, long long d, long long replica_stride,
                     void* stream);
 
+/* ---- producers and round drivers for the synthetic end-to-end problems ------------------ */
+
+/* Per-sample gradients of the logistic loss (Algorithm 1, "compute per-sample
+ * gradients"): row i of worker m is (sigmoid(a^T x^m) - y) a with a = A[idx[m][i]].
+ *   A [n][d] fp32 features, y [n] fp32 labels in {0,1}, idx [M][idx_stride] int32
+ *   sample indices (the first b of each row are used), X [M][d] parameters,
+ *   G [M][b][d] output (contiguous).                                              */
+int abs_logreg_grads(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
+                     const int* idx, long long idx_stride, const float* X, int M, long long b,
+                     float* G, void* stream);
+
+/* One communication round of local SGD on the logistic problem (Algorithm 2's
+ * structure, Algorithm 1's per-sample statistic evaluated once per round, Section
+ * 4.3): for h < H: per-sample gradients of batch idx[h] -> statistics and batch
+ * gradient -> local SGD step (the last one fused with the model averaging); then
+ * the batch-size update from the statistics of the last local step.
+ *   idx [H][M][idx_stride] int32;  b the current batch size (host value, equal to
+ *   *b_dev);  G_scratch [M][b][d], Gb_scratch [M][d], stats [M], T_out [M] or NULL;
+ *   b_dev device int64: holds b on entry and the next batch size afterwards.
+ * Only enqueues; read b_dev back before sizing the next round.                    */
+int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
+                     const int* idx, long long idx_stride, float* X, int M, int H, long long b,
+                     float lr, const abs_test_cfg* cfg, float* G_scratch, float* Gb_scratch,
+                     abs_stats* stats, long long* T_out, long long* b_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -55,6 +55,13 @@ EXPORTS = {
                                ctypes.c_void_p],
     "abs_next_batch": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(TestCfg),
                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_logreg_grads": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_longlong,
+                         ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
+                         ctypes.c_void_p, ctypes.c_void_p],
+    "abs_logreg_round": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_longlong,
+                         ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                         ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p, ctypes.c_void_p,
+                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "local_sgd_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
                        ctypes.c_longlong, ctypes.c_float, ctypes.c_int, ctypes.c_void_p],
     "local_adamw_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -218,6 +225,24 @@ class Context:
         self._check(self._lib.local_shb_step(self._h, _ptr(X2), _ptr(Buf), _ptr(Gb), M, d, stride, float(lr),
                                              float(momentum), float(weight_decay), int(bool(average_after)),
                                              _stream(stream)), "local_shb_step")
+
+    # ---- producers and rounds ----------------------------------------------------------------
+    def abs_logreg_grads(self, A, y, idx, X, b, G, stream=None):
+        """A [n, d], y [n], idx [M, >=b] int32, X [M, d] -> G [M, b, d] (all device tensors)."""
+        n, d = A.shape
+        M = X.shape[0]
+        self._check(self._lib.abs_logreg_grads(self._h, _ptr(A), _ptr(y), n, d, _ptr(idx), idx.stride(0), _ptr(X), M,
+                                               int(b), _ptr(G), _stream(stream)), "abs_logreg_grads")
+
+    def abs_logreg_round(self, A, y, idx, X, H, b, lr, cfg, G_scratch, Gb_scratch, stats, b_dev, T_out=None,
+                         stream=None):
+        """idx [H, M, >=b] int32 (contiguous in H and M); b_dev int64 device tensor holding b."""
+        n, d = A.shape
+        M = X.shape[0]
+        self._check(self._lib.abs_logreg_round(self._h, _ptr(A), _ptr(y), n, d, _ptr(idx), idx.stride(1), _ptr(X), M,
+                                               int(H), int(b), float(lr), ctypes.byref(cfg), _ptr(G_scratch),
+                                               _ptr(Gb_scratch), _ptr(stats), _ptr(T_out), _ptr(b_dev),
+                                               _stream(stream)), "abs_logreg_round")
 
     def replica_average(self, X, stream=None):
         X2, M, d, stride = self._replicas(X)
