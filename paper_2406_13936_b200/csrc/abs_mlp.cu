@@ -1,0 +1,331 @@
+// Producer for the MLP end-to-end problem: forward and backward pass of a three-layer ReLU
+// classifier with softmax cross-entropy for M workers at once, the batch gradients, and -- for
+// the batch-size test -- the per-sample gradients written out as rows (Algorithm 1, "compute
+// per-sample gradients"; they are outer products delta_l,i (x) h_{l-1},i).
+//
+// Parameter layout of one replica (flat, fp32): W1 [n1][n0], b1 [n1], W2 [n2][n1], b2 [n2],
+// W3 [n3][n2], b3 [n3], each W row-major [out][in].
+// Scratch layout per worker (floats): Xin [b][n0], H1 [b][n1], H2 [b][n2], D3 [b][n3], D2 [b][n2],
+// D1 [b][n1].
+#include "abs_internal.cuh"
+
+namespace absk {
+namespace {
+
+struct MlpShape {
+  int n0, n1, n2, n3;
+  long long oW1, ob1, oW2, ob2, oW3, ob3, d;      // offsets into the flat parameter vector
+  long long sX, sH1, sH2, sD3, sD2, sD1, per_worker;   // offsets into a worker's scratch
+};
+
+MlpShape make_shape(const int* dims, long long b) {
+  MlpShape s;
+  s.n0 = dims[0]; s.n1 = dims[1]; s.n2 = dims[2]; s.n3 = dims[3];
+  s.oW1 = 0;
+  s.ob1 = s.oW1 + static_cast<long long>(s.n1) * s.n0;
+  s.oW2 = s.ob1 + s.n1;
+  s.ob2 = s.oW2 + static_cast<long long>(s.n2) * s.n1;
+  s.oW3 = s.ob2 + s.n2;
+  s.ob3 = s.oW3 + static_cast<long long>(s.n3) * s.n2;
+  s.d = s.ob3 + s.n3;
+  s.sX = 0;
+  s.sH1 = s.sX + b * s.n0;
+  s.sH2 = s.sH1 + b * s.n1;
+  s.sD3 = s.sH2 + b * s.n2;
+  s.sD2 = s.sD3 + b * s.n3;
+  s.sD1 = s.sD2 + b * s.n2;
+  s.per_worker = (s.sD1 + b * s.n1 + 3) / 4 * 4;
+  return s;
+}
+
+// ---- batched fp32 GEMM with strided operands and a small epilogue ---------------------------
+struct GemmArgs {
+  const float* A; long long a_rs, a_cs, a_bs;    // element (r, k) at A[z*a_bs + r*a_rs + k*a_cs]
+  const float* B; long long b_rs, b_cs, b_bs;    // element (k, c)
+  float* C; long long c_rs, c_bs;                // element (r, c) at C[z*c_bs + r*c_rs + c]
+  const float* bias; long long bias_bs;          // per column (modes 1, 2)
+  const float* mask; long long mask_rs, mask_bs; // shape of C (mode 3)
+  int rows, cols, K;
+  float alpha;
+  int mode;   // 0: alpha*acc   1: relu(acc + bias)   2: acc + bias   3: acc where mask > 0, else 0
+};
+
+constexpr int kTile = 64, kTileK = 16;
+
+__global__ void __launch_bounds__(256)
+sgemm_kernel(const GemmArgs g) {
+  __shared__ float As[kTileK][kTile + 4];
+  __shared__ float Bs[kTileK][kTile + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int z = blockIdx.z;
+  const long long r0 = static_cast<long long>(blockIdx.y) * kTile, c0 = static_cast<long long>(blockIdx.x) * kTile;
+  const float* A = g.A + z * g.a_bs;
+  const float* B = g.B + z * g.b_bs;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < g.K; k0 += kTileK) {
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const int e = tid + t * 256;
+      int r, k;
+      if (g.a_cs == 1) { r = e / kTileK; k = e % kTileK; } else { r = e % kTile; k = e / kTile; }
+      const long long rr = r0 + r;
+      const int kk = k0 + k;
+      As[k][r] = (rr < g.rows && kk < g.K) ? A[rr * g.a_rs + kk * g.a_cs] : 0.f;
+      int c;
+      if (g.b_cs == 1) { k = e / kTile; c = e % kTile; } else { c = e / kTileK; k = e % kTileK; }
+      const long long cc = c0 + c;
+      const int kb = k0 + k;
+      Bs[k][c] = (cc < g.cols && kb < g.K) ? B[kb * g.b_rs + cc * g.b_cs] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kTileK; ++k) {
+      float a[4], bb[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[k][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bb[j] = Bs[k][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long long r = r0 + ty * 4 + i;
+    if (r >= g.rows) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const long long c = c0 + tx * 4 + j;
+      if (c >= g.cols) continue;
+      float v = acc[i][j];
+      if (g.mode == 0) v *= g.alpha;
+      else if (g.mode == 1) v = fmaxf(v + g.bias[z * g.bias_bs + c], 0.f);
+      else if (g.mode == 2) v += g.bias[z * g.bias_bs + c];
+      else v = g.mask[z * g.mask_bs + r * g.mask_rs + c] > 0.f ? v : 0.f;
+      g.C[z * g.c_bs + r * g.c_rs + c] = v;
+    }
+  }
+}
+
+void launch_gemm(const GemmArgs& g, int batch, cudaStream_t st) {
+  const dim3 grid((g.cols + kTile - 1) / kTile, (g.rows + kTile - 1) / kTile, batch);
+  sgemm_kernel<<<grid, 256, 0, st>>>(g);
+}
+
+// Xin[m][i][:] = inputs[idx[m][i]][:]
+__global__ void gather_rows_kernel(const float* __restrict__ inputs, const int* __restrict__ idx, long long idx_stride,
+                                   long long b, int n0, float* __restrict__ scratch, long long per_worker) {
+  const int m = blockIdx.y;
+  const long long i = blockIdx.x;
+  const float* src = inputs + static_cast<long long>(idx[m * idx_stride + i]) * n0;
+  float* dst = scratch + m * per_worker + i * n0;
+  for (int j = threadIdx.x; j < n0; j += blockDim.x) dst[j] = src[j];
+}
+
+// In place on the logits: D3[i][:] = softmax(logits_i) - onehot(label_i); one thread per sample.
+__global__ void softmax_delta_kernel(float* __restrict__ scratch, long long per_worker, long long off, long long b,
+                                     int n3, const int* __restrict__ labels, const int* __restrict__ idx,
+                                     long long idx_stride) {
+  const int m = blockIdx.y;
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= b) return;
+  float* z = scratch + m * per_worker + off + i * n3;
+  float mx = z[0];
+  for (int c = 1; c < n3; ++c) mx = fmaxf(mx, z[c]);
+  float sum = 0.f;
+  for (int c = 0; c < n3; ++c) {
+    const float e = expf(z[c] - mx);
+    z[c] = e;
+    sum += e;
+  }
+  const int label = labels[idx[m * idx_stride + i]];
+  for (int c = 0; c < n3; ++c) z[c] = z[c] / sum - (c == label ? 1.f : 0.f);
+}
+
+// db[o] = (1/b) sum_i D[i][o]; one thread per output unit and worker.
+__global__ void bias_grad_kernel(const float* __restrict__ scratch, long long per_worker, long long off, long long b,
+                                 int n, float* __restrict__ Gb, long long d, long long ob) {
+  const int m = blockIdx.y;
+  const int o = blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= n) return;
+  const float* D = scratch + m * per_worker + off;
+  float acc = 0.f;
+  for (long long i = 0; i < b; ++i) acc += D[i * n + o];
+  Gb[m * d + ob + o] = acc / static_cast<float>(b);
+}
+
+// Row i of G: the flat gradient of sample i of one worker.  One thread per parameter.
+__global__ void __launch_bounds__(256)
+per_sample_rows_kernel(const float* __restrict__ ws, const MlpShape s, float* __restrict__ G, long long row_stride) {
+  const long long i = blockIdx.y;
+  const long long j = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (j >= s.d) return;
+  float v;
+  if (j < s.ob1) {
+    const long long o = j / s.n0, k = j % s.n0;
+    v = ws[s.sD1 + i * s.n1 + o] * ws[s.sX + i * s.n0 + k];
+  } else if (j < s.oW2) {
+    v = ws[s.sD1 + i * s.n1 + (j - s.ob1)];
+  } else if (j < s.ob2) {
+    const long long o = (j - s.oW2) / s.n1, k = (j - s.oW2) % s.n1;
+    v = ws[s.sD2 + i * s.n2 + o] * ws[s.sH1 + i * s.n1 + k];
+  } else if (j < s.oW3) {
+    v = ws[s.sD2 + i * s.n2 + (j - s.ob2)];
+  } else if (j < s.ob3) {
+    const long long o = (j - s.oW3) / s.n2, k = (j - s.oW3) % s.n2;
+    v = ws[s.sD3 + i * s.n3 + o] * ws[s.sH2 + i * s.n2 + k];
+  } else {
+    v = ws[s.sD3 + i * s.n3 + (j - s.ob3)];
+  }
+  G[i * row_stride + j] = v;
+}
+
+int check_dims(abs_ctx* ctx, const int* dims) {
+  if (dims == nullptr) return set_error(ctx, ABS_ERR_INVALID_ARG, "dims is null");
+  for (int l = 0; l < 4; ++l)
+    if (dims[l] < 1) return set_error(ctx, ABS_ERR_INVALID_ARG, "layer widths must be >= 1");
+  return ABS_OK;
+}
+
+}  // namespace
+}  // namespace absk
+
+using namespace absk;
+
+extern "C" int abs_mlp_param_count(const int* dims, long long* out) {
+  if (dims == nullptr || out == nullptr) return ABS_ERR_INVALID_ARG;
+  *out = make_shape(dims, 1).d;
+  return ABS_OK;
+}
+
+extern "C" int abs_mlp_scratch_bytes(int M, long long b, const int* dims, size_t* out) {
+  if (dims == nullptr || out == nullptr || M < 1 || b < 1) return ABS_ERR_INVALID_ARG;
+  *out = static_cast<size_t>(M) * make_shape(dims, b).per_worker * sizeof(float);
+  return ABS_OK;
+}
+
+extern "C" int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* labels, long long n, const int* dims,
+                             const int* idx, long long idx_stride, const float* X, int M, long long b, float* Gb,
+                             void* scratch, size_t scratch_bytes, void* stream) {
+  if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
+  int rc = check_dims(ctx, dims);
+  if (rc != ABS_OK) return rc;
+  if (inputs == nullptr || labels == nullptr || idx == nullptr || X == nullptr || Gb == nullptr || scratch == nullptr)
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
+  if (n < 1 || M < 1 || M > 65535 || b < 1 || idx_stride < b)
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "need n, b >= 1, 1 <= M <= 65535 and idx_stride >= b");
+  const MlpShape s = make_shape(dims, b);
+  if (scratch_bytes < static_cast<size_t>(M) * s.per_worker * sizeof(float))
+    return set_error(ctx, ABS_ERR_WORKSPACE, "abs_mlp_grads needs %zu scratch bytes, got %zu",
+                     static_cast<size_t>(M) * s.per_worker * sizeof(float), scratch_bytes);
+  int prev = -1;
+  ABS_CUDA_TRY(ctx, cudaGetDevice(&prev));
+  if (prev != ctx->device) ABS_CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* ws = static_cast<float*>(scratch);
+  const long long pw = s.per_worker, d = s.d;
+  const float inv_b = 1.0f / static_cast<float>(b);
+
+  gather_rows_kernel<<<dim3(static_cast<unsigned>(b), M), 128, 0, st>>>(inputs, idx, idx_stride, b, s.n0, ws, pw);
+
+  GemmArgs g;
+  // forward: H1 = relu(Xin W1^T + b1), H2 = relu(H1 W2^T + b2), logits = H2 W3^T + b3
+  g = GemmArgs{ws + s.sX, s.n0, 1, pw, X + s.oW1, 1, s.n0, d, ws + s.sH1, s.n1, pw, X + s.ob1, d, nullptr, 0, 0,
+               static_cast<int>(b), s.n1, s.n0, 1.f, 1};
+  launch_gemm(g, M, st);
+  g = GemmArgs{ws + s.sH1, s.n1, 1, pw, X + s.oW2, 1, s.n1, d, ws + s.sH2, s.n2, pw, X + s.ob2, d, nullptr, 0, 0,
+               static_cast<int>(b), s.n2, s.n1, 1.f, 1};
+  launch_gemm(g, M, st);
+  g = GemmArgs{ws + s.sH2, s.n2, 1, pw, X + s.oW3, 1, s.n2, d, ws + s.sD3, s.n3, pw, X + s.ob3, d, nullptr, 0, 0,
+               static_cast<int>(b), s.n3, s.n2, 1.f, 2};
+  launch_gemm(g, M, st);
+  softmax_delta_kernel<<<dim3(static_cast<unsigned>((b + 127) / 128), M), 128, 0, st>>>(ws, pw, s.sD3, b, s.n3, labels,
+                                                                                       idx, idx_stride);
+  // backward: D2 = (D3 W3) .* (H2 > 0), D1 = (D2 W2) .* (H1 > 0)
+  g = GemmArgs{ws + s.sD3, s.n3, 1, pw, X + s.oW3, s.n2, 1, d, ws + s.sD2, s.n2, pw, nullptr, 0, ws + s.sH2, s.n2, pw,
+               static_cast<int>(b), s.n2, s.n3, 1.f, 3};
+  launch_gemm(g, M, st);
+  g = GemmArgs{ws + s.sD2, s.n2, 1, pw, X + s.oW2, s.n1, 1, d, ws + s.sD1, s.n1, pw, nullptr, 0, ws + s.sH1, s.n1, pw,
+               static_cast<int>(b), s.n1, s.n2, 1.f, 3};
+  launch_gemm(g, M, st);
+  // batch gradients: dW_l = (1/b) D_l^T H_{l-1}, db_l = (1/b) sum_i D_l[i]
+  g = GemmArgs{ws + s.sD3, 1, s.n3, pw, ws + s.sH2, s.n2, 1, pw, Gb + s.oW3, s.n2, d, nullptr, 0, nullptr, 0, 0,
+               s.n3, s.n2, static_cast<int>(b), inv_b, 0};
+  launch_gemm(g, M, st);
+  g = GemmArgs{ws + s.sD2, 1, s.n2, pw, ws + s.sH1, s.n1, 1, pw, Gb + s.oW2, s.n1, d, nullptr, 0, nullptr, 0, 0,
+               s.n2, s.n1, static_cast<int>(b), inv_b, 0};
+  launch_gemm(g, M, st);
+  g = GemmArgs{ws + s.sD1, 1, s.n1, pw, ws + s.sX, s.n0, 1, pw, Gb + s.oW1, s.n0, d, nullptr, 0, nullptr, 0, 0,
+               s.n1, s.n0, static_cast<int>(b), inv_b, 0};
+  launch_gemm(g, M, st);
+  bias_grad_kernel<<<dim3((s.n3 + 127) / 128, M), 128, 0, st>>>(ws, pw, s.sD3, b, s.n3, Gb, d, s.ob3);
+  bias_grad_kernel<<<dim3((s.n2 + 127) / 128, M), 128, 0, st>>>(ws, pw, s.sD2, b, s.n2, Gb, d, s.ob2);
+  bias_grad_kernel<<<dim3((s.n1 + 127) / 128, M), 128, 0, st>>>(ws, pw, s.sD1, b, s.n1, Gb, d, s.ob1);
+  const cudaError_t e = cudaGetLastError();
+  if (prev != ctx->device) cudaSetDevice(prev);
+  if (e != cudaSuccess) return set_error(ctx, ABS_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return ABS_OK;
+}
+
+extern "C" int abs_mlp_per_sample(abs_ctx* ctx, const int* dims, long long b, int worker, const void* scratch, float* G,
+                                  long long row_stride, void* stream) {
+  if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
+  int rc = check_dims(ctx, dims);
+  if (rc != ABS_OK) return rc;
+  const MlpShape s = make_shape(dims, b);
+  if (scratch == nullptr || G == nullptr || b < 1 || b > 65535 || worker < 0 || row_stride < s.d)
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "need scratch, G, 1 <= b <= 65535, worker >= 0, row_stride >= d");
+  int prev = -1;
+  ABS_CUDA_TRY(ctx, cudaGetDevice(&prev));
+  if (prev != ctx->device) ABS_CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+  const float* ws = static_cast<const float*>(scratch) + static_cast<long long>(worker) * s.per_worker;
+  const dim3 grid(static_cast<unsigned>((s.d + 255) / 256), static_cast<unsigned>(b));
+  per_sample_rows_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(ws, s, G, row_stride);
+  const cudaError_t e = cudaGetLastError();
+  if (prev != ctx->device) cudaSetDevice(prev);
+  if (e != cudaSuccess) return set_error(ctx, ABS_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return ABS_OK;
+}
+
+// One communication round of local SGD on the MLP problem (Algorithm 2's structure, the
+// per-sample statistic of Algorithm 1 once per round on the last local step, one worker's
+// per-sample gradients materialised at a time).
+extern "C" int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* labels, long long n, const int* dims,
+                             const int* idx, long long idx_stride, float* X, int M, int H, long long b, float lr,
+                             const abs_test_cfg* cfg, void* scratch, size_t scratch_bytes, float* G_scratch,
+                             long long g_row_stride, float* Gb_scratch, abs_stats* stats, long long* T_out,
+                             long long* b_dev, void* stream) {
+  if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
+  if (cfg == nullptr || G_scratch == nullptr || Gb_scratch == nullptr || stats == nullptr || b_dev == nullptr)
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
+  if (H < 1 || b < 2) return set_error(ctx, ABS_ERR_INVALID_ARG, "need H >= 1 and b >= 2");
+  int rc = check_dims(ctx, dims);
+  if (rc != ABS_OK) return rc;
+  const long long d = make_shape(dims, b).d;
+  for (int h = 0; h < H; ++h) {
+    const int* idx_h = idx + static_cast<long long>(h) * M * idx_stride;
+    rc = abs_mlp_grads(ctx, inputs, labels, n, dims, idx_h, idx_stride, X, M, b, Gb_scratch, scratch, scratch_bytes,
+                       stream);
+    if (rc != ABS_OK) return rc;
+    if (h == H - 1) {
+      for (int m = 0; m < M; ++m) {
+        rc = abs_mlp_per_sample(ctx, dims, b, m, scratch, G_scratch, g_row_stride, stream);
+        if (rc != ABS_OK) return rc;
+        rc = abs_test_stats(ctx, G_scratch, ABS_F32, 1, b, d, g_row_stride, b * g_row_stride, nullptr, stats + m,
+                            stream);
+        if (rc != ABS_OK) return rc;
+      }
+    }
+    rc = local_sgd_step(ctx, X, Gb_scratch, M, d, d, lr, h == H - 1 ? 1 : 0, stream);
+    if (rc != ABS_OK) return rc;
+  }
+  return abs_next_batch(ctx, stats, M, cfg, b_dev, T_out, b_dev, stream);
+}
