@@ -263,6 +263,39 @@ int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, long long n, 
                      float lr, const abs_test_cfg* cfg, float* G_scratch, float* Gb_scratch,
                      abs_stats* stats, long long* T_out, long long* b_dev, void* stream);
 
+/* Three-layer ReLU MLP with softmax cross-entropy (the second synthetic problem).
+ * dims = {n0, n1, n2, n3} layer widths.  One replica's parameters are a flat fp32
+ * vector W1 [n1][n0], b1 [n1], W2 [n2][n1], b2 [n2], W3 [n3][n2], b3 [n3] (each W
+ * row-major [out][in]); abs_mlp_param_count gives its length d.                    */
+int abs_mlp_param_count(const int* dims, long long* out);
+/* Bytes of scratch abs_mlp_grads needs for M workers and batch size b. */
+int abs_mlp_scratch_bytes(int M, long long b, const int* dims, size_t* out);
+
+/* Forward and backward pass of all M workers on their batches (Algorithm 2,
+ * "compute the local batch gradient"): writes the batch gradients Gb [M][d] and
+ * leaves activations and deltas in `scratch` (device, caller-owned) for
+ * abs_mlp_per_sample.  inputs [n][n0] fp32, labels [n] int32, idx [M][idx_stride]
+ * int32 sample indices (first b used), X [M][d] parameters (replica stride d).     */
+int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* labels, long long n, const int* dims,
+                  const int* idx, long long idx_stride, const float* X, int M, long long b,
+                  float* Gb, void* scratch, size_t scratch_bytes, void* stream);
+
+/* Per-sample gradients of one worker as rows G [b][row_stride] (row_stride >= d; a
+ * multiple of 4 keeps the rows 16-byte aligned for the fast statistics kernels),
+ * from the scratch a preceding abs_mlp_grads call with the same b filled
+ * (Algorithm 1, "compute per-sample gradients").  b <= 65535.                       */
+int abs_mlp_per_sample(abs_ctx* ctx, const int* dims, long long b, int worker, const void* scratch,
+                       float* G, long long row_stride, void* stream);
+
+/* One communication round of local SGD on the MLP problem, as abs_logreg_round; the
+ * per-sample gradients are materialised for one worker at a time in G_scratch
+ * [b][g_row_stride] at the last local step.  Gb_scratch [M][d].                     */
+int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* labels, long long n, const int* dims,
+                  const int* idx, long long idx_stride, float* X, int M, int H, long long b, float lr,
+                  const abs_test_cfg* cfg, void* scratch, size_t scratch_bytes, float* G_scratch,
+                  long long g_row_stride, float* Gb_scratch, abs_stats* stats, long long* T_out,
+                  long long* b_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

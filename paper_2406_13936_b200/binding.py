@@ -62,6 +62,19 @@ EXPORTS = {
                          ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                          ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p, ctypes.c_void_p,
                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_mlp_param_count": [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_longlong)],
+    "abs_mlp_scratch_bytes": [ctypes.c_int, ctypes.c_longlong, ctypes.POINTER(ctypes.c_int),
+                              ctypes.POINTER(ctypes.c_size_t)],
+    "abs_mlp_grads": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
+                      ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int,
+                      ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p],
+    "abs_mlp_per_sample": [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.c_longlong, ctypes.c_int,
+                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p],
+    "abs_mlp_round": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
+                      ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int,
+                      ctypes.c_int, ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p,
+                      ctypes.c_size_t, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p,
+                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "local_sgd_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
                        ctypes.c_longlong, ctypes.c_float, ctypes.c_int, ctypes.c_void_p],
     "local_adamw_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -243,6 +256,41 @@ class Context:
                                                int(H), int(b), float(lr), ctypes.byref(cfg), _ptr(G_scratch),
                                                _ptr(Gb_scratch), _ptr(stats), _ptr(T_out), _ptr(b_dev),
                                                _stream(stream)), "abs_logreg_round")
+
+    def mlp_param_count(self, dims):
+        out = ctypes.c_longlong()
+        self._check(self._lib.abs_mlp_param_count((ctypes.c_int * 4)(*dims), ctypes.byref(out)), "abs_mlp_param_count")
+        return out.value
+
+    def mlp_scratch(self, M, b, dims):
+        """Device scratch tensor (uint8) large enough for abs_mlp_grads with M workers and batch size b."""
+        out = ctypes.c_size_t()
+        self._check(self._lib.abs_mlp_scratch_bytes(int(M), int(b), (ctypes.c_int * 4)(*dims), ctypes.byref(out)),
+                    "abs_mlp_scratch_bytes")
+        return torch.empty(out.value, dtype=torch.uint8, device="cuda:%d" % self.device)
+
+    def abs_mlp_grads(self, inputs_, labels, dims, idx, X, b, Gb, scratch, stream=None):
+        n = inputs_.shape[0]
+        M = X.shape[0]
+        self._check(self._lib.abs_mlp_grads(self._h, _ptr(inputs_), _ptr(labels), n, (ctypes.c_int * 4)(*dims),
+                                            _ptr(idx), idx.stride(0), _ptr(X), M, int(b), _ptr(Gb), _ptr(scratch),
+                                            scratch.numel(), _stream(stream)), "abs_mlp_grads")
+
+    def abs_mlp_per_sample(self, dims, b, worker, scratch, G, stream=None):
+        """G: [b, row_stride] device tensor view with stride(0) >= d."""
+        self._check(self._lib.abs_mlp_per_sample(self._h, (ctypes.c_int * 4)(*dims), int(b), int(worker),
+                                                 _ptr(scratch), _ptr(G), G.stride(0), _stream(stream)),
+                    "abs_mlp_per_sample")
+
+    def abs_mlp_round(self, inputs_, labels, dims, idx, X, H, b, lr, cfg, scratch, G_scratch, g_row_stride,
+                      Gb_scratch, stats, b_dev, T_out=None, stream=None):
+        n = inputs_.shape[0]
+        M = X.shape[0]
+        self._check(self._lib.abs_mlp_round(self._h, _ptr(inputs_), _ptr(labels), n, (ctypes.c_int * 4)(*dims),
+                                            _ptr(idx), idx.stride(1), _ptr(X), M, int(H), int(b), float(lr),
+                                            ctypes.byref(cfg), _ptr(scratch), scratch.numel(), _ptr(G_scratch),
+                                            int(g_row_stride), _ptr(Gb_scratch), _ptr(stats), _ptr(T_out),
+                                            _ptr(b_dev), _stream(stream)), "abs_mlp_round")
 
     def replica_average(self, X, stream=None):
         X2, M, d, stride = self._replicas(X)

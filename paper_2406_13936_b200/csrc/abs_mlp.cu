@@ -61,13 +61,21 @@ sgemm_kernel(const GemmArgs g) {
   const long long r0 = static_cast<long long>(blockIdx.y) * kTile, c0 = static_cast<long long>(blockIdx.x) * kTile;
   const float* A = g.A + z * g.a_bs;
   const float* B = g.B + z * g.b_bs;
-  float acc[4][4];
+  // fp32 products are summed in fp32 over one 16-deep slice and the slices in fp64: the rounding
+  // error of a long dot product then stays near one fp32 ulp, which the 1e-6 parity bound on the
+  // parameters needs
+  double dacc[4][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int j = 0; j < 4; ++j) dacc[i][j] = 0.0;
 
   for (int k0 = 0; k0 < g.K; k0 += kTileK) {
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 #pragma unroll
     for (int t = 0; t < 4; ++t) {
       const int e = tid + t * 256;
@@ -95,6 +103,10 @@ sgemm_kernel(const GemmArgs g) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
     }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dacc[i][j] += static_cast<double>(acc[i][j]);
     __syncthreads();
   }
 #pragma unroll
@@ -105,10 +117,10 @@ sgemm_kernel(const GemmArgs g) {
     for (int j = 0; j < 4; ++j) {
       const long long c = c0 + tx * 4 + j;
       if (c >= g.cols) continue;
-      float v = acc[i][j];
-      if (g.mode == 0) v *= g.alpha;
-      else if (g.mode == 1) v = fmaxf(v + g.bias[z * g.bias_bs + c], 0.f);
-      else if (g.mode == 2) v += g.bias[z * g.bias_bs + c];
+      float v = static_cast<float>(g.mode == 0 ? dacc[i][j] * static_cast<double>(g.alpha) : dacc[i][j]);
+      if (g.mode == 0) {}
+      else if (g.mode == 1) v = fmaxf(static_cast<float>(dacc[i][j] + g.bias[z * g.bias_bs + c]), 0.f);
+      else if (g.mode == 2) v = static_cast<float>(dacc[i][j] + g.bias[z * g.bias_bs + c]);
       else v = g.mask[z * g.mask_bs + r * g.mask_rs + c] > 0.f ? v : 0.f;
       g.C[z * g.c_bs + r * g.c_rs + c] = v;
     }
@@ -157,9 +169,9 @@ __global__ void bias_grad_kernel(const float* __restrict__ scratch, long long pe
   const int o = blockIdx.x * blockDim.x + threadIdx.x;
   if (o >= n) return;
   const float* D = scratch + m * per_worker + off;
-  float acc = 0.f;
-  for (long long i = 0; i < b; ++i) acc += D[i * n + o];
-  Gb[m * d + ob + o] = acc / static_cast<float>(b);
+  double acc = 0.0;
+  for (long long i = 0; i < b; ++i) acc += static_cast<double>(D[i * n + o]);
+  Gb[m * d + ob + o] = static_cast<float>(acc / static_cast<double>(b));
 }
 
 // Row i of G: the flat gradient of sample i of one worker.  One thread per parameter.

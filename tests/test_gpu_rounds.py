@@ -109,3 +109,126 @@ def test_end_to_end_logistic_rounds(ctx, rounds):
     assert all(x <= y_ for x, y_ in zip(history, history[1:]))
     assert logistic_loss(An, yn, f64(X)[0]) < 0.8 * loss0
     assert torch.equal(X[0], X[M - 1])              # replicas agree after the averaging
+
+
+# ------------------------------------------------------------------ MLP producer and rounds
+def mlp_problem(seed, n, dims, M, device="cuda"):
+    inp, lab = inputs.gaussian_mixture(seed, n, dim=dims[0], classes=dims[3], device=device)
+    x0 = inputs.mlp_init(seed + 1, dims, device=device)
+    X = x0.unsqueeze(0).repeat(M, 1).contiguous()
+    return inp, lab, X
+
+
+@pytest.mark.parametrize("dims,M,b", [((6, 5, 4, 3), 2, 4), ((20, 33, 17, 7), 3, 9), ((70, 130, 65, 10), 2, 67),
+                                      ((784, 1024, 1024, 10), 1, 3)])
+def test_mlp_batch_and_per_sample_gradients(ctx, dims, M, b):
+    n = 300
+    inp, lab, X = mlp_problem(5, n, dims, M)
+    X += 0.05 * torch.randn(X.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(9))  # distinct replicas, non-zero biases
+    d = ctx.mlp_param_count(dims)
+    assert d == orc.mlp_param_count(dims)
+    idx = inputs.batch_indices(6, (M, b + 2), n, device="cuda")
+    scratch = ctx.mlp_scratch(M, b, dims)
+    Gb = torch.empty((M, d), device="cuda")
+    ctx.abs_mlp_grads(inp, lab, dims, idx, X, b, Gb, scratch)
+    stride = (d + 3) // 4 * 4
+    G = torch.zeros((b, stride), device="cuda")
+    In, inp_n, lab_n = idx.cpu().numpy(), f64(inp), lab.cpu().numpy()
+    for m in range(M):
+        ctx.abs_mlp_per_sample(dims, b, m, scratch, G)
+        rows = In[m, :b]
+        ref = orc.mlp_per_sample_grads(inp_n[rows], lab_n[rows], f64(X[m]), dims)
+        got = f64(G[:, :d])
+        assert np.abs(got - ref).max() <= 1e-5 * np.abs(ref).max()
+        ref_b = orc.batch_mean(ref)
+        assert np.abs(f64(Gb[m]) - ref_b).max() <= 1e-5 * np.abs(ref_b).max()
+        assert torch.all(G[:, d:] == 0)          # the padding columns are left alone
+
+
+def run_mlp_rounds(ctx, dims, n, M, H, lr, b, b_max, rounds, check_rounds, theta=0.5, nu=0.5, seed=5):
+    """Runs `rounds` rounds on the GPU; the first `check_rounds` are compared with the oracle."""
+    inp, lab, X = mlp_problem(seed, n, dims, M)
+    d = ctx.mlp_param_count(dims)
+    stride = (d + 3) // 4 * 4
+    idx = inputs.batch_indices(seed + 7, (rounds, H, M, b_max), n, device="cuda")
+    scratch = ctx.mlp_scratch(M, b_max, dims)
+    G = torch.empty((b_max, stride), device="cuda")
+    Gb = torch.empty((M, d), device="cuda")
+    stats = ctx.new_stats(M)
+    T_out = torch.zeros(M, dtype=torch.int64, device="cuda")
+    b_dev = torch.tensor([b], dtype=torch.int64, device="cuda")
+    cfg = pkg.make_test_cfg("aug_ip", b_max, theta=theta, nu=nu)
+    inp_n, lab_n = (f64(inp), lab.cpu().numpy()) if check_rounds else (None, None)
+    history = [b]
+    for k in range(rounds):
+        X0 = f64(X) if k < check_rounds else None
+        ctx.abs_mlp_round(inp, lab, dims, idx[k], X, H, b, lr, cfg, scratch, G, stride, Gb, stats, b_dev, T_out)
+        torch.cuda.synchronize()
+        recs = pkg.stats_to_dicts(stats)
+        assert all(r["status"] == 0 and r["rows"] == b for r in recs)
+        if k < check_rounds:
+            In = idx[k].cpu().numpy()
+
+            def grads(m, h, x, b=b, In=In):
+                rows = In[h, m, :b]
+                return orc.mlp_per_sample_grads(inp_n[rows], lab_n[rows], x, dims)
+            Xr, b_ref, T_ref, st_ref = orc.local_round(X0, grads, H, lr, b, b_max, "aug_ip", theta=theta, nu=nu)
+            params_close(X, Xr)
+            for m in range(M):
+                # the producers differ by fp32 rounding, so the statistics of the two pipelines agree
+                # to a few 1e-6; parity on identical inputs is covered by test_gpu_stats
+                for key in ("gbar_sq", "var_norm", "var_ip", "var_orth"):
+                    assert recs[m][key] == pytest.approx(st_ref[m][key], rel=2e-4)
+                N = st_ref[m]["gbar_sq"]
+                ratios = [st_ref[m]["var_ip"] / (theta ** 2 * N * N), st_ref[m]["var_orth"] / (nu ** 2 * N)]
+                if not any(near_integer(r, 1e-3) for r in ratios):
+                    assert T_out[m].item() == T_ref[m]
+            if T_out.tolist() == T_ref:
+                assert int(b_dev.item()) == b_ref
+        b_new = int(b_dev.item())
+        assert b <= b_new <= b_max
+        b = b_new
+        history.append(b)
+    return X, history, (inp, lab)
+
+
+def test_mlp_rounds_small_network_teacher_forced(ctx):
+    X, history, _ = run_mlp_rounds(ctx, (64, 48, 32, 10), n=4096, M=8, H=4, lr=0.05, b=8, b_max=512, rounds=12,
+                                   check_rounds=12)
+    assert history[-1] > history[0]
+    assert torch.equal(X[0], X[7])
+
+
+def test_mlp_rounds_full_network_first_rounds(ctx):
+    # the 784-1024-1024-10 classifier with two workers: the oracle is too slow for more
+    run_mlp_rounds(ctx, (784, 1024, 1024, 10), n=8192, M=2, H=4, lr=0.01, b=32, b_max=4096, rounds=2, check_rounds=2)
+
+
+def mlp_loss(ctx, inp, lab, x, dims):
+    """Mean cross-entropy on the first 4096 samples, evaluated with torch (test-side check only)."""
+    a = inp[:4096]
+    off = 0
+    for l in range(3):
+        nin, nout = dims[l], dims[l + 1]
+        W = x[off:off + nin * nout].view(nout, nin)
+        off += nin * nout
+        bias = x[off:off + nout]
+        off += nout
+        a = a @ W.t() + bias
+        if l < 2:
+            a = torch.relu(a)
+    return torch.nn.functional.cross_entropy(a, lab[:4096].long()).item()
+
+
+def test_end_to_end_mlp_200_rounds(ctx):
+    # 784-1024-1024-10, n = 1,048,576, M=8, H=4, augmented inner-product test, b from 32, cap 4096
+    dims = (784, 1024, 1024, 10)
+    inp, lab, X0 = mlp_problem(5, 1_048_576, dims, 1)
+    loss0 = mlp_loss(ctx, inp, lab, X0[0], dims)
+    del inp, lab, X0
+    X, history, (inp, lab) = run_mlp_rounds(ctx, dims, n=1_048_576, M=8, H=4, lr=0.01, b=32, b_max=4096, rounds=200,
+                                            check_rounds=0)
+    assert all(x <= y_ for x, y_ in zip(history, history[1:]))
+    assert history[-1] > history[0]
+    assert torch.equal(X[0], X[7])
+    assert mlp_loss(ctx, inp, lab, X[0], dims) < 0.5 * loss0
