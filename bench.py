@@ -205,7 +205,58 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
                                  frac_of_peak=gbs / peak)
         del G
         torch.cuda.empty_cache()
+    # fp32 statistics at the large-batch end of the sweep (rows split over a thread-block cluster)
+    if torch.cuda.mem_get_info()[0] > 60e9:
+        G = inputs.gaussian_rows(2, 1, 1024, 11_200_000, 1.0, device="cuda")
+        stats = ctx.new_stats(1)
+        sec = time_steps(torch, lambda i: ctx.abs_test_stats(G, stats), 5, 3)
+        gbs = G.numel() * 4 / sec / 1e9
+        out["stats_f32_b1024"] = dict(workload="G fp32 [1, 1024, 11,200,000]", ms=sec * 1e3, GBps=gbs,
+                                      frac_of_peak=gbs / peak)
+        del G
+        torch.cuda.empty_cache()
+    out["rounds_logreg"] = end_to_end_rounds(torch, pkg, inputs, ctx, "logreg")
+    out["rounds_mlp"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp")
     return out
+
+
+def end_to_end_rounds(torch, pkg, inputs, ctx, which):
+    """rounds/s of the two end-to-end configurations (producer + statistics + local SGD + averaging +
+    batch-size update per round; the batch size is read back once per round to size the next one)."""
+    if which == "logreg":
+        n, d, M, H, lr, b, b_max, rounds = 65536, 256, 4, 8, 0.1, 16, 1024, 50
+        A, y = inputs.logreg_dataset(1, n, d, device="cuda")
+        cfg = pkg.make_test_cfg("norm", b_max, eta=0.5)
+        X = torch.zeros((M, d), device="cuda")
+        G = torch.empty((M, b_max, d), device="cuda")
+    else:
+        dims = (784, 1024, 1024, 10)
+        n, M, H, lr, b, b_max, rounds = 1_048_576, 8, 4, 0.01, 32, 4096, 200
+        inp, lab = inputs.gaussian_mixture(5, n, dim=dims[0], classes=dims[3], device="cuda")
+        d = ctx.mlp_param_count(dims)
+        X = inputs.mlp_init(6, dims, device="cuda").unsqueeze(0).repeat(M, 1).contiguous()
+        cfg = pkg.make_test_cfg("aug_ip", b_max, theta=0.5, nu=0.5)
+        stride = (d + 3) // 4 * 4
+        scratch = ctx.mlp_scratch(M, b_max, dims)
+        G = torch.empty((b_max, stride), device="cuda")
+    idx = inputs.batch_indices(11, (rounds, H, M, b_max), n, device="cuda")
+    Gb = torch.empty((M, d), device="cuda")
+    stats = ctx.new_stats(M)
+    b_dev = torch.tensor([b], dtype=torch.int64, device="cuda")
+    history = [b]
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for k in range(rounds):
+        if which == "logreg":
+            ctx.abs_logreg_round(A, y, idx[k], X, H, b, lr, cfg, G, Gb, stats, b_dev)
+        else:
+            ctx.abs_mlp_round(inp, lab, dims, idx[k], X, H, b, lr, cfg, scratch, G, stride, Gb, stats, b_dev)
+        b = int(b_dev.item())          # one 8-byte read-back per round
+        history.append(b)
+    torch.cuda.synchronize()
+    sec = time.perf_counter() - t0
+    return dict(rounds=rounds, rounds_per_s=rounds / sec, seconds=sec, M=M, H=H, b_first=history[0],
+                b_last=history[-1], rounds_until_cap=next((i for i, v in enumerate(history) if v >= b_max), None))
 
 
 PROFILE_CASES = {
