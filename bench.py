@@ -147,6 +147,20 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def aggregate_over_ranks(seconds, units_per_rank, dist=None, device="cuda"):
+    """Whole-job figures of a weak-scaling run: every rank processed `units_per_rank` in `seconds` of its
+    own; returns (maximum of the ranks' times, all ranks' units divided by it).  dist=None: one rank."""
+    world = 1
+    if dist is not None:
+        import torch
+        world = dist.get_world_size()
+        t = torch.tensor([seconds], dtype=torch.float64, device=device)
+        dist.barrier()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        seconds = float(t.item())
+    return seconds, world * units_per_rank / seconds
+
+
 # --------------------------------------------------------------------------- GPU legs
 def time_steps(torch, fn, steps, warmup):
     """CUDA-event timing of `steps` calls of fn(i) after `warmup` untimed ones; returns seconds per call."""
@@ -371,12 +385,8 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     sec = t0.elapsed_time(t1) / 1e3
     stats_ms = sum(a.elapsed_time(z) for a, z in ev) / n_ev
-    if dist is not None:
-        tt = torch.tensor([sec], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        sec = tt.item()
+    sec, value = aggregate_over_ranks(sec, g_bytes * args.steps / 1e9, dist)
     ms_per_step = sec / args.steps * 1e3
-    value = world * g_bytes * args.steps / sec / 1e9
     launches_per_step = 2 + 2 + 1      # tiled statistics + finalise, two next-batch kernels, fused AdamW
     rec = pkg.stats_to_dicts(stats)[0]
 
@@ -403,11 +413,8 @@ def run_ours(args):
             host_step(1 + i)
         torch.cuda.synchronize()
         e2e_sec = (time.perf_counter() - w0) / n_e2e
-        if dist is not None:
-            tt = torch.tensor([e2e_sec], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_sec = tt.item()
-        e2e = dict(value=world * g_bytes / e2e_sec / 1e9, unit="GB/s", h2d_bytes_per_step=g_bytes,
+        e2e_sec, e2e_value = aggregate_over_ranks(e2e_sec, g_bytes / 1e9, dist)
+        e2e = dict(value=e2e_value, unit="GB/s", h2d_bytes_per_step=g_bytes,
                    d2h_bytes_per_step=56 * M + 8, steps=n_e2e, ms_per_step=e2e_sec * 1e3)
         del G_host
 

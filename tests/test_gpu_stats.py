@@ -343,3 +343,32 @@ def test_full_size_launch_configuration(ctx, dtype, M, b, d, d0):
         got = gbar[m, :d0].cpu().numpy()
         np.testing.assert_allclose(got, ref["gbar"], rtol=1e-5, atol=1e-6 * np.abs(ref["gbar"]).max())
         assert torch.equal(gbar[m, d0:2 * d0], gbar[m, :d0])
+
+
+# ------------------------------------------------------------------ worker-gradient estimator (Section 4.3)
+@pytest.mark.parametrize("M,b_local,d", [(4, 16, 30000), (8, 64, 12000), (2, 512, 5000)])
+def test_worker_gradient_estimator(ctx, M, b_local, d):
+    """The implemented test of the paper (Eq. test_stat_actual, Algorithm 2): the rows are the M workers'
+    batch gradients, one row stands for b_local samples and the ratio carries an extra 1/M."""
+    per_sample = inputs.gaussian_rows(123, M, b_local, d, 2.0, device="cuda")
+    # the workers' batch gradients, produced by the library itself
+    st = ctx.new_stats(M)
+    Gb = torch.empty((M, d), device="cuda")
+    ctx.abs_test_stats(per_sample, st, Gb)
+    rows = Gb.unsqueeze(0)                                    # G[1, M, d]
+    stats = ctx.new_stats(1)
+    ctx.abs_test_stats(rows, stats)
+    b_cur = torch.tensor([b_local], dtype=torch.int64, device="cuda")
+    b_next = torch.zeros(1, dtype=torch.int64, device="cuda")
+    T_out = torch.zeros(1, dtype=torch.int64, device="cuda")
+    cfg = pkg.make_test_cfg("norm", 1 << 20, eta=0.5, row_weight=b_local, divisor=M)
+    ctx.abs_next_batch(stats, cfg, b_cur, b_next, T_out)
+    torch.cuda.synchronize()
+    ref = orc.batch_test_stats(to_f64(Gb))
+    rec = pkg.stats_to_dicts(stats)[0]
+    check_record(rec, ref, 1e-5, M)
+    exp_b, exp_T = orc.next_batch([rec], b_local, 1 << 20, "norm", eta=0.5, row_weight=b_local, divisor=M)
+    assert T_out.tolist() == exp_T and b_next.item() == exp_b
+    # Var_m(batch gradients) * b_local estimates the per-sample variance (2^2 * d here)
+    if M >= 4:
+        assert b_local * rec["var_norm"] == pytest.approx(4.0 * d, rel=0.1)
