@@ -26,6 +26,9 @@ WORKLOAD = dict(name="stats sweep centre: G fp32 [M=1, b=256, d=11.2M], sigma=1,
                 M=1, b=256, d=11_200_000, sigma=1.0, seed=2)
 HP = dict(lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) of one abs_stats_tiled_kernel<float,16,keep,full> launch on the 1.024 GB case
+# of profiles/stats_tiled_f32_b256_d1m.txt; traffic grows in proportion to the columns processed.
+NCU_TRAFFIC_SMALL = dict(dram_bytes=1.024164e9 + 4.269e6, d=1_000_000)
 
 
 def measured_peak():
@@ -435,9 +438,12 @@ def run_ours(args):
                              "with fused replica_average",
                         shard="one independent problem per GPU, no collective"),
             rounds_per_s=world * args.steps / sec,
-            roofline=dict(bound="hbm", kernel="abs_stats_tiled_kernel<float,16,keep> (+ finalise)",
+            roofline=dict(bound="hbm", kernel="abs_stats_tiled_kernel<float,16,keep,full> (+ finalise and a 4-byte memset)",
                           achieved=achieved, peak=peak, unit="GB/s", frac=achieved / peak, peak_kind=peak_kind,
-                          frac_of_nominal_8TBps=achieved / 8000.0, ms=stats_ms, traffic=None),
+                          frac_of_nominal_8TBps=achieved / 8000.0, ms=stats_ms,
+                          traffic=NCU_TRAFFIC_SMALL["dram_bytes"] * d / NCU_TRAFFIC_SMALL["d"],
+                          traffic_note="ncu DRAM read+write of the 1.024 GB case scaled by d; algorithmic bytes "
+                                       "are config.bytes_per_step"),
             cpu_baseline=cpu, e2e=e2e, gpu_launches=launches_per_step * args.steps, clocks=clocks,
             result=dict(b_next=int(b_next.item()), var_norm=rec["var_norm"], gbar_sq=rec["gbar_sq"],
                         status=rec["status"]),
