@@ -296,7 +296,12 @@ def run_profile_case(args):
     import torch
     import paper_2406_13936_b200 as pkg
     from paper_2406_13936_b200 import inputs
-    case = PROFILE_CASES[args.case]
+    if args.shape:
+        M_, b_, d_, dt_ = args.shape.split(",")
+        case = dict(kind="stats", M=int(M_), b=int(b_), d=int(d_), dtype=dt_)
+        args.case = "shape:" + args.shape
+    else:
+        case = PROFILE_CASES[args.case]
     pkg.build.build()
     ctx = pkg.Context(0)
     for kv in args.tune:
@@ -463,10 +468,11 @@ def main():
     ap.add_argument("--no-extra", action="store_true")
     ap.add_argument("--case", default=None, choices=sorted(PROFILE_CASES),
                     help="run only a few launches of one kernel on a small case (for profiler captures)")
+    ap.add_argument("--shape", default=None, help="M,b,d,f32|bf16: time abs_test_stats on that shape only")
     ap.add_argument("--tune", action="append", default=[], help="key=value passed to abs_set_tuning (with --case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
-    if args.case:
+    if args.case or args.shape:
         run_profile_case(args)
     elif args.impl == "reference":
         run_reference(args)

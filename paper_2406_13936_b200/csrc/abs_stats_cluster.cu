@@ -155,18 +155,21 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
       const int s = static_cast<int>(i % S);
       mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>((i / S) & 1), abort_flag, prm.timeout_cycles);
       const uint32_t base = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + my_off;
+      const uint32_t base0 = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(cv) * 16u;
       float cs[VE];
 #pragma unroll
       for (int j = 0; j < VE; ++j) cs[j] = 0.f;
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
-        if (FULL || k < n_rows_mine) {
-          cur[k] = lds128(base + static_cast<uint32_t>(k) * row_step);
-          float x[VE];
-          Vec<T>::unpack(cur[k], x);
+        // rows past the batch: safe address, zeroed by a select (no branch around the loads)
+        const bool ok = FULL || k < n_rows_mine;
+        uint4 u = lds128(ok ? base + static_cast<uint32_t>(k) * row_step : base0);
+        if (!ok) u = make_uint4(0u, 0u, 0u, 0u);
+        cur[k] = u;
+        float x[VE];
+        Vec<T>::unpack(u, x);
 #pragma unroll
-          for (int j = 0; j < VE; ++j) cs[j] += x[j];
-        }
+        for (int j = 0; j < VE; ++j) cs[j] += x[j];
       }
       for (int off = lpr; off < 32; off <<= 1) {
 #pragma unroll
@@ -248,21 +251,20 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
       for (int j = 0; j < VE; ++j) vl[j] = 0.f;
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
-        if (FULL || k < n_rows_mine) {
-          float x[VE];
-          Vec<T>::unpack(prev[k], x);
-          float ea = 0.f, eb = 0.f;
+        const bool ok = FULL || k < n_rows_mine;
+        float x[VE];
+        Vec<T>::unpack(prev[k], x);
+        float ea = 0.f, eb = 0.f;
 #pragma unroll
-          for (int j = 0; j < VE; j += 2) {
-            const float d0 = x[j] - g[j];
-            const float d1 = x[j + 1] - g[j + 1];
-            vl[j] = fmaf(d0, d0, vl[j]);
-            vl[j + 1] = fmaf(d1, d1, vl[j + 1]);
-            ea = fmaf(d0, g[j], ea);
-            eb = fmaf(d1, g[j + 1], eb);
-          }
-          e[k] += ea + eb;
+        for (int j = 0; j < VE; j += 2) {
+          const float d0 = ok ? x[j] - g[j] : 0.f;
+          const float d1 = ok ? x[j + 1] - g[j + 1] : 0.f;
+          vl[j] = fmaf(d0, d0, vl[j]);
+          vl[j + 1] = fmaf(d1, d1, vl[j + 1]);
+          ea = fmaf(d0, g[j], ea);
+          eb = fmaf(d1, g[j + 1], eb);
         }
+        e[k] += ea + eb;
       }
       {
         float vs = 0.f;

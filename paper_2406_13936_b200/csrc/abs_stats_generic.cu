@@ -130,12 +130,29 @@ abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, con
   const size_t rec = static_cast<size_t>(b) + 2;
   const double* base = ws + static_cast<size_t>(m) * P * rec;
 
+  // Rows are spread over the threads; when b < 1024 several threads share a row and split the P
+  // records between them (record p goes to thread group p mod tpr), then the groups' sums are
+  // added in group order: the order of additions is fixed, the loads run in parallel.
+  __shared__ double esum[kFinalThreads];
+  int rb = 1;
+  while (rb < kFinalThreads && rb < b) rb <<= 1;          // rows handled per pass (power of two)
+  const int tpr = kFinalThreads / rb;                     // threads per row
+  const int col = tid & (rb - 1), grp = tid / rb;
   double se = 0.0, see = 0.0;
-  for (long long r = tid; r < b; r += kFinalThreads) {
+  for (long long r0 = 0; r0 < b; r0 += rb) {
+    const long long r = r0 + col;
     double e = 0.0;
-    for (int p = 0; p < P; ++p) e += base[p * rec + r];
-    se += e;
-    see += e * e;
+    if (r < b)
+      for (int p = grp; p < P; p += tpr) e += base[p * rec + r];
+    esum[tid] = e;
+    __syncthreads();
+    if (grp == 0 && r < b) {
+      double tot = 0.0;
+      for (int g2 = 0; g2 < tpr; ++g2) tot += esum[g2 * rb + col];
+      se += tot;
+      see += tot * tot;
+    }
+    __syncthreads();
   }
   // V and N: thread t takes the records p = t, t + 1024, ...
   double vn = 0.0, nn = 0.0;
