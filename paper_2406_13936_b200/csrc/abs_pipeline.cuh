@@ -65,6 +65,22 @@ __device__ __forceinline__ void named_bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
+// 16-byte shared-memory accesses for per-thread groups of VE floats (VE = 4 or 8): a warp then
+// touches 512 contiguous bytes per instruction instead of striding scalars across the banks.
+template <int VE>
+__device__ __forceinline__ void smem_store_vec(float* dst, const float (&v)[VE]) {
+#pragma unroll
+  for (int j = 0; j < VE; j += 4) *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+}
+template <int VE>
+__device__ __forceinline__ void smem_add_vec(const float* src, float (&acc)[VE]) {
+#pragma unroll
+  for (int j = 0; j < VE; j += 4) {
+    const float4 t = *reinterpret_cast<const float4*>(src + j);
+    acc[j] += t.x; acc[j + 1] += t.y; acc[j + 2] += t.z; acc[j + 3] += t.w;
+  }
+}
+
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);

@@ -177,8 +177,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
       }
       float* buf = part + static_cast<size_t>(i & 1) * (kCW * cols);
       if (sub == 0) {
-#pragma unroll
-        for (int j = 0; j < VE; ++j) buf[warp * cols + cv * VE + j] = cs[j];
+        smem_store_vec<VE>(buf + warp * cols + cv * VE, cs);
       }
       __syncthreads();     // partial sums visible; every thread has its rows in registers
       if (tid == 0 && i + S < n_mine) issue_load(i + S);     // the buffer is free: refill it
@@ -193,11 +192,9 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
 #pragma unroll
           for (int j = 0; j < VE; ++j) tot[j] = 0.f;
           for (int w = 0; w < kCW; ++w) {
-#pragma unroll
-            for (int j = 0; j < VE; ++j) tot[j] += buf[w * cols + lane * VE + j];
+            smem_add_vec<VE>(buf + w * cols + lane * VE, tot);
           }
-#pragma unroll
-          for (int j = 0; j < VE; ++j) mine[lane * VE + j] = tot[j];
+          smem_store_vec<VE>(mine + lane * VE, tot);
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads what was just written
         }
         __syncwarp();
@@ -220,8 +217,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
       for (int j = 0; j < VE; ++j) g[j] = 0.f;
       for (int peer = 0; peer < C; ++peer) {      // fixed order: the same mean in every CTA
         const float* src = xsum + (q * kMaxCluster + peer) * cols + cv * VE;
-#pragma unroll
-        for (int j = 0; j < VE; ++j) g[j] += src[j];
+        smem_add_vec<VE>(src, g);
       }
 #pragma unroll
       for (int j = 0; j < VE; ++j) g[j] *= inv_b;

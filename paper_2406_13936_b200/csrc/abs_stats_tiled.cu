@@ -49,8 +49,9 @@ struct TiledParams {
 };
 
 // ---- the kernel ----------------------------------------------------------------------------
-// RMAX: upper bound on the rows a thread owns; KEEP: the rows stay in registers between the
-// sweeps; FULL: every thread owns exactly RMAX rows (no per-row predicates).  Variants with
+// RMAX: rows a thread owns (exactly ceil(b / row groups) when KEEP, an upper bound otherwise);
+// KEEP: the rows stay in registers between the sweeps; FULL: every thread owns exactly RMAX
+// rows (no predicates at all).  Variants with
 // at most 8 rows per thread are compiled for two CTAs per SM.
 template <typename T, int RMAX, bool KEEP, bool FULL>
 __global__ void __launch_bounds__(kThreads, (RMAX <= 8 ? 2 : 1))
@@ -137,6 +138,9 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
     const int RG = rs * subs;                     // row groups per box
     const int rg = wr * subs + sub;
     const int n_rows_mine = (b > rg) ? (b - rg + RG - 1) / RG : 0;   // rows rg, rg+RG, ...
+    // In the register-resident variants RMAX is exactly ceil(b / RG): every thread owns rows
+    // 0..RMAX-2 of its group and only the last one can fall past the batch.
+    const bool last_ok = n_rows_mine >= RMAX;
     const unsigned row_step = static_cast<unsigned>(RG) * row_bytes;
     const uint32_t my_off = static_cast<uint32_t>(q) * prm.box_bytes + static_cast<uint32_t>(rg) * row_bytes +
                             static_cast<uint32_t>(cv) * 16u;
@@ -166,7 +170,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
       for (int k = 0; k < RMAX; ++k) {
         // Rows past the batch are loaded from a safe address and zeroed by a select: no branch,
         // so the loads of a sweep are issued back to back.
-        const bool ok = FULL || k < n_rows_mine;
+        const bool ok = FULL || (KEEP ? (k < RMAX - 1 || last_ok) : k < n_rows_mine);
         uint4 u = lds128(ok ? base + static_cast<uint32_t>(k) * row_step : base0);
         if (!ok) u = make_uint4(0u, 0u, 0u, 0u);
         if (KEEP) v[k] = u;
@@ -186,8 +190,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
       if (rs > 1) {
         float* buf = part + static_cast<size_t>(i & 1) * (kConsumerWarps * lpr * VE);
         if (sub == 0) {
-#pragma unroll
-          for (int j = 0; j < VE; ++j) buf[(warp * lpr + cv) * VE + j] = cs[j];
+          smem_store_vec<VE>(buf + (warp * lpr + cv) * VE, cs);
         }
         named_bar_sync(1 + q, rs * 32);
 #pragma unroll
@@ -195,8 +198,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
         const int w0 = q << prm.rs_log2;
         for (int w = 0; w < rs; ++w) {
           const float* src = buf + ((w0 + w) * lpr + cv) * VE;
-#pragma unroll
-          for (int j = 0; j < VE; ++j) cs[j] += src[j];
+          smem_add_vec<VE>(src, cs);
         }
       }
       float g[VE];
@@ -230,7 +232,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
       for (int j = 0; j < VE; ++j) vl[j] = 0.f;
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
-        const bool ok = FULL || k < n_rows_mine;
+        const bool ok = FULL || (KEEP ? (k < RMAX - 1 || last_ok) : k < n_rows_mine);
         const uint4 u = KEEP ? v[k] : lds128(ok ? base + static_cast<uint32_t>(k) * row_step : base0);
         float x[VE];
         Vec<T>::unpack(u, x);
@@ -263,7 +265,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
         for (int k = 0; k < RMAX; ++k) {
           float ek = e[k];
           for (int off = 1; off < lpr; off <<= 1) ek += __shfl_xor_sync(0xffffffffu, ek, off);
-          if (cv == 0 && (FULL || k < n_rows_mine)) e_mine[rg + k * RG] += static_cast<double>(ek);
+          if (cv == 0 && (FULL || (KEEP ? (k < RMAX - 1 || last_ok) : k < n_rows_mine))) e_mine[rg + k * RG] += static_cast<double>(ek);
           e[k] = 0.f;
         }
       }
@@ -348,8 +350,8 @@ bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, 
       c->box_rows = box_rows;
       c->n_row_boxes = n_row_boxes;
       c->keep = (pass == 0);
-      c->rmax = pass == 0 ? (R <= 4 ? 4 : (R <= 8 ? 8 : 16)) : 32;
-      c->full = (b % RG == 0) && (R == c->rmax);
+      c->rmax = pass == 0 ? static_cast<int>(R) : 32;
+      c->full = (b % RG == 0) && (pass == 0 ? (R == 2 || R == 4 || R == 8 || R == 16) : R == 32);
       c->box_bytes = static_cast<unsigned>(rows_pad * lpr * 16);
       c->stage_bytes = static_cast<unsigned>(stage);
       c->smem_bytes = stages * stage + extras_bytes(lpr, ve, bx, b, stages) + 128;
@@ -369,22 +371,30 @@ int launch_variant(abs_ctx* ctx, const CUtensorMap& tmap, const TiledParams& prm
   return ABS_OK;
 }
 
-template <typename T, bool FULL>
-int launch_full(abs_ctx* ctx, const TileChoice& c, const CUtensorMap& tmap, const TiledParams& prm, dim3 grid,
-                cudaStream_t stream) {
-  if (!c.keep) return launch_variant<T, 32, false, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-  switch (c.rmax) {
-    case 4: return launch_variant<T, 4, true, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-    case 8: return launch_variant<T, 8, true, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-    default: return launch_variant<T, 16, true, FULL>(ctx, tmap, prm, grid, c.smem_bytes, stream);
-  }
-}
-
 template <typename T>
 int launch_typed(abs_ctx* ctx, const TileChoice& c, const CUtensorMap& tmap, const TiledParams& prm, dim3 grid,
                  cudaStream_t stream) {
-  return c.full ? launch_full<T, true>(ctx, c, tmap, prm, grid, stream)
-                : launch_full<T, false>(ctx, c, tmap, prm, grid, stream);
+  const size_t smem = c.smem_bytes;
+  if (!c.keep)
+    return c.full ? launch_variant<T, 32, false, true>(ctx, tmap, prm, grid, smem, stream)
+                  : launch_variant<T, 32, false, false>(ctx, tmap, prm, grid, smem, stream);
+  if (c.full) {
+    switch (c.rmax) {
+      case 2: return launch_variant<T, 2, true, true>(ctx, tmap, prm, grid, smem, stream);
+      case 4: return launch_variant<T, 4, true, true>(ctx, tmap, prm, grid, smem, stream);
+      case 8: return launch_variant<T, 8, true, true>(ctx, tmap, prm, grid, smem, stream);
+      default: return launch_variant<T, 16, true, true>(ctx, tmap, prm, grid, smem, stream);
+    }
+  }
+  switch (c.rmax) {
+#define ABS_TILED_CASE(R) \
+  case R: return launch_variant<T, R, true, false>(ctx, tmap, prm, grid, smem, stream);
+    ABS_TILED_CASE(1) ABS_TILED_CASE(2) ABS_TILED_CASE(3) ABS_TILED_CASE(4) ABS_TILED_CASE(5) ABS_TILED_CASE(6)
+    ABS_TILED_CASE(7) ABS_TILED_CASE(8) ABS_TILED_CASE(9) ABS_TILED_CASE(10) ABS_TILED_CASE(11) ABS_TILED_CASE(12)
+    ABS_TILED_CASE(13) ABS_TILED_CASE(14) ABS_TILED_CASE(15)
+#undef ABS_TILED_CASE
+    default: return launch_variant<T, 16, true, false>(ctx, tmap, prm, grid, smem, stream);
+  }
 }
 
 }  // namespace
