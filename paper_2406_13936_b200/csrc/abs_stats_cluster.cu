@@ -70,8 +70,8 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// RMAX: rows per thread and register set (two sets alternate); FULL: every thread of every CTA
-// owns exactly RMAX rows, so the row loops need no predicates.
+// RMAX: rows per thread and register set, exactly ceil(rows per CTA / row groups) (two sets
+// alternate); FULL: every thread of every CTA owns exactly RMAX rows, so nothing is predicated.
 template <typename T, int RMAX, bool FULL>
 __global__ void __launch_bounds__(kThreadsC, 1)
 abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const ClusterParams prm) {
@@ -137,6 +137,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
   const int RG = kCW * subs;                     // row groups
   const int rg = warp * subs + sub;
   const int n_rows_mine = (b_loc > rg) ? (b_loc - rg + RG - 1) / RG : 0;
+  const bool last_ok = n_rows_mine >= RMAX;       // RMAX is exactly ceil(RC / RG): only the last row can be missing
   const unsigned row_step = static_cast<unsigned>(RG) * row_bytes;
   const uint32_t my_off = static_cast<uint32_t>(rg) * row_bytes + static_cast<uint32_t>(cv) * 16u;
   const float inv_b = 1.0f / static_cast<float>(b);
@@ -162,7 +163,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
         // rows past the batch: safe address, zeroed by a select (no branch around the loads)
-        const bool ok = FULL || k < n_rows_mine;
+        const bool ok = FULL || k < RMAX - 1 || last_ok;
         uint4 u = lds128(ok ? base + static_cast<uint32_t>(k) * row_step : base0);
         if (!ok) u = make_uint4(0u, 0u, 0u, 0u);
         cur[k] = u;
@@ -247,7 +248,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
       for (int j = 0; j < VE; ++j) vl[j] = 0.f;
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
-        const bool ok = FULL || k < n_rows_mine;
+        const bool ok = FULL || k < RMAX - 1 || last_ok;
         float x[VE];
         Vec<T>::unpack(prev[k], x);
         float ea = 0.f, eb = 0.f;
@@ -274,7 +275,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
         for (int k = 0; k < RMAX; ++k) {
           float ek = e[k];
           for (int off = 1; off < lpr; off <<= 1) ek += __shfl_xor_sync(0xffffffffu, ek, off);
-          if (cv == 0 && (FULL || k < n_rows_mine)) e_acc[rg + k * RG] += static_cast<double>(ek);
+          if (cv == 0 && (FULL || k < RMAX - 1 || last_ok)) e_acc[rg + k * RG] += static_cast<double>(ek);
           e[k] = 0.f;
         }
       }
@@ -367,7 +368,7 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   const int subs = 32 / lpr;
   const int RG = kCW * subs;
   const int R = (RC + RG - 1) / RG;                                // rows per thread, <= 16
-  const int rmax = R <= 8 ? 8 : 16;
+  const int rmax = R;
   const int n_row_boxes = (RC + 255) / 256;
   const int box_rows = (RC + n_row_boxes - 1) / n_row_boxes;
   const int rows_pad = box_rows * n_row_boxes;
@@ -400,15 +401,25 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.timeout_cycles = 4000000000ll;
-  const bool full = (a.b % C == 0) && (RC % RG == 0) && (RC / RG == rmax);
-#define ABS_CLUSTER_DISPATCH(T)                                                                          \
-  (rmax == 8 ? (full ? launch_cluster_variant<T, 8, true>(ctx, tmap, prm, a, C, smem, P_out)             \
-                     : launch_cluster_variant<T, 8, false>(ctx, tmap, prm, a, C, smem, P_out))           \
-             : (full ? launch_cluster_variant<T, 16, true>(ctx, tmap, prm, a, C, smem, P_out)            \
-                     : launch_cluster_variant<T, 16, false>(ctx, tmap, prm, a, C, smem, P_out)))
-  if (a.dtype == ABS_F32) return ABS_CLUSTER_DISPATCH(float);
-  return ABS_CLUSTER_DISPATCH(__nv_bfloat16);
+  const bool full = (a.b % C == 0) && (RC % RG == 0) && (rmax == 8 || rmax == 16);
+#define ABS_CLUSTER_CASE(T, R) \
+  case R: return launch_cluster_variant<T, R, false>(ctx, tmap, prm, a, C, smem, P_out);
+#define ABS_CLUSTER_DISPATCH(T)                                                                        \
+  if (full) {                                                                                          \
+    return rmax == 8 ? launch_cluster_variant<T, 8, true>(ctx, tmap, prm, a, C, smem, P_out)           \
+                     : launch_cluster_variant<T, 16, true>(ctx, tmap, prm, a, C, smem, P_out);         \
+  }                                                                                                    \
+  switch (rmax) {                                                                                      \
+    ABS_CLUSTER_CASE(T, 1) ABS_CLUSTER_CASE(T, 2) ABS_CLUSTER_CASE(T, 3) ABS_CLUSTER_CASE(T, 4)        \
+    ABS_CLUSTER_CASE(T, 5) ABS_CLUSTER_CASE(T, 6) ABS_CLUSTER_CASE(T, 7) ABS_CLUSTER_CASE(T, 8)        \
+    ABS_CLUSTER_CASE(T, 9) ABS_CLUSTER_CASE(T, 10) ABS_CLUSTER_CASE(T, 11) ABS_CLUSTER_CASE(T, 12)     \
+    ABS_CLUSTER_CASE(T, 13) ABS_CLUSTER_CASE(T, 14) ABS_CLUSTER_CASE(T, 15)                            \
+    default: return launch_cluster_variant<T, 16, false>(ctx, tmap, prm, a, C, smem, P_out);           \
+  }
+  if (a.dtype == ABS_F32) { ABS_CLUSTER_DISPATCH(float) }
+  ABS_CLUSTER_DISPATCH(__nv_bfloat16)
 #undef ABS_CLUSTER_DISPATCH
+#undef ABS_CLUSTER_CASE
 }
 
 }  // namespace
