@@ -443,7 +443,7 @@ def run_ours(args):
                              "with fused replica_average",
                         shard="one independent problem per GPU, no collective"),
             rounds_per_s=world * args.steps / sec,
-            roofline=dict(bound="hbm", kernel="abs_stats_tiled_kernel<float,16,keep,full> (+ finalise and a 4-byte memset)",
+            roofline=dict(bound="hbm", kernel="abs_stats_tiled_kernel<float,16,keep,full> (+ finalise)",
                           achieved=achieved, peak=peak, unit="GB/s", frac=achieved / peak, peak_kind=peak_kind,
                           frac_of_nominal_8TBps=achieved / 8000.0, ms=stats_ms,
                           traffic=NCU_TRAFFIC_SMALL["dram_bytes"] * d / NCU_TRAFFIC_SMALL["d"],

@@ -45,7 +45,8 @@ int validate_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long lon
 }
 
 int run_stats(abs_ctx* ctx, const StatsLaunch& a) {
-  ABS_CUDA_TRY(ctx, cudaMemsetAsync(ctx->flags, 0, sizeof(unsigned), a.stream));
+  // ctx->flags[0] (time-out flag) is zero here: abs_create clears it and the finalisation kernel
+  // of the previous call cleared it again after reading it.
   int P = 0;
   int rc = ABS_ERR_UNSUPPORTED;
   if (!ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_gram) rc = launch_stats_gram(ctx, a, &P);

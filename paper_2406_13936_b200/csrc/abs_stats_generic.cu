@@ -122,7 +122,7 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
 constexpr int kFinalThreads = 1024;
 
 __global__ void __launch_bounds__(kFinalThreads)
-abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, const unsigned* __restrict__ flags,
+abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, unsigned* __restrict__ flags,
                           abs_stats* __restrict__ stats_out) {
   __shared__ double red[4][kFinalThreads / 32];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -189,7 +189,14 @@ abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, con
     unsigned status = 0u;
     if (!(isfinite(V) && isfinite(N) && isfinite(s_ee))) status |= ABS_STATUS_NONFINITE;
     if (N == 0.0) status |= ABS_STATUS_ZERO_MEAN;
-    if (flags[0] != 0u) status |= ABS_STATUS_TIMEOUT;
+    if (*reinterpret_cast<volatile unsigned*>(flags) != 0u) status |= ABS_STATUS_TIMEOUT;
+    // The last worker's block to get here clears the time-out flag (flags[0]) and the arrival
+    // counter (flags[1]) for the next call, which saves a memset per call.
+    __threadfence();
+    if (atomicAdd(flags + 1, 1u) == gridDim.x - 1) {
+      flags[0] = 0u;
+      flags[1] = 0u;
+    }
     abs_stats s;
     s.gbar_sq = N;
     s.var_norm = var_norm;
