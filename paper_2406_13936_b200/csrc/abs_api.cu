@@ -143,6 +143,12 @@ extern "C" int abs_set_tuning(abs_ctx* ctx, const char* key, long long value) {
   } else if (strcmp(key, "stats_stage_kb") == 0) {
     if (value != 0 && (value < 4 || value > 200)) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_stage_kb must be 0 or 4..200");
     ctx->tuning.stats_stage_kb = value;
+  } else if (strcmp(key, "stats_timeout_cycles") == 0) {
+    if (value != 0 && (value < 100000 || value > 4000000000ll))
+      return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_timeout_cycles must be 0 or 1e5..4e9");
+    ctx->tuning.stats_timeout_cycles = value;
+  } else if (strcmp(key, "stats_fault_drop_loads") == 0) {
+    ctx->tuning.stats_fault_drop_loads = value ? 1 : 0;
   } else if (strcmp(key, "stats_cluster_rows") == 0) {
     if (value != 0 && (value < 16 || value > 512)) return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_cluster_rows must be 0 or 16..512");
     ctx->tuning.stats_cluster_rows = value;

@@ -14,7 +14,8 @@ namespace absk {
 
 constexpr int kSmCountFallback = 148;
 constexpr size_t kDefaultWorkspace = 64ull << 20;
-constexpr int kMaxFastRows = 4096;          // largest b the tiled statistics kernel covers
+constexpr int kMaxFastRows = 4096;
+constexpr long long kDefaultTimeoutCycles = 4000000000ll;   // about two seconds of SM clock          // largest b the tiled statistics kernel covers
 
 struct Tuning {
   long long stats_stages = 0;
@@ -26,6 +27,8 @@ struct Tuning {
   long long stats_no_gram = 0;
   long long stats_no_cluster = 0;
   long long stats_cluster_rows = 0;
+  long long stats_timeout_cycles = 0;      // 0: about two seconds of SM clock
+  long long stats_fault_drop_loads = 0;    // test hook: the tiled kernel's loader issues no copies
 };
 
 }  // namespace absk

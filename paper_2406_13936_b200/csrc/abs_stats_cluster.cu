@@ -400,7 +400,7 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   prm.ws = static_cast<double*>(ctx->workspace);
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
-  prm.timeout_cycles = 4000000000ll;
+  prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
   const bool full = (a.b % C == 0) && (RC % RG == 0) && (rmax == 8 || rmax == 16);
 #define ABS_CLUSTER_CASE(T, R) \
   case R: return launch_cluster_variant<T, R, false>(ctx, tmap, prm, a, C, smem, P_out);

@@ -323,7 +323,7 @@ int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.ws = static_cast<double*>(ctx->workspace);
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
-  prm.timeout_cycles = 4000000000ll;
+  prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
   const size_t smem = smem_for(stages);
   const bool gb = a.gbar_out != nullptr;

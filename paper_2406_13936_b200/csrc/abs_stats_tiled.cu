@@ -46,6 +46,7 @@ struct TiledParams {
   float* gbar_out;
   unsigned* flags;
   long long timeout_cycles;
+  int drop_loads;        // fault injection for the bounded waits: the loader issues nothing
 };
 
 // ---- the kernel ----------------------------------------------------------------------------
@@ -108,6 +109,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
         const long long use = i / S;
         if (use > 0)
           mbar_wait(empty_u32 + 8u * s, static_cast<uint32_t>((use - 1) & 1), abort_flag, prm.timeout_cycles);
+        if (prm.drop_loads) continue;     // test hook: the consumers' waits must run out, not hang
         const uint32_t full = full_u32 + 8u * s;
         mbar_expect_tx(full, prm.stage_bytes);
         const long long it = p + i * prm.P;
@@ -456,7 +458,8 @@ int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.ws = static_cast<double*>(ctx->workspace);
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
-  prm.timeout_cycles = 4000000000ll;   // about two seconds of SM clock
+  prm.drop_loads = ctx->tuning.stats_fault_drop_loads ? 1 : 0;
+  prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
 
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
   int rc;

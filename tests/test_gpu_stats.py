@@ -372,3 +372,25 @@ def test_worker_gradient_estimator(ctx, M, b_local, d):
     # Var_m(batch gradients) * b_local estimates the per-sample variance (2^2 * d here)
     if M >= 4:
         assert b_local * rec["var_norm"] == pytest.approx(4.0 * d, rel=0.1)
+
+
+# ------------------------------------------------------------------ bounded waits
+def test_wait_that_runs_out_is_reported_and_the_context_stays_usable(ctx):
+    """Failure detection without a fault: with the loader switched off no tile ever arrives, every
+    wait gives up after its (shortened) limit, the kernel returns normally and the records carry
+    ABS_STATUS_TIMEOUT; the next ordinary call on the same context is correct again."""
+    G = make_G(77, 2, 40, 6000, torch.float32)
+    ctx.set_tuning("stats_no_cluster", 1)
+    ctx.set_tuning("stats_timeout_cycles", 2_000_000)        # about a millisecond
+    ctx.set_tuning("stats_fault_drop_loads", 1)
+    try:
+        flagged, _ = run_gpu(ctx, G, want_gbar=False)
+    finally:
+        ctx.set_tuning("stats_fault_drop_loads", 0)
+        ctx.set_tuning("stats_timeout_cycles", 0)
+        ctx.set_tuning("stats_no_cluster", 0)
+    assert all(r["status"] & pkg.binding.STATUS_TIMEOUT for r in flagged)
+    recs, _ = run_gpu(ctx, G, want_gbar=False)                # same context, ordinary call
+    H = to_f64(G)
+    for m in range(2):
+        check_record(recs[m], orc.batch_test_stats(H[m]), 1e-5, 40)
