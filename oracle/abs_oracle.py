@@ -195,6 +195,36 @@ def next_batch(stats_per_worker, b_cur, b_max, kind, **cfg):
     return min(b_max, b_next), T
 
 
+def next_batch_local(stats_per_worker, b_cur_per_worker, b_max, kind, eta_per_worker=None, **cfg):
+    """Per-worker next local batch sizes, b^m_{k+1} = max{T^m, b^m_k} capped at b_max, with one
+    norm-test constant eta_m per worker (Eq. approx_norm_local, Eq. test_stat, Alg. 1) and no
+    maximum over the workers.  Returns ([b^1..b^M], [T^1..T^M])."""
+    out, T = [], []
+    for m, s in enumerate(stats_per_worker):
+        c = dict(cfg)
+        if eta_per_worker is not None:
+            c["eta"] = eta_per_worker[m]
+        t = batch_test_statistic(s, kind, **c)
+        T.append(t)
+        out.append(min(b_max, max(b_cur_per_worker[m], t)))
+    return out, T
+
+
+def merge_norm_stats(mean_a, n_a, var_a, mean_b, n_b, var_b):
+    """Batch gradient and norm-test variance of the union of two disjoint sub-batches from their
+    own means and variances (gradient accumulation over micro-batches, Section 6):
+      mean = (n_a mean_a + n_b mean_b) / n
+      sum_i ||g_i - mean||^2 = S_a + S_b + ||mean_a - mean_b||^2 n_a n_b / n,  S = (n-1) Var (Eq. def_var)
+    Returns (mean, n, var, ||mean||^2)."""
+    mean_a = np.asarray(mean_a, dtype=np.float64)
+    mean_b = np.asarray(mean_b, dtype=np.float64)
+    n = n_a + n_b
+    mean = (n_a * mean_a + n_b * mean_b) / n
+    diff = mean_a - mean_b
+    S = (n_a - 1) * var_a + (n_b - 1) * var_b + float(np.dot(diff, diff)) * n_a * n_b / n
+    return mean, n, S / (n - 1), float(np.dot(mean, mean))
+
+
 # ----------------------------------------------------------------------------
 # local updates
 # ----------------------------------------------------------------------------

@@ -407,3 +407,32 @@ def test_round_structure_on_a_quadratic():
             Y[m] = Y[m] - lr * (Y[m] - xi[m, h].mean(axis=0))
     np.testing.assert_allclose(X, np.tile(Y.mean(axis=0), (M, 1)), rtol=1e-13)
     assert b_next == max([b] + T)
+
+
+# ---------------------------------------------------------------- per-worker sizes, merged sub-batches
+def test_per_worker_batch_sizes():
+    stats = [_fake(var_norm=0.25 * r) for r in (3.2, 90.5, 17.0)]
+    b, T = orc.next_batch_local(stats, [8, 8, 40], 64, "norm", eta=0.5)
+    assert T == [4, 91, 17] and b == [8, 64, 40]
+    # a worker with a looser constant asks for less: eta_m = 1 quarters the ratio of eta = 1/2
+    b, T = orc.next_batch_local(stats, [2, 2, 2], 1000, "norm", eta_per_worker=[0.5, 1.0, 0.25])
+    assert T == [4, math.ceil(90.5 / 4), 68] and b == T
+
+
+@pytest.mark.parametrize("n_a,n_b", [(2, 2), (5, 3), (16, 1), (1, 7)])
+def test_merged_sub_batches_equal_the_whole_batch(n_a, n_b):
+    rng = np.random.default_rng(n_a * 10 + n_b)
+    G = rng.standard_normal((n_a + n_b, 33)) * 2.0 + 0.7
+    whole = orc.batch_test_stats(G) if n_a + n_b >= 2 else None
+    def part(rows):
+        if rows.shape[0] >= 2:
+            s = orc.batch_test_stats(rows)
+            return s["gbar"], s["var_norm"]
+        return rows[0], 0.0                       # a single row: no spread
+    ma, va = part(G[:n_a])
+    mb, vb = part(G[n_a:])
+    mean, n, var, N = orc.merge_norm_stats(ma, n_a, va, mb, n_b, vb)
+    assert n == n_a + n_b
+    np.testing.assert_allclose(mean, whole["gbar"], rtol=1e-13, atol=1e-15)
+    assert var == pytest.approx(whole["var_norm"], rel=1e-12)
+    assert N == pytest.approx(whole["gbar_sq"], rel=1e-12)
