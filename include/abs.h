@@ -53,6 +53,8 @@ extern "C" {
 /* ---- status bits written to abs_stats.status ------------------------------ */
 #define ABS_STATUS_NONFINITE  1u  /* an input or an accumulator was not finite (or overflowed) */
 #define ABS_STATUS_ZERO_MEAN  2u  /* ||gbar||^2 == 0: the test ratios are undefined            */
+#define ABS_STATUS_NORM_ONLY  8u  /* a record merged from sub-batches: only gbar_sq, var_norm,
+                                     sum_sq and rows are meaningful (abs_stats_merge)          */
 #define ABS_STATUS_TIMEOUT    4u  /* an asynchronous tile copy did not arrive in time; the
                                      numbers in this record are not valid                      */
 
@@ -204,6 +206,30 @@ typedef struct {
  *           (may alias b_cur).  M <= 1024.                                          */
 int abs_next_batch(abs_ctx* ctx, const abs_stats* stats, int M, const abs_test_cfg* cfg,
                    const long long* b_cur, long long* T_out, long long* b_next, void* stream);
+
+/* Per-worker next local batch sizes (Eq. test_stat before the practical maximum
+ * over workers; Algorithm 1: b^m <- max{T^m, b^m}), with one norm-test constant
+ * per worker (eta_m of Eq. approx_norm_local):
+ *   b_next[m] = min( b_max, max( b_cur[m], T^m ) ),  T^m as in abs_next_batch.
+ * eta_m: DEVICE array [M] of constants, or NULL to use cfg->eta for every worker
+ * (ignored by the augmented inner-product test).  b_cur, b_next, T_out: device [M]
+ * (b_next may alias b_cur; T_out may be NULL).  cfg is a HOST pointer.            */
+int abs_next_batch_local(abs_ctx* ctx, const abs_stats* stats, int M, const abs_test_cfg* cfg,
+                         const double* eta_m, const long long* b_cur, long long* T_out,
+                         long long* b_next, void* stream);
+
+/* Norm-test statistics of a batch that arrives in sub-batches (gradient
+ * accumulation over micro-batches, Section 6): folds sub-batch b into the running
+ * pair a.  Per worker m, with n = rows, S = (n-1) var_norm (Eq. def_var):
+ *   mean_a <- (n_a mean_a + n_b mean_b) / (n_a + n_b)                  (in place)
+ *   S      <- S_a + S_b + ||mean_a - mean_b||^2 n_a n_b / (n_a + n_b)
+ * rec_a [M] receives rows, var_norm, gbar_sq = ||mean||^2, sum_sq and the status
+ * bit ABS_STATUS_NORM_ONLY (var_ip / var_orth cannot be merged: they are set to 0
+ * and abs_next_batch gives T = 0 for the augmented test on such a record).
+ * mean_a, mean_b: [M][d] fp32 batch gradients as written by abs_test_stats
+ * (gbar_out); rec_a, rec_b: the matching records.  All device pointers.           */
+int abs_stats_merge(abs_ctx* ctx, float* mean_a, const float* mean_b, int M, long long d,
+                    abs_stats* rec_a, const abs_stats* rec_b, void* stream);
 
 /* Local SGD step for all replicas (Eq. local_sgd_alt): X[m] <- X[m] - lr * Gb[m],
  * m < M, in fp32.  X, Gb: [M][d] fp32 with replica m at + m*replica_stride

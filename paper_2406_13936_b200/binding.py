@@ -14,7 +14,7 @@ from . import build as _build
 
 ABS_F32, ABS_BF16 = 0, 1
 ABS_TEST_NORM, ABS_TEST_AUG_INNER_PRODUCT = 0, 1
-STATUS_NONFINITE, STATUS_ZERO_MEAN, STATUS_TIMEOUT = 1, 2, 4
+STATUS_NONFINITE, STATUS_ZERO_MEAN, STATUS_TIMEOUT, STATUS_NORM_ONLY = 1, 2, 4, 8
 STATS_RECORD_BYTES = 56
 
 
@@ -75,6 +75,10 @@ EXPORTS = {
                       ctypes.c_int, ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p,
                       ctypes.c_size_t, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p,
                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_next_batch_local": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(TestCfg), ctypes.c_void_p,
+                             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_stats_merge": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
+                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "local_sgd_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
                        ctypes.c_longlong, ctypes.c_float, ctypes.c_int, ctypes.c_void_p],
     "local_adamw_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -203,6 +207,20 @@ class Context:
                                       _ptr(b_next), _stream(stream))
         self._check(rc, "abs_next_batch")
         return b_next
+
+    def abs_next_batch_local(self, stats, cfg, b_cur, b_next, eta_m=None, T_out=None, stream=None):
+        """Per-worker sizes: b_cur / b_next int64 device tensors [M]; eta_m float64 device tensor [M] or None."""
+        M = stats.shape[0]
+        self._check(self._lib.abs_next_batch_local(self._h, _ptr(stats), M, ctypes.byref(cfg), _ptr(eta_m),
+                                                   _ptr(b_cur), _ptr(T_out), _ptr(b_next), _stream(stream)),
+                    "abs_next_batch_local")
+        return b_next
+
+    def abs_stats_merge(self, mean_a, mean_b, rec_a, rec_b, stream=None):
+        """Folds sub-batch (mean_b, rec_b) into the running (mean_a, rec_a); mean tensors [M, d] fp32."""
+        M, d = mean_a.shape
+        self._check(self._lib.abs_stats_merge(self._h, _ptr(mean_a), _ptr(mean_b), M, d, _ptr(rec_a), _ptr(rec_b),
+                                              _stream(stream)), "abs_stats_merge")
 
     # ---- local updates -------------------------------------------------------------------
     @staticmethod

@@ -28,7 +28,9 @@ abs_next_batch_kernel(const abs_stats* __restrict__ stats, int M, abs_test_cfg c
   long long T = 0;
   if (tid < M) {
     const abs_stats s = stats[tid];
-    if ((s.status & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) == 0u) {
+    const bool usable = (s.status & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) == 0u &&
+                        (cfg.kind == ABS_TEST_NORM || (s.status & ABS_STATUS_NORM_ONLY) == 0u);
+    if (usable) {
       const double scale = cfg.row_weight / cfg.divisor;
       const double N = s.gbar_sq;
       if (cfg.kind == ABS_TEST_NORM) {

@@ -394,3 +394,68 @@ def test_wait_that_runs_out_is_reported_and_the_context_stays_usable(ctx):
     H = to_f64(G)
     for m in range(2):
         check_record(recs[m], orc.batch_test_stats(H[m]), 1e-5, 40)
+
+
+# ------------------------------------------------------------------ per-worker sizes, merged sub-batches
+def test_per_worker_batch_sizes_with_heterogeneous_constants(ctx):
+    M, b, d = 5, 24, 9000
+    G = make_G(300, M, b, d, torch.float32, sigma=0.7)
+    stats = ctx.new_stats(M)
+    ctx.abs_test_stats(G, stats)
+    etas = [0.3, 0.5, 0.8, 0.95, 0.5]
+    cur = [24, 24, 24, 5000, 10]
+    eta_dev = torch.tensor(etas, dtype=torch.float64, device="cuda")
+    b_cur = torch.tensor(cur, dtype=torch.int64, device="cuda")
+    b_next = torch.zeros(M, dtype=torch.int64, device="cuda")
+    T_out = torch.zeros(M, dtype=torch.int64, device="cuda")
+    cfg = pkg.make_test_cfg("norm", 4096, eta=0.5)
+    ctx.abs_next_batch_local(stats, cfg, b_cur, b_next, eta_m=eta_dev, T_out=T_out)
+    torch.cuda.synchronize()
+    recs = pkg.stats_to_dicts(stats)
+    exp_b, exp_T = orc.next_batch_local(recs, cur, 4096, "norm", eta_per_worker=etas)
+    assert T_out.tolist() == exp_T and b_next.tolist() == exp_b
+    # no per-worker constants: cfg.eta for everybody, and the augmented test
+    for kind, kw in (("norm", dict(eta=0.5)), ("aug_ip", dict(theta=0.5, nu=0.5))):
+        ctx.abs_next_batch_local(stats, pkg.make_test_cfg(kind, 4096, **kw), b_cur, b_next, T_out=T_out)
+        exp_b, exp_T = orc.next_batch_local(recs, cur, 4096, kind, **kw)
+        assert T_out.tolist() == exp_T and b_next.tolist() == exp_b
+
+
+@pytest.mark.parametrize("M,d,chunks", [(1, 5000, (16, 16)), (3, 12345, (8, 24, 5, 2)), (2, 70001, (64, 3, 33))])
+def test_statistics_accumulated_over_micro_batches(ctx, M, d, chunks):
+    """Gradient accumulation: the rows arrive in sub-batches, each goes through abs_test_stats and is
+    folded into a running (mean, record) pair; the result equals the statistics of the whole batch."""
+    b = sum(chunks)
+    G = make_G(400 + b, M, b, d, torch.float32, sigma=1.3)
+    run_mean = torch.empty((M, d), device="cuda")
+    run_rec = ctx.new_stats(M)
+    part_mean = torch.empty((M, d), device="cuda")
+    part_rec = ctx.new_stats(M)
+    lo = 0
+    for k, n in enumerate(chunks):
+        rows = G[:, lo:lo + n]
+        lo += n
+        if k == 0:
+            ctx.abs_test_stats(rows, run_rec, run_mean)
+        else:
+            ctx.abs_test_stats(rows, part_rec, part_mean)
+            ctx.abs_stats_merge(run_mean, part_mean, run_rec, part_rec)
+    torch.cuda.synchronize()
+    recs = pkg.stats_to_dicts(run_rec)
+    H = to_f64(G)
+    b_cur = torch.tensor([b], dtype=torch.int64, device="cuda")
+    b_next = torch.zeros(1, dtype=torch.int64, device="cuda")
+    T_out = torch.zeros(M, dtype=torch.int64, device="cuda")
+    for m in range(M):
+        ref = orc.batch_test_stats(H[m])
+        assert recs[m]["rows"] == b and recs[m]["status"] == pkg.binding.STATUS_NORM_ONLY
+        for key in ("gbar_sq", "var_norm", "sum_sq"):
+            assert recs[m][key] == pytest.approx(ref[key], rel=1e-5)
+        np.testing.assert_allclose(run_mean[m].cpu().numpy(), ref["gbar"], rtol=1e-5,
+                                   atol=2e-6 * np.abs(ref["gbar"]).max())
+    # the merged records drive the norm test; the augmented test declines them
+    ctx.abs_next_batch(run_rec, pkg.make_test_cfg("norm", 1 << 20, eta=0.5), b_cur, b_next, T_out)
+    exp_b, exp_T = orc.next_batch(recs, b, 1 << 20, "norm", eta=0.5)
+    assert T_out.tolist() == exp_T and b_next.item() == exp_b
+    ctx.abs_next_batch(run_rec, pkg.make_test_cfg("aug_ip", 1 << 20, theta=0.5, nu=0.5), b_cur, b_next, T_out)
+    assert T_out.tolist() == [0] * M and b_next.item() == b
