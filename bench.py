@@ -205,6 +205,9 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
         sec = time_steps(torch, lambda i: ctx.local_sgd_step(X, grads[i % 2], 1e-3), 8, 3)
         out["sgd_step"] = dict(workload="M=8 d=124,439,808 fp32, 12 B/element", ms=sec * 1e3,
                                GBps=12.0 * M * d / sec / 1e9, frac_of_peak=12.0 * M * d / sec / 1e9 / peak)
+        sec = time_steps(torch, lambda i: ctx.local_shb_step(X, m1, grads[i % 2], 1e-3, 0.9, 1e-4), 8, 3)
+        out["shb_step"] = dict(workload="M=8 d=124,439,808 fp32, 20 B/element", ms=sec * 1e3,
+                               GBps=20.0 * M * d / sec / 1e9, frac_of_peak=20.0 * M * d / sec / 1e9 / peak)
         sec = time_steps(torch, lambda i: ctx.replica_average(X), 8, 3)
         out["replica_average"] = dict(workload="stand-alone, 8 B/element/replica", ms=sec * 1e3,
                                       GBps=8.0 * M * d / sec / 1e9, frac_of_peak=8.0 * M * d / sec / 1e9 / peak)
