@@ -174,9 +174,43 @@ __global__ void bias_grad_kernel(const float* __restrict__ scratch, long long pe
   Gb[m * d + ob + o] = static_cast<float>(acc / static_cast<double>(b));
 }
 
-// Row i of G: the flat gradient of sample i of one worker.  One thread per parameter.
+// Row i of G: the flat gradient of sample i of one worker.  The weight segment of a layer is the
+// outer product delta_i (x) h_i: a thread writes 16 bytes (four consecutive inputs of one output
+// unit), so the kernel runs at the speed of the stores.  Needs n_in % 4 == 0 and 16-byte aligned
+// segment starts and rows; per_sample_rows_scalar_kernel covers everything else.
 __global__ void __launch_bounds__(256)
-per_sample_rows_kernel(const float* __restrict__ ws, const MlpShape s, float* __restrict__ G, long long row_stride) {
+per_sample_layer_kernel(const float* __restrict__ delta, const float* __restrict__ h, unsigned n_out, unsigned n_in,
+                        float* __restrict__ G, long long row_stride, long long seg_off) {
+  const long long i = blockIdx.y;
+  const unsigned quads = n_out * (n_in / 4u);
+  const float* di = delta + i * n_out;
+  const float4* hi = reinterpret_cast<const float4*>(h + i * n_in);
+  float4* out = reinterpret_cast<float4*>(G + i * row_stride + seg_off);
+  const unsigned q_in = n_in / 4u;
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const unsigned f = (blockIdx.x * 4u + u) * 256u + threadIdx.x;
+    if (f < quads) {
+      const unsigned o = f / q_in, k4 = f - o * q_in;
+      const float dv = __ldg(di + o);
+      const float4 hv = __ldg(hi + k4);
+      __stcs(out + f, make_float4(dv * hv.x, dv * hv.y, dv * hv.z, dv * hv.w));
+    }
+  }
+}
+
+// bias segments: G[i][seg_off + o] = delta[i][o]
+__global__ void per_sample_bias_kernel(const float* __restrict__ delta, unsigned n_out, float* __restrict__ G,
+                                       long long row_stride, long long seg_off) {
+  const long long i = blockIdx.y;
+  const unsigned o = blockIdx.x * blockDim.x + threadIdx.x;
+  if (o < n_out) G[i * row_stride + seg_off + o] = delta[i * n_out + o];
+}
+
+// Alignment-free variant: one thread per parameter.
+__global__ void __launch_bounds__(256)
+per_sample_rows_scalar_kernel(const float* __restrict__ ws, const MlpShape s, float* __restrict__ G,
+                              long long row_stride) {
   const long long i = blockIdx.y;
   const long long j = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (j >= s.d) return;
@@ -299,8 +333,27 @@ extern "C" int abs_mlp_per_sample(abs_ctx* ctx, const int* dims, long long b, in
   ABS_CUDA_TRY(ctx, cudaGetDevice(&prev));
   if (prev != ctx->device) ABS_CUDA_TRY(ctx, cudaSetDevice(ctx->device));
   const float* ws = static_cast<const float*>(scratch) + static_cast<long long>(worker) * s.per_worker;
-  const dim3 grid(static_cast<unsigned>((s.d + 255) / 256), static_cast<unsigned>(b));
-  per_sample_rows_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(ws, s, G, row_stride);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool vec = (s.n0 % 4 == 0) && (s.n1 % 4 == 0) && (s.n2 % 4 == 0) && (row_stride % 4 == 0) &&
+                   (s.oW2 % 4 == 0) && (s.oW3 % 4 == 0) && (s.per_worker % 4 == 0) && ((b * s.n0) % 4 == 0) &&
+                   ((b * s.n1) % 4 == 0) && ((b * s.n2) % 4 == 0) && ((b * s.n3) % 4 == 0) &&
+                   (reinterpret_cast<uintptr_t>(G) % 16 == 0) && (reinterpret_cast<uintptr_t>(ws) % 16 == 0);
+  if (vec) {
+    const unsigned rows = static_cast<unsigned>(b);
+    auto layer = [&](long long sD, long long sH, int n_out, int n_in, long long oW, long long ob) {
+      const unsigned quads = static_cast<unsigned>(n_out) * static_cast<unsigned>(n_in / 4);
+      per_sample_layer_kernel<<<dim3((quads + 1023) / 1024, rows), 256, 0, st>>>(
+          ws + sD, ws + sH, static_cast<unsigned>(n_out), static_cast<unsigned>(n_in), G, row_stride, oW);
+      per_sample_bias_kernel<<<dim3((n_out + 127) / 128, rows), 128, 0, st>>>(ws + sD, static_cast<unsigned>(n_out), G,
+                                                                             row_stride, ob);
+    };
+    layer(s.sD1, s.sX, s.n1, s.n0, s.oW1, s.ob1);
+    layer(s.sD2, s.sH1, s.n2, s.n1, s.oW2, s.ob2);
+    layer(s.sD3, s.sH2, s.n3, s.n2, s.oW3, s.ob3);
+  } else {
+    const dim3 grid(static_cast<unsigned>((s.d + 255) / 256), static_cast<unsigned>(b));
+    per_sample_rows_scalar_kernel<<<grid, 256, 0, st>>>(ws, s, G, row_stride);
+  }
   const cudaError_t e = cudaGetLastError();
   if (prev != ctx->device) cudaSetDevice(prev);
   if (e != cudaSuccess) return set_error(ctx, ABS_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
