@@ -430,7 +430,12 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
 int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if (a.b <= 256 || a.b > kMaxFastRows || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
   int C = 2;
-  const int want_rows = ctx->tuning.stats_cluster_rows > 0 ? static_cast<int>(ctx->tuning.stats_cluster_rows) : 256;
+  // Up to 2048 rows: at most 256 rows of 256 bytes per CTA.  Beyond: clusters of 8 with up to 512
+  // rows of 128 bytes (a cluster of 16 leaves too many SMs without a cluster; tried: 3.9 vs 4.6 TB/s
+  // at b = 4096).  Direct st.shared::cluster stores with cluster-scope fences instead of the bulk
+  // copies were also tried: 40 % slower.
+  const int want_rows = ctx->tuning.stats_cluster_rows > 0 ? static_cast<int>(ctx->tuning.stats_cluster_rows)
+                                                           : (a.b > 2048 ? 512 : 256);
   while (C < kMaxCluster && (a.b + C - 1) / C > want_rows) C *= 2;
   for (; C >= 2; C /= 2) {
     const int rc = try_cluster_size(ctx, a, C, P_out);
