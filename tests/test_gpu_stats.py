@@ -328,7 +328,26 @@ def _tiled_reference(small, d, b):
                 sum_sq=(b - 1) * V + b * N, status=0, gbar=A["gbar"])
 
 
+@pytest.mark.parametrize("b,d,offset,noise", [(64, 40000, 5.0, 0.01), (256, 9000, -300.0, 0.5), (1024, 3000, 2.0, 1e-3),
+                                              (20, 50000, 1e3, 1.0)])
+def test_mean_dominated_rows(ctx, b, d, offset, noise):
+    """Rows that are a large common vector plus small noise: the centred accumulation keeps the
+    variances at full accuracy although every entry is dominated by the mean."""
+    gen = torch.Generator().manual_seed(b + d)
+    common = offset * (1.0 + 0.1 * torch.randn(d, generator=gen))
+    G = (common + noise * torch.randn((1, b, d), generator=gen)).cuda()
+    recs, gbar = run_gpu(ctx, G)
+    ref = orc.batch_test_stats(to_f64(G)[0])
+    assert recs[0]["status"] == 0
+    assert recs[0]["gbar_sq"] == pytest.approx(ref["gbar_sq"], rel=1e-5)
+    assert recs[0]["var_norm"] == pytest.approx(ref["var_norm"], rel=1e-5)
+    assert recs[0]["var_ip"] == pytest.approx(ref["var_ip"], rel=1e-5)
+    assert abs(recs[0]["var_orth"] - ref["var_orth"]) <= 1e-5 * ref["var_norm"]
+    np.testing.assert_allclose(gbar[0].cpu().numpy(), ref["gbar"], rtol=1e-6)
+
+
 @pytest.mark.parametrize("dtype,M,b,d,d0", [(torch.float32, 1, 256, 11_200_000, 100_003),
+                                            (torch.float32, 1, 1024, 2_800_000, 50_003),
                                             (torch.bfloat16, 8, 16, 24_887_968, 250_007)])
 def test_full_size_launch_configuration(ctx, dtype, M, b, d, d0):
     # the benchmark's launch shape (same b, M, dtype; d as large as a test should hold), checked
