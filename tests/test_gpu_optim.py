@@ -120,3 +120,33 @@ def test_invalid_arguments(ctx):
         ctx.local_adamw_step(X, X.clone(), X.clone(), X.clone(), pkg.make_adamw_cfg(1e-3, 0.9, 0.95, 1e-8, 0.0, 0))
     with pytest.raises(pkg.AbsError):
         ctx.local_adamw_step(X, X.clone(), X.clone(), X.clone(), pkg.make_adamw_cfg(1e-3, 1.0, 0.95, 1e-8, 0.0, 1))
+
+
+def test_full_size_adamw_rounds_on_column_subsets(ctx):
+    """The fused local AdamW configuration at full size: M=8 fp32 replicas of d=124,439,808 parameters,
+    beta=(0.9, 0.95), wd=0.1, lr=3e-4, H=16 local steps per round with the averaging fused into the
+    last, 20 rounds.  The update is coordinate-separable, so the oracle follows three column subsets
+    (first, last and random 2^16 columns), restarted every round from the GPU's state."""
+    from paper_2406_13936_b200 import inputs
+    M, d, H, rounds, pool = 8, 124_439_808, 16, 20, 4
+    hp = dict(lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+    X, m1, m2, grads = inputs.adamw_problem(4, M, d, pool=pool, device="cuda")
+    gen = torch.Generator().manual_seed(1)
+    cols = torch.cat([torch.arange(0, 1 << 16), torch.arange(d - (1 << 16), d),
+                      torch.randint(0, d, (1 << 16,), generator=gen)]).cuda()
+    g_sub = [f64(g[:, cols]) for g in grads]
+    t = 0
+    for k in range(rounds):
+        xs, ms, vs = f64(X[:, cols]), f64(m1[:, cols]), f64(m2[:, cols])      # teacher forcing
+        for h in range(H):
+            t += 1
+            last = h == H - 1
+            ctx.local_adamw_step(X, m1, m2, grads[(t - 1) % pool], pkg.make_adamw_cfg(step=t, **hp),
+                                 average_after=last)
+            xs, ms, vs = orc.adamw_step(xs, ms, vs, g_sub[(t - 1) % pool], t=t, **hp)
+            if last:
+                xs = orc.replica_average(xs)
+        close(X[:, cols], xs)
+        close(m1[:, cols], ms)
+        close(m2[:, cols], vs)
+    assert torch.equal(X[0], X[M - 1])          # every replica holds the average after a round
