@@ -318,9 +318,21 @@ int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* labels, long lon
 int abs_mlp_per_sample(abs_ctx* ctx, const int* dims, long long b, int worker, const void* scratch,
                        float* G, long long row_stride, void* stream);
 
-/* One communication round of local SGD on the MLP problem, as abs_logreg_round; the
- * per-sample gradients are materialised for one worker at a time in G_scratch
- * [b][g_row_stride] at the last local step.  Gb_scratch [M][d].                     */
+/* The statistics of all M workers without forming the per-sample gradient matrix
+ * (a per-sample gradient of a layer is the outer product delta_i (x) h_i, so
+ * ||g_i||^2 = sum_l ||delta_l,i||^2 (||h_{l-1},i||^2 + 1) and
+ * <g_i, gbar> = sum_l delta_l,i^T (dW_l h_{l-1},i + db_l); Eq. def_var expanded):
+ * reads the activations and deltas a preceding abs_mlp_grads call with the same b
+ * and M left in `scratch` and the batch gradients Gb [M][d] it wrote; writes
+ * stats [M].  The expansion sum_i ||g_i||^2 - b N loses accuracy only when the
+ * variance is far below b N, i.e. when the test is satisfied by a wide margin.      */
+int abs_mlp_fused_stats(abs_ctx* ctx, const int* dims, long long b, int M, void* scratch,
+                        size_t scratch_bytes, const float* Gb, abs_stats* stats, void* stream);
+
+/* One communication round of local SGD on the MLP problem, as abs_logreg_round.  At
+ * the last local step the statistics come either from per-sample gradients
+ * materialised for one worker at a time in G_scratch [b][g_row_stride], or, when
+ * G_scratch is NULL, from abs_mlp_fused_stats.  Gb_scratch [M][d].                  */
 int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* labels, long long n, const int* dims,
                   const int* idx, long long idx_stride, float* X, int M, int H, long long b, float lr,
                   const abs_test_cfg* cfg, void* scratch, size_t scratch_bytes, float* G_scratch,

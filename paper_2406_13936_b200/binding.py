@@ -70,6 +70,8 @@ EXPORTS = {
                       ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p],
     "abs_mlp_per_sample": [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.c_longlong, ctypes.c_int,
                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p],
+    "abs_mlp_fused_stats": [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.c_longlong, ctypes.c_int,
+                            ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "abs_mlp_round": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
                       ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int,
                       ctypes.c_int, ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p,
@@ -299,6 +301,13 @@ class Context:
         self._check(self._lib.abs_mlp_per_sample(self._h, (ctypes.c_int * 4)(*dims), int(b), int(worker),
                                                  _ptr(scratch), _ptr(G), G.stride(0), _stream(stream)),
                     "abs_mlp_per_sample")
+
+    def abs_mlp_fused_stats(self, dims, b, scratch, Gb, stats, stream=None):
+        """Statistics of all workers from the scratch and the batch gradients of abs_mlp_grads."""
+        M = Gb.shape[0]
+        self._check(self._lib.abs_mlp_fused_stats(self._h, (ctypes.c_int * 4)(*dims), int(b), M, _ptr(scratch),
+                                                  scratch.numel(), _ptr(Gb), _ptr(stats), _stream(stream)),
+                    "abs_mlp_fused_stats")
 
     def abs_mlp_round(self, inputs_, labels, dims, idx, X, H, b, lr, cfg, scratch, G_scratch, g_row_stride,
                       Gb_scratch, stats, b_dev, T_out=None, stream=None):

@@ -6,16 +6,27 @@
 // Parameter layout of one replica (flat, fp32): W1 [n1][n0], b1 [n1], W2 [n2][n1], b2 [n2],
 // W3 [n3][n2], b3 [n3], each W row-major [out][in].
 // Scratch layout per worker (floats): Xin [b][n0], H1 [b][n1], H2 [b][n2], D3 [b][n3], D2 [b][n2],
-// D1 [b][n1].
+// D1 [b][n1], then work space of the fused statistics.
+//
+// Fused statistics (abs_mlp_fused_stats): the per-sample gradient of a layer is the outer product
+// delta_i (x) h_i (plus delta_i for the bias), so the two per-sample quantities the batch-size
+// test needs follow from activations and deltas without writing the b x d gradient matrix:
+//   ||g_i||^2    = sum_l ||delta_l,i||^2 (||h_{l-1},i||^2 + 1)
+//   <g_i, gbar>  = sum_l delta_l,i^T (dW_l h_{l-1},i + db_l)          (dW_l, db_l: the batch gradient)
+// and with N = ||gbar||^2:  sum_i ||g_i - gbar||^2 = sum_i ||g_i||^2 - b N  (Eq. def_var expanded),
+// Var_i <g_i, gbar> directly.  The expansions cancel only when the variance is far below b N,
+// i.e. when the test is satisfied by a wide margin anyway.
 #include "abs_internal.cuh"
 
 namespace absk {
 namespace {
 
+constexpr int kNormParts = 64;    // blocks per worker that sum ||gbar||^2
+
 struct MlpShape {
   int n0, n1, n2, n3;
   long long oW1, ob1, oW2, ob2, oW3, ob3, d;      // offsets into the flat parameter vector
-  long long sX, sH1, sH2, sD3, sD2, sD1, per_worker;   // offsets into a worker's scratch
+  long long sX, sH1, sH2, sD3, sD2, sD1, sU, sCQ, per_worker;   // offsets into a worker's scratch
 };
 
 MlpShape make_shape(const int* dims, long long b) {
@@ -34,7 +45,12 @@ MlpShape make_shape(const int* dims, long long b) {
   s.sD3 = s.sH2 + b * s.n2;
   s.sD2 = s.sD3 + b * s.n3;
   s.sD1 = s.sD2 + b * s.n2;
-  s.per_worker = (s.sD1 + b * s.n1 + 3) / 4 * 4;
+  // used by the fused statistics only: U [b][max width] products, then c_i, q_i [2][b] and 64 partial
+  // sums of ||gbar||^2 as doubles
+  const long long widest = s.n1 > s.n2 ? (s.n1 > s.n3 ? s.n1 : s.n3) : (s.n2 > s.n3 ? s.n2 : s.n3);
+  s.sU = (s.sD1 + b * s.n1 + 3) / 4 * 4;
+  s.sCQ = (s.sU + b * widest + 3) / 4 * 4;
+  s.per_worker = (s.sCQ + 2 * (2 * b + kNormParts) + 3) / 4 * 4;
   return s;
 }
 
@@ -234,6 +250,138 @@ per_sample_rows_scalar_kernel(const float* __restrict__ ws, const MlpShape s, fl
   G[i * row_stride + j] = v;
 }
 
+// ---- fused statistics ------------------------------------------------------------------------
+// One warp per sample: q_i += ||delta_i||^2 (||h_i||^2 + 1).
+__global__ void __launch_bounds__(256)
+fused_rownorm_kernel(float* __restrict__ scratch, long long per_worker, long long sD, long long sH, long long sCQ,
+                     long long b, int n_out, int n_in) {
+  const int m = blockIdx.y;
+  const long long i = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (i >= b) return;
+  const float* ws = scratch + m * per_worker;
+  const float* dl = ws + sD + i * n_out;
+  const float* hl = ws + sH + i * n_in;
+  float dn = 0.f, hn = 0.f;
+  for (int o = lane; o < n_out; o += 32) dn = fmaf(dl[o], dl[o], dn);
+  for (int k = lane; k < n_in; k += 32) hn = fmaf(hl[k], hl[k], hn);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    dn += __shfl_xor_sync(0xffffffffu, dn, off);
+    hn += __shfl_xor_sync(0xffffffffu, hn, off);
+  }
+  if (lane == 0) {
+    double* q = reinterpret_cast<double*>(scratch + m * per_worker + sCQ) + b;
+    q[i] += static_cast<double>(dn) * (static_cast<double>(hn) + 1.0);
+  }
+}
+
+// One warp per sample: c_i += sum_o delta_i[o] (U_i[o] + db[o]), U = h dW^T.
+__global__ void __launch_bounds__(256)
+fused_rowdot_kernel(float* __restrict__ scratch, long long per_worker, long long sD, long long sU, long long sCQ,
+                    long long b, int n_out, const float* __restrict__ Gb, long long d, long long ob) {
+  const int m = blockIdx.y;
+  const long long i = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (i >= b) return;
+  const float* ws = scratch + m * per_worker;
+  const float* dl = ws + sD + i * n_out;
+  const float* ul = ws + sU + i * n_out;
+  const float* db = Gb + m * d + ob;
+  float acc = 0.f;
+  for (int o = lane; o < n_out; o += 32) acc = fmaf(dl[o], ul[o] + db[o], acc);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (lane == 0) reinterpret_cast<double*>(scratch + m * per_worker + sCQ)[i] += static_cast<double>(acc);
+}
+
+// ||gbar||^2 of every worker in kNormParts partial sums, and c_i = q_i = 0.
+__global__ void __launch_bounds__(256)
+fused_norm_kernel(const float* __restrict__ Gb, long long d, float* __restrict__ scratch, long long per_worker,
+                  long long sCQ, long long b) {
+  __shared__ double red[8];
+  const int m = blockIdx.y, p = blockIdx.x, tid = threadIdx.x;
+  double* cq = reinterpret_cast<double*>(scratch + m * per_worker + sCQ);
+  for (long long i = static_cast<long long>(p) * 256 + tid; i < 2 * b; i += static_cast<long long>(kNormParts) * 256)
+    cq[i] = 0.0;
+  const float* g = Gb + m * d;
+  double acc = 0.0;
+  for (long long j0 = static_cast<long long>(p) * 1024; j0 < d; j0 += static_cast<long long>(kNormParts) * 1024) {
+    float a = 0.f;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long j = j0 + u * 256 + tid;
+      if (j < d) a = fmaf(g[j], g[j], a);
+    }
+    acc += static_cast<double>(a);
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if ((tid & 31) == 0) red[tid >> 5] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += red[w];
+    cq[2 * b + p] = t;
+  }
+}
+
+// One block per worker: abs_stats from c_i, q_i and N.
+__global__ void __launch_bounds__(1024)
+fused_finalize_kernel(const float* __restrict__ scratch, long long per_worker, long long sCQ, long long b,
+                      abs_stats* __restrict__ stats) {
+  __shared__ double red[3][32];
+  const int m = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const double* cq = reinterpret_cast<const double*>(scratch + m * per_worker + sCQ);
+  const double bd = static_cast<double>(b);
+  auto block_sum = [&](double v, int slot) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    if (lane == 0) red[slot][warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int w = 0; w < 32; ++w) t += red[slot][w];
+    __syncthreads();
+    return t;
+  };
+  double sc = 0.0, sq = 0.0;
+  for (long long i = tid; i < b; i += 1024) {
+    sc += cq[i];
+    sq += cq[b + i];
+  }
+  const double csum = block_sum(sc, 0);
+  const double qsum = block_sum(sq, 1);
+  const double cbar = csum / bd;
+  double sv = 0.0;
+  for (long long i = tid; i < b; i += 1024) {
+    const double e = cq[i] - cbar;
+    sv += e * e;
+  }
+  const double ss = block_sum(sv, 2);
+  if (tid == 0) {
+    double N = 0.0;
+    for (int p = 0; p < kNormParts; ++p) N += cq[2 * b + p];
+    double S = qsum - bd * N;                 // sum_i ||g_i - gbar||^2
+    if (S < 0.0) S = 0.0;
+    abs_stats o;
+    o.gbar_sq = N;
+    o.var_norm = S / (bd - 1.0);
+    o.var_ip = ss / (bd - 1.0);
+    o.var_orth = o.var_norm;
+    if (N > 0.0) {
+      o.var_orth = o.var_norm - o.var_ip / N;
+      if (o.var_orth < 0.0) o.var_orth = 0.0;
+    }
+    o.sum_sq = qsum;
+    o.rows = b;
+    o.status = 0u;
+    if (!(isfinite(qsum) && isfinite(N) && isfinite(ss))) o.status |= ABS_STATUS_NONFINITE;
+    if (N == 0.0) o.status |= ABS_STATUS_ZERO_MEAN;
+    o.reserved = 0u;
+    stats[m] = o;
+  }
+}
+
 int check_dims(abs_ctx* ctx, const int* dims) {
   if (dims == nullptr) return set_error(ctx, ABS_ERR_INVALID_ARG, "dims is null");
   for (int l = 0; l < 4; ++l)
@@ -360,6 +508,46 @@ extern "C" int abs_mlp_per_sample(abs_ctx* ctx, const int* dims, long long b, in
   return ABS_OK;
 }
 
+
+// Statistics of all M workers straight from the activations and deltas that abs_mlp_grads left in
+// `scratch` and from the batch gradients Gb it wrote: no per-sample gradient matrix is formed.
+extern "C" int abs_mlp_fused_stats(abs_ctx* ctx, const int* dims, long long b, int M, void* scratch,
+                                   size_t scratch_bytes, const float* Gb, abs_stats* stats, void* stream) {
+  if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
+  int rc = check_dims(ctx, dims);
+  if (rc != ABS_OK) return rc;
+  if (scratch == nullptr || Gb == nullptr || stats == nullptr || b < 2 || M < 1 || M > 65535)
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "need scratch, Gb, stats, b >= 2 and 1 <= M <= 65535");
+  const MlpShape s = make_shape(dims, b);
+  if (scratch_bytes < static_cast<size_t>(M) * s.per_worker * sizeof(float))
+    return set_error(ctx, ABS_ERR_WORKSPACE, "abs_mlp_fused_stats needs %zu scratch bytes, got %zu",
+                     static_cast<size_t>(M) * s.per_worker * sizeof(float), scratch_bytes);
+  int prev = -1;
+  ABS_CUDA_TRY(ctx, cudaGetDevice(&prev));
+  if (prev != ctx->device) ABS_CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* ws = static_cast<float*>(scratch);
+  const long long pw = s.per_worker, d = s.d;
+  const unsigned warp_blocks = static_cast<unsigned>((b * 32 + 255) / 256);
+  fused_norm_kernel<<<dim3(kNormParts, M), 256, 0, st>>>(Gb, d, ws, pw, s.sCQ, b);
+  auto layer = [&](long long sD, long long sH, int n_out, int n_in, long long oW, long long ob) {
+    fused_rownorm_kernel<<<dim3(warp_blocks, M), 256, 0, st>>>(ws, pw, sD, sH, s.sCQ, b, n_out, n_in);
+    // U[i][o] = sum_k h[i][k] dW[o][k]
+    GemmArgs g{ws + sH, n_in, 1, pw, Gb + oW, 1, n_in, d, ws + s.sU, n_out, pw, nullptr, 0, nullptr, 0, 0,
+               static_cast<int>(b), n_out, n_in, 1.f, 0};
+    launch_gemm(g, M, st);
+    fused_rowdot_kernel<<<dim3(warp_blocks, M), 256, 0, st>>>(ws, pw, sD, s.sU, s.sCQ, b, n_out, Gb, d, ob);
+  };
+  layer(s.sD1, s.sX, s.n1, s.n0, s.oW1, s.ob1);
+  layer(s.sD2, s.sH1, s.n2, s.n1, s.oW2, s.ob2);
+  layer(s.sD3, s.sH2, s.n3, s.n2, s.oW3, s.ob3);
+  fused_finalize_kernel<<<M, 1024, 0, st>>>(ws, pw, s.sCQ, b, stats);
+  const cudaError_t e = cudaGetLastError();
+  if (prev != ctx->device) cudaSetDevice(prev);
+  if (e != cudaSuccess) return set_error(ctx, ABS_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return ABS_OK;
+}
+
 // One communication round of local SGD on the MLP problem (Algorithm 2's structure, the
 // per-sample statistic of Algorithm 1 once per round on the last local step, one worker's
 // per-sample gradients materialised at a time).
@@ -369,7 +557,7 @@ extern "C" int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* label
                              long long g_row_stride, float* Gb_scratch, abs_stats* stats, long long* T_out,
                              long long* b_dev, void* stream) {
   if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
-  if (cfg == nullptr || G_scratch == nullptr || Gb_scratch == nullptr || stats == nullptr || b_dev == nullptr)
+  if (cfg == nullptr || Gb_scratch == nullptr || stats == nullptr || b_dev == nullptr)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
   if (H < 1 || b < 2) return set_error(ctx, ABS_ERR_INVALID_ARG, "need H >= 1 and b >= 2");
   int rc = check_dims(ctx, dims);
@@ -380,7 +568,10 @@ extern "C" int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* label
     rc = abs_mlp_grads(ctx, inputs, labels, n, dims, idx_h, idx_stride, X, M, b, Gb_scratch, scratch, scratch_bytes,
                        stream);
     if (rc != ABS_OK) return rc;
-    if (h == H - 1) {
+    if (h == H - 1 && G_scratch == nullptr) {
+      rc = abs_mlp_fused_stats(ctx, dims, b, M, scratch, scratch_bytes, Gb_scratch, stats, stream);
+      if (rc != ABS_OK) return rc;
+    } else if (h == H - 1) {
       for (int m = 0; m < M; ++m) {
         rc = abs_mlp_per_sample(ctx, dims, b, m, scratch, G_scratch, g_row_stride, stream);
         if (rc != ABS_OK) return rc;

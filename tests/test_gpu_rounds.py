@@ -145,14 +145,43 @@ def test_mlp_batch_and_per_sample_gradients(ctx, dims, M, b):
         assert torch.all(G[:, d:] == 0)          # the padding columns are left alone
 
 
-def run_mlp_rounds(ctx, dims, n, M, H, lr, b, b_max, rounds, check_rounds, theta=0.5, nu=0.5, seed=5):
+@pytest.mark.parametrize("dims,M,b", [((20, 33, 17, 7), 3, 9), ((70, 130, 65, 10), 2, 67),
+                                      ((784, 1024, 1024, 10), 2, 40), ((784, 1024, 1024, 10), 1, 600)])
+def test_mlp_fused_statistics_match_materialised_gradients(ctx, dims, M, b):
+    """Same activations, two routes: the statistics from outer-product identities against
+    abs_test_stats on the per-sample gradient rows written out."""
+    n = 5000
+    inp, lab, X = mlp_problem(5, n, dims, M)
+    X += 0.02 * torch.randn(X.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(9))
+    d = ctx.mlp_param_count(dims)
+    idx = inputs.batch_indices(6, (M, b), n, device="cuda")
+    scratch = ctx.mlp_scratch(M, b, dims)
+    Gb = torch.empty((M, d), device="cuda")
+    ctx.abs_mlp_grads(inp, lab, dims, idx, X, b, Gb, scratch)
+    fused = ctx.new_stats(M)
+    ctx.abs_mlp_fused_stats(dims, b, scratch, Gb, fused)
+    stride = (d + 3) // 4 * 4
+    G = torch.zeros((b, stride), device="cuda")
+    rows = ctx.new_stats(M)
+    for m in range(M):
+        ctx.abs_mlp_per_sample(dims, b, m, scratch, G)
+        ctx.abs_test_stats(G.unsqueeze(0)[:, :, :d], rows[m:m + 1])
+    torch.cuda.synchronize()
+    for f, r in zip(pkg.stats_to_dicts(fused), pkg.stats_to_dicts(rows)):
+        assert f["rows"] == r["rows"] == b and f["status"] == r["status"] == 0
+        for key in ("gbar_sq", "var_norm", "var_ip", "sum_sq"):
+            assert f[key] == pytest.approx(r[key], rel=2e-5)
+        assert abs(f["var_orth"] - r["var_orth"]) <= 2e-5 * r["var_norm"]
+
+
+def run_mlp_rounds(ctx, dims, n, M, H, lr, b, b_max, rounds, check_rounds, theta=0.5, nu=0.5, seed=5, fused=False):
     """Runs `rounds` rounds on the GPU; the first `check_rounds` are compared with the oracle."""
     inp, lab, X = mlp_problem(seed, n, dims, M)
     d = ctx.mlp_param_count(dims)
     stride = (d + 3) // 4 * 4
     idx = inputs.batch_indices(seed + 7, (rounds, H, M, b_max), n, device="cuda")
     scratch = ctx.mlp_scratch(M, b_max, dims)
-    G = torch.empty((b_max, stride), device="cuda")
+    G = None if fused else torch.empty((b_max, stride), device="cuda")
     Gb = torch.empty((M, d), device="cuda")
     stats = ctx.new_stats(M)
     T_out = torch.zeros(M, dtype=torch.int64, device="cuda")
@@ -192,9 +221,10 @@ def run_mlp_rounds(ctx, dims, n, M, H, lr, b, b_max, rounds, check_rounds, theta
     return X, history, (inp, lab)
 
 
-def test_mlp_rounds_small_network_teacher_forced(ctx):
+@pytest.mark.parametrize("fused", [False, True])
+def test_mlp_rounds_small_network_teacher_forced(ctx, fused):
     X, history, _ = run_mlp_rounds(ctx, (64, 48, 32, 10), n=4096, M=8, H=4, lr=0.05, b=8, b_max=512, rounds=12,
-                                   check_rounds=12)
+                                   check_rounds=12, fused=fused)
     assert history[-1] > history[0]
     assert torch.equal(X[0], X[7])
 
@@ -220,14 +250,15 @@ def mlp_loss(ctx, inp, lab, x, dims):
     return torch.nn.functional.cross_entropy(a, lab[:4096].long()).item()
 
 
-def test_end_to_end_mlp_200_rounds(ctx):
+@pytest.mark.parametrize("fused", [False, True])
+def test_end_to_end_mlp_200_rounds(ctx, fused):
     # 784-1024-1024-10, n = 1,048,576, M=8, H=4, augmented inner-product test, b from 32, cap 4096
     dims = (784, 1024, 1024, 10)
     inp, lab, X0 = mlp_problem(5, 1_048_576, dims, 1)
     loss0 = mlp_loss(ctx, inp, lab, X0[0], dims)
     del inp, lab, X0
     X, history, (inp, lab) = run_mlp_rounds(ctx, dims, n=1_048_576, M=8, H=4, lr=0.01, b=32, b_max=4096, rounds=200,
-                                            check_rounds=0)
+                                            check_rounds=0, fused=fused)
     assert all(x <= y_ for x, y_ in zip(history, history[1:]))
     assert history[-1] > history[0]
     assert torch.equal(X[0], X[7])
