@@ -237,6 +237,7 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
         torch.cuda.empty_cache()
     out["rounds_logreg"] = end_to_end_rounds(torch, pkg, inputs, ctx, "logreg")
     out["rounds_mlp"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp")
+    out["rounds_mlp_fused_stats"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp_fused")
     return out
 
 
@@ -258,7 +259,9 @@ def end_to_end_rounds(torch, pkg, inputs, ctx, which):
         cfg = pkg.make_test_cfg("aug_ip", b_max, theta=0.5, nu=0.5)
         stride = (d + 3) // 4 * 4
         scratch = ctx.mlp_scratch(M, b_max, dims)
-        G = torch.empty((b_max, stride), device="cuda")
+        # "mlp": per-sample gradient rows are written out and read by abs_test_stats;
+        # "mlp_fused": the statistics come from activations and deltas (abs_mlp_fused_stats)
+        G = torch.empty((b_max, stride), device="cuda") if which == "mlp" else None
     idx = inputs.batch_indices(11, (rounds, H, M, b_max), n, device="cuda")
     Gb = torch.empty((M, d), device="cuda")
     stats = ctx.new_stats(M)
