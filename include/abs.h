@@ -130,6 +130,29 @@ int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long lon
                    long long row_stride, long long worker_stride,
                    float* gbar_out, abs_stats* stats_out, void* stream);
 
+/* What abs_test_stats would launch for a shape: the host-side planning of the
+ * statistics kernels, exposed for inspection and for tests that need no GPU.
+ * aligned != 0 means base address and strides are multiples of 16 bytes.          */
+typedef struct {
+  int route;              /* 0 Gram (bf16, b <= 32), 1 cluster, 2 tiled, 3 generic two-sweep  */
+  int lanes_per_row;      /* 16-byte vectors per tile row: a tile row has 16*lanes_per_row bytes */
+  int warps_per_box;      /* consumer warps that share one box of rows                        */
+  int boxes_per_stage;
+  int stages;             /* tile buffers in the ring                                         */
+  int box_rows;           /* rows of one TMA box (<= 256)                                     */
+  int row_boxes;          /* boxes stacked to cover the rows of a tile                        */
+  int rows_per_thread;
+  int keep_in_registers;  /* the tile stays in registers between the two sweeps               */
+  int full;               /* every thread owns exactly rows_per_thread rows                   */
+  int cluster_size;       /* CTAs per cluster (1 outside the cluster route)                   */
+  int rows_per_cta;
+  unsigned stage_bytes;
+  unsigned reserved;
+  size_t smem_bytes;      /* dynamic shared memory per CTA                                    */
+} abs_stats_plan;
+int abs_plan_stats(abs_dtype dtype, long long b, int aligned, int sm_count, size_t smem_optin,
+                   abs_stats_plan* out);
+
 /* Same computation for HOST buffers: G_host is copied to a device buffer owned
  * by the context (grown on demand), the statistics are computed and copied back
  * to stats_host [M] and, if not NULL, gbar_host [M][d]; the call returns after

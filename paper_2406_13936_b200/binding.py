@@ -40,7 +40,16 @@ class Stats(ctypes.Structure):
                 ("status", ctypes.c_uint), ("reserved", ctypes.c_uint)]
 
 
+class StatsPlan(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_int) for name in
+                ("route", "lanes_per_row", "warps_per_box", "boxes_per_stage", "stages", "box_rows", "row_boxes",
+                 "rows_per_thread", "keep_in_registers", "full", "cluster_size", "rows_per_cta")] + \
+               [("stage_bytes", ctypes.c_uint), ("reserved", ctypes.c_uint), ("smem_bytes", ctypes.c_size_t)]
+
+
 EXPORTS = {
+    "abs_plan_stats": [ctypes.c_int, ctypes.c_longlong, ctypes.c_int, ctypes.c_int, ctypes.c_size_t,
+                       ctypes.POINTER(StatsPlan)],
     "abs_create": [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_size_t],
     "abs_destroy": [ctypes.c_void_p],
     "abs_set_tuning": [ctypes.c_void_p, ctypes.c_char_p, ctypes.c_longlong],
@@ -342,6 +351,17 @@ def abs_test_stats_noalloc(G, stats_out, gbar_out=None, stream=None):
     if rc != 0:
         raise AbsError("abs_test_stats_noalloc failed (%d): %s" % (rc, lib.abs_noalloc_last_error().decode()))
     return stats_out
+
+
+def plan_stats(dtype, b, aligned=True, sm_count=148, smem_optin=232448):
+    """The kernel and tile shape abs_test_stats would use for b rows of `dtype` ("f32" / "bf16"); needs no GPU."""
+    lib = load_library()
+    plan = StatsPlan()
+    rc = lib.abs_plan_stats({"f32": ABS_F32, "bf16": ABS_BF16}[dtype], int(b), int(bool(aligned)), int(sm_count),
+                            int(smem_optin), ctypes.byref(plan))
+    if rc != 0:
+        raise AbsError("abs_plan_stats failed (%d)" % rc)
+    return {name: getattr(plan, name) for name, _ in StatsPlan._fields_ if name != "reserved"}
 
 
 def _record_to_dict(r):

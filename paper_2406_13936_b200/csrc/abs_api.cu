@@ -165,6 +165,26 @@ extern "C" int abs_set_tuning(abs_ctx* ctx, const char* key, long long value) {
   return ABS_OK;
 }
 
+extern "C" int abs_plan_stats(abs_dtype dtype, long long b, int aligned, int sm_count, size_t smem_optin,
+                              abs_stats_plan* out) {
+  if (out == nullptr || b < 2 || (dtype != ABS_F32 && dtype != ABS_BF16) || sm_count < 1) return ABS_ERR_INVALID_ARG;
+  const Tuning t;     // the automatic choices
+  int rc = ABS_ERR_UNSUPPORTED;
+  if (aligned) {
+    rc = plan_stats_gram(t, smem_optin, dtype, b, out);
+    if (rc == ABS_ERR_UNSUPPORTED) rc = plan_stats_cluster(t, smem_optin, dtype, b, 0, out);
+    if (rc == ABS_ERR_UNSUPPORTED) rc = plan_stats_tiled(t, smem_optin, dtype, b, out);
+  }
+  if (rc == ABS_ERR_UNSUPPORTED) {
+    memset(out, 0, sizeof(*out));
+    out->route = 3;
+    out->cluster_size = 1;
+    out->rows_per_cta = static_cast<int>(b > 0x7fffffff ? 0x7fffffff : b);
+    rc = ABS_OK;
+  }
+  return rc;
+}
+
 extern "C" int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long long b, long long d,
                               long long row_stride, long long worker_stride, float* gbar_out, abs_stats* stats_out,
                               void* stream) {

@@ -85,4 +85,10 @@ int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out);   // 2
 int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
 int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P);
 
+// Host-side planning shared by the launchers and abs_plan_stats; ABS_OK or ABS_ERR_UNSUPPORTED.
+int plan_stats_gram(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out);
+int plan_stats_cluster(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, int cluster_size,
+                       abs_stats_plan* out);   // cluster_size 0: the preferred size
+int plan_stats_tiled(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out);
+
 }  // namespace absk

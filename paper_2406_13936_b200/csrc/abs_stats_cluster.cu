@@ -358,28 +358,59 @@ int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams 
 }
 
 // One attempt with a given cluster size; ABS_ERR_UNSUPPORTED if that size cannot be used.
-int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
-  const int es = a.dtype == ABS_F32 ? 4 : 2;
+struct ClusterGeom {
+  int RC, lpr_log2, RG, rmax, n_row_boxes, box_rows, stages, cols;
+  unsigned stage_bytes;
+  size_t smem;
+  bool full;
+};
+
+// Tile geometry of a cluster of C CTAs for b rows; false if that size cannot be used.
+bool cluster_geometry(const Tuning& t, size_t smem_optin, int es, long long b, int C, ClusterGeom* g) {
   const int ve = 16 / es;
-  const int RC = static_cast<int>((a.b + C - 1) / C);
-  if (RC > 512) return ABS_ERR_UNSUPPORTED;
-  const int lpr_log2 = RC <= 256 ? 4 : 3;                          // 256-byte rows; 128-byte for 257..512 rows
-  const int lpr = 1 << lpr_log2;
+  g->RC = static_cast<int>((b + C - 1) / C);
+  if (g->RC > 512) return false;
+  g->lpr_log2 = g->RC <= 256 ? 4 : 3;                       // 256-byte rows; 128-byte for 257..512 rows
+  const int lpr = 1 << g->lpr_log2;
   const int subs = 32 / lpr;
-  const int RG = kCW * subs;
-  const int R = (RC + RG - 1) / RG;                                // rows per thread, <= 16
-  const int rmax = R;
-  const int n_row_boxes = (RC + 255) / 256;
-  const int box_rows = (RC + n_row_boxes - 1) / n_row_boxes;
-  const int rows_pad = box_rows * n_row_boxes;
-  const unsigned stage_bytes = static_cast<unsigned>(rows_pad) * lpr * 16u;
-  const int cols = lpr * ve;
-  const size_t extras = static_cast<size_t>(2 * kCW * cols + kDepth * kMaxCluster * cols) * 4 +
-                        static_cast<size_t>(RC) * 8 + 2 * kCW * 8 + kDepth * 8 + 16 + 128;
-  int stages = static_cast<int>(ctx->tuning.stats_stages > 0 ? ctx->tuning.stats_stages : 4);
-  while (stages > 2 && stages * static_cast<size_t>(stage_bytes) + extras + stages * 8 > ctx->smem_optin) --stages;
-  const size_t smem = stages * static_cast<size_t>(stage_bytes) + extras + stages * 8;
-  if (smem > ctx->smem_optin) return ABS_ERR_UNSUPPORTED;
+  g->RG = kCW * subs;
+  g->rmax = (g->RC + g->RG - 1) / g->RG;                    // rows per thread, <= 16
+  g->n_row_boxes = (g->RC + 255) / 256;
+  g->box_rows = (g->RC + g->n_row_boxes - 1) / g->n_row_boxes;
+  const int rows_pad = g->box_rows * g->n_row_boxes;
+  g->stage_bytes = static_cast<unsigned>(rows_pad) * lpr * 16u;
+  g->cols = lpr * ve;
+  const size_t extras = static_cast<size_t>(2 * kCW * g->cols + kDepth * kMaxCluster * g->cols) * 4 +
+                        static_cast<size_t>(g->RC) * 8 + 2 * kCW * 8 + kDepth * 8 + 16 + 128;
+  g->stages = static_cast<int>(t.stats_stages > 0 ? t.stats_stages : 4);
+  while (g->stages > 2 && g->stages * static_cast<size_t>(g->stage_bytes) + extras + g->stages * 8 > smem_optin)
+    --g->stages;
+  g->smem = g->stages * static_cast<size_t>(g->stage_bytes) + extras + g->stages * 8;
+  if (g->smem > smem_optin) return false;
+  g->full = (b % C == 0) && (g->RC % g->RG == 0) && (g->rmax == 8 || g->rmax == 16);
+  return true;
+}
+
+// Up to 2048 rows: at most 256 rows of 256 bytes per CTA.  Beyond: clusters of 8 with up to 512
+// rows of 128 bytes (a cluster of 16 leaves too many SMs without a cluster; tried: 3.9 vs 4.6 TB/s
+// at b = 4096).  Direct st.shared::cluster stores with cluster-scope fences instead of the bulk
+// copies were also tried: 40 % slower.
+int preferred_cluster_size(const Tuning& t, long long b) {
+  const int want_rows = t.stats_cluster_rows > 0 ? static_cast<int>(t.stats_cluster_rows) : (b > 2048 ? 512 : 256);
+  int C = 2;
+  while (C < kMaxCluster && (b + C - 1) / C > want_rows) C *= 2;
+  return C;
+}
+
+// One attempt with a given cluster size; ABS_ERR_UNSUPPORTED if that size cannot be used.
+int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
+  ClusterGeom geo;
+  if (!cluster_geometry(ctx->tuning, ctx->smem_optin, a.dtype == ABS_F32 ? 4 : 2, a.b, C, &geo))
+    return ABS_ERR_UNSUPPORTED;
+  const int RC = geo.RC, lpr_log2 = geo.lpr_log2, rmax = geo.rmax, n_row_boxes = geo.n_row_boxes;
+  const int box_rows = geo.box_rows, stages = geo.stages, cols = geo.cols;
+  const unsigned stage_bytes = geo.stage_bytes;
+  const size_t smem = geo.smem;
 
   CUtensorMap tmap;
   int rc = encode_g_tensor_map(ctx, a, cols, box_rows, &tmap);
@@ -401,7 +432,7 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
-  const bool full = (a.b % C == 0) && (RC % RG == 0) && (rmax == 8 || rmax == 16);
+  const bool full = geo.full;
 #define ABS_CLUSTER_CASE(T, R) \
   case R: return launch_cluster_variant<T, R, false>(ctx, tmap, prm, a, C, smem, P_out);
 #define ABS_CLUSTER_DISPATCH(T)                                                                        \
@@ -429,19 +460,35 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
 // smaller clusters when the larger one cannot be scheduled.
 int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if (a.b <= 256 || a.b > kMaxFastRows || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
-  int C = 2;
-  // Up to 2048 rows: at most 256 rows of 256 bytes per CTA.  Beyond: clusters of 8 with up to 512
-  // rows of 128 bytes (a cluster of 16 leaves too many SMs without a cluster; tried: 3.9 vs 4.6 TB/s
-  // at b = 4096).  Direct st.shared::cluster stores with cluster-scope fences instead of the bulk
-  // copies were also tried: 40 % slower.
-  const int want_rows = ctx->tuning.stats_cluster_rows > 0 ? static_cast<int>(ctx->tuning.stats_cluster_rows)
-                                                           : (a.b > 2048 ? 512 : 256);
-  while (C < kMaxCluster && (a.b + C - 1) / C > want_rows) C *= 2;
-  for (; C >= 2; C /= 2) {
+  for (int C = preferred_cluster_size(ctx->tuning, a.b); C >= 2; C /= 2) {
     const int rc = try_cluster_size(ctx, a, C, P_out);
     if (rc != ABS_ERR_UNSUPPORTED) return rc;
   }
   return ABS_ERR_UNSUPPORTED;
+}
+
+int plan_stats_cluster(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, int cluster_size,
+                       abs_stats_plan* out) {
+  if (b <= 256 || b > kMaxFastRows) return ABS_ERR_UNSUPPORTED;
+  const int C = cluster_size > 0 ? cluster_size : preferred_cluster_size(t, b);
+  ClusterGeom g;
+  if (!cluster_geometry(t, smem_optin, dtype == ABS_F32 ? 4 : 2, b, C, &g)) return ABS_ERR_UNSUPPORTED;
+  memset(out, 0, sizeof(*out));
+  out->route = 1;
+  out->lanes_per_row = 1 << g.lpr_log2;
+  out->warps_per_box = kCW;
+  out->boxes_per_stage = 1;
+  out->stages = g.stages;
+  out->box_rows = g.box_rows;
+  out->row_boxes = g.n_row_boxes;
+  out->rows_per_thread = g.rmax;
+  out->keep_in_registers = 1;
+  out->full = g.full ? 1 : 0;
+  out->cluster_size = C;
+  out->rows_per_cta = g.RC;
+  out->stage_bytes = g.stage_bytes;
+  out->smem_bytes = g.smem;
+  return ABS_OK;
 }
 
 }  // namespace absk

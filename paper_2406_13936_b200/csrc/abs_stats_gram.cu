@@ -278,6 +278,28 @@ int launch_gram_variant(abs_ctx* ctx, const CUtensorMap& tmap, const GramParams&
 
 }  // namespace
 
+int plan_stats_gram(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out) {
+  if (dtype != ABS_BF16 || b < 2 || b > 32) return ABS_ERR_UNSUPPORTED;
+  const int NB = b <= 16 ? 1 : 2;
+  const unsigned box_bytes = static_cast<unsigned>(16 * NB) * static_cast<unsigned>(box_cols_for(NB)) * 2u;
+  int stages = static_cast<int>(t.stats_stages > 0 ? t.stats_stages : 3);
+  while (stages > 2 && static_cast<size_t>(stages) * box_bytes * kWarpsC + 1024 > smem_optin) --stages;
+  memset(out, 0, sizeof(*out));
+  out->route = 0;
+  out->lanes_per_row = box_cols_for(NB) / 8;
+  out->warps_per_box = 1;
+  out->boxes_per_stage = kWarpsC;
+  out->stages = stages;
+  out->box_rows = static_cast<int>(b);
+  out->row_boxes = 1;
+  out->rows_per_thread = 0;
+  out->cluster_size = 1;
+  out->rows_per_cta = static_cast<int>(b);
+  out->stage_bytes = box_bytes * kWarpsC;
+  out->smem_bytes = static_cast<size_t>(stages) * box_bytes * kWarpsC + 1024;
+  return ABS_OK;
+}
+
 int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if (a.dtype != ABS_BF16 || a.b > 32 || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
   const int NB = a.b <= 16 ? 1 : 2;

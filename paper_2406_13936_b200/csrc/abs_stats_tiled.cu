@@ -363,6 +363,16 @@ bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, 
   return false;
 }
 
+// The tile shape for b rows: two resident CTAs per SM with 32 KiB tile buffers and 8 rows per
+// thread, or (default) one CTA with 64 KiB buffers and 16 rows per thread.
+bool tiled_choice(const Tuning& t, size_t smem_optin, int ve, long long b, TileChoice* c) {
+  const int per_sm = t.stats_ctas_per_sm > 0 ? static_cast<int>(t.stats_ctas_per_sm) : 1;
+  const size_t stage_max = t.stats_stage_kb > 0 ? static_cast<size_t>(t.stats_stage_kb) << 10
+                                                : (per_sm == 2 ? (32u << 10) : (64u << 10));
+  return choose_tile(b, ve, smem_optin, t.stats_stages, stage_max, per_sm == 2 ? 8 : 16, c) ||
+         choose_tile(b, ve, smem_optin, t.stats_stages, 64u << 10, 16, c);
+}
+
 template <typename T, int RMAX, bool KEEP, bool FULL>
 int launch_variant(abs_ctx* ctx, const CUtensorMap& tmap, const TiledParams& prm, dim3 grid, size_t smem,
                    cudaStream_t stream) {
@@ -401,20 +411,35 @@ int launch_typed(abs_ctx* ctx, const TileChoice& c, const CUtensorMap& tmap, con
 
 }  // namespace
 
+int plan_stats_tiled(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out) {
+  if (b < 2 || b > kMaxFastRows) return ABS_ERR_UNSUPPORTED;
+  TileChoice c;
+  if (!tiled_choice(t, smem_optin, dtype == ABS_F32 ? 4 : 8, b, &c)) return ABS_ERR_UNSUPPORTED;
+  memset(out, 0, sizeof(*out));
+  out->route = 2;
+  out->lanes_per_row = 1 << c.lpr_log2;
+  out->warps_per_box = 1 << c.rs_log2;
+  out->boxes_per_stage = c.bx;
+  out->stages = c.stages;
+  out->box_rows = c.box_rows;
+  out->row_boxes = c.n_row_boxes;
+  out->rows_per_thread = c.rmax;
+  out->keep_in_registers = c.keep ? 1 : 0;
+  out->full = c.full ? 1 : 0;
+  out->cluster_size = 1;
+  out->rows_per_cta = static_cast<int>(b);
+  out->stage_bytes = c.stage_bytes;
+  out->smem_bytes = c.smem_bytes;
+  return ABS_OK;
+}
+
 int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   const int es = a.dtype == ABS_F32 ? 4 : 2;
   const int ve = 16 / es;
   if (a.b > kMaxFastRows || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
 
   TileChoice c;
-  // two resident CTAs per SM with 32 KiB tile buffers and 8 rows per thread, or one CTA with 64 KiB
-  // buffers and 16 rows per thread
-  const int per_sm = ctx->tuning.stats_ctas_per_sm > 0 ? static_cast<int>(ctx->tuning.stats_ctas_per_sm) : 1;
-  const size_t stage_max = ctx->tuning.stats_stage_kb > 0 ? static_cast<size_t>(ctx->tuning.stats_stage_kb) << 10
-                                                          : (per_sm == 2 ? (32u << 10) : (64u << 10));
-  if (!choose_tile(a.b, ve, ctx->smem_optin, ctx->tuning.stats_stages, stage_max, per_sm == 2 ? 8 : 16, &c) &&
-      !choose_tile(a.b, ve, ctx->smem_optin, ctx->tuning.stats_stages, 64u << 10, 16, &c))
-    return ABS_ERR_UNSUPPORTED;
+  if (!tiled_choice(ctx->tuning, ctx->smem_optin, ve, a.b, &c)) return ABS_ERR_UNSUPPORTED;
 
   const int lpr = 1 << c.lpr_log2;
   const long long box_cols = static_cast<long long>(lpr) * ve;
