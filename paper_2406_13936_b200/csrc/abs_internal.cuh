@@ -14,8 +14,8 @@ namespace absk {
 
 constexpr int kSmCountFallback = 148;
 constexpr size_t kDefaultWorkspace = 64ull << 20;
-constexpr int kMaxFastRows = 4096;
-constexpr long long kDefaultTimeoutCycles = 4000000000ll;   // about two seconds of SM clock          // largest b the tiled statistics kernel covers
+constexpr int kMaxFastRows = 4096;                          // largest b the tiled and cluster kernels cover
+constexpr long long kDefaultTimeoutCycles = 4000000000ll;   // about two seconds of SM clock
 
 struct Tuning {
   long long stats_stages = 0;
