@@ -49,7 +49,10 @@ int run_stats(abs_ctx* ctx, const StatsLaunch& a) {
   // of the previous call cleared it again after reading it.
   int P = 0;
   int rc = ABS_ERR_UNSUPPORTED;
-  if (!ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_gram) rc = launch_stats_gram(ctx, a, &P);
+  if (!ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_gram) {
+    rc = launch_stats_gram(ctx, a, &P);
+    if (rc == ABS_ERR_UNSUPPORTED) rc = launch_stats_umma(ctx, a, &P);
+  }
   if (rc == ABS_ERR_UNSUPPORTED && !ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_cluster)
     rc = launch_stats_cluster(ctx, a, &P);
   if (rc == ABS_ERR_UNSUPPORTED && !ctx->tuning.stats_force_generic) rc = launch_stats_tiled(ctx, a, &P);
@@ -172,6 +175,7 @@ extern "C" int abs_plan_stats(abs_dtype dtype, long long b, int aligned, int sm_
   int rc = ABS_ERR_UNSUPPORTED;
   if (aligned) {
     rc = plan_stats_gram(t, smem_optin, dtype, b, out);
+    if (rc == ABS_ERR_UNSUPPORTED) rc = plan_stats_umma(t, smem_optin, dtype, b, out);
     if (rc == ABS_ERR_UNSUPPORTED) rc = plan_stats_cluster(t, smem_optin, dtype, b, 0, out);
     if (rc == ABS_ERR_UNSUPPORTED) rc = plan_stats_tiled(t, smem_optin, dtype, b, out);
   }

@@ -81,12 +81,14 @@ struct StatsLaunch {
 // (alignment, b too large); *P_out receives the number of partial records per worker.
 int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
 int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // bf16, b <= 32
+int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // bf16, 32 < b <= 128 (tcgen05)
 int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out);   // 256 < b <= 4096
 int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
 int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P);
 
 // Host-side planning shared by the launchers and abs_plan_stats; ABS_OK or ABS_ERR_UNSUPPORTED.
 int plan_stats_gram(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out);
+int plan_stats_umma(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out);
 int plan_stats_cluster(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, int cluster_size,
                        abs_stats_plan* out);   // cluster_size 0: the preferred size
 int plan_stats_tiled(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out);

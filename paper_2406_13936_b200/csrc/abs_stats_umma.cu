@@ -1,0 +1,429 @@
+// Gram-matrix statistics kernel for bf16 rows and 32 < b <= 128 on the tcgen05 tensor cores, sm_100a.
+//
+// As in the small-batch Gram kernel, K = G G^T carries everything the batch-size test needs
+// (Eq. batch_grad and Eq. def_var expanded):
+//   N = 1^T K 1 / b^2,  c_i = (K 1)_i / b,  sum_i ||g_i - gbar||^2 = tr K - 1^T K 1 / b.
+// The CUDA-core route needs about six instructions per bf16 element and stalls near 4 TB/s for
+// these batch sizes; a 128 x b x 16 tcgen05.mma takes the 4 KiB it consumes off the critical path.
+// Products of two bf16 values are exact in fp32; the tensor core adds them in fp32 over
+// kFoldTiles * 256 columns in TMEM, then four warps read the accumulator back (tcgen05.ld),
+// reduce each row to (K 1)_i and K_ii and add those to fp64 registers, which is where the
+// cancellation in c_i - N happens.  Two accumulators alternate, so the read-back overlaps the
+// next fold's MMAs.
+//
+// Operands: both A and B are the same shared-memory tile (K-major, 128-byte swizzle): rows of G,
+// 64 columns per k-block, four k-blocks per stage.  A tensor-map copy into that layout is limited
+// to 128-byte box rows, which the copy engine serves at about two thirds of the HBM rate, so the
+// tile is filled by four loader warps with 16-byte cp.async copies (a warp covers 512 contiguous
+// bytes of one row) that apply the swizzle themselves.  A k-block holds ceil8(b) rows; the A
+// descriptor always spans 128 rows and the B descriptor ceil16(b), so both may run into the next
+// k-block: what they pick up there lands in rows / columns >= b of K, which nobody reads.
+//
+// Warp roles: 0-3 loaders, 4-7 accumulator read-back (warp w owns TMEM lanes 32 (w % 4) ..),
+// 8 MMA issue and TMEM allocation, 9-12 column means on the CUDA cores when gbar is wanted.
+// Every wait is bounded; a wait that runs out raises the CTA's abort flag, every role falls
+// through its loop, TMEM is freed and the records come back flagged ABS_STATUS_TIMEOUT.
+#include <cuda_bf16.h>
+
+#include "abs_pipeline.cuh"
+
+namespace absk {
+namespace {
+
+constexpr int kLoadWarps = 4;
+constexpr int kTileCols = 256;       // columns per stage: four k-blocks of 64 (128-byte swizzle span)
+constexpr int kFoldTiles = 4;        // stages accumulated in TMEM before the fold into fp64
+constexpr int kMaxStagesU = 8;
+constexpr int kBarsU = 2 * kMaxStagesU + 5;
+
+struct UmmaParams {
+  const __nv_bfloat16* G;
+  long long b, d, row_stride, worker_stride;   // strides in elements
+  int n_dim;              // ceil16(b): N of the MMA
+  int acc_cols;           // TMEM columns per accumulator (n_dim rounded up to a power of two >= 32)
+  int stages;
+  int lag;                // copy groups a loader keeps in flight
+  unsigned kb_bytes;      // ceil8(b) * 128
+  unsigned stage_bytes;   // 4 k-blocks
+  long long n_tiles;
+  int P;
+  double* ws;
+  float* gbar_out;
+  unsigned* flags;
+  long long timeout_cycles;
+};
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait(int pending) {
+  switch (pending) {
+    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+  }
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major operand, 128-byte swizzle: 8-row groups 1024 bytes apart; version 1 (sm_100).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  return static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// D (fp32, TMEM) (+)= A (bf16, smem) * B^T (bf16, smem); issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+}
+
+template <bool WANT_GBAR>
+__global__ void __launch_bounds__(WANT_GBAR ? 416 : 288, 1)
+abs_stats_umma_kernel(const UmmaParams prm) {
+  extern __shared__ unsigned char smem_dyn[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m = blockIdx.y, p = blockIdx.x;
+  const int b = static_cast<int>(prm.b);
+  const int S = prm.stages;
+
+  // the swizzle is a function of the address: k-blocks start on 1024-byte boundaries
+  const uint32_t raw_u32 = smem_u32(smem_dyn);
+  const uint32_t ring_u32 = (raw_u32 + 1023u) & ~1023u;
+  unsigned char* ring = smem_dyn + (ring_u32 - raw_u32);
+  const uint32_t pad = (128u - prm.kb_bytes / 128u) * 128u;       // room the 128-row A descriptor may run into
+  unsigned char* tail = ring + static_cast<size_t>(S) * prm.stage_bytes + pad;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);
+  volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + kBarsU);
+  unsigned* tmem_slot = const_cast<unsigned*>(abort_flag) + 1;
+  double* red = reinterpret_cast<double*>(bars + kBarsU + 1);     // [128] row sums, [128] diagonal, [2]
+  const uint32_t full_u32 = smem_u32(bars);
+  const uint32_t empty_u32 = full_u32 + 8u * kMaxStagesU;
+  const uint32_t accfull_u32 = empty_u32 + 8u * kMaxStagesU;      // 2
+  const uint32_t accempty_u32 = accfull_u32 + 16u;                // 2
+  const uint32_t done_u32 = accempty_u32 + 16u;                   // 1
+
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_u32 + 8u * s, kLoadWarps);
+      mbar_init(empty_u32 + 8u * s, WANT_GBAR ? 5 : 1);
+    }
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(accfull_u32 + 8u * k, 1);
+      mbar_init(accempty_u32 + 8u * k, 128);
+    }
+    mbar_init(done_u32, 1);
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  const uint32_t tmem_cols = static_cast<uint32_t>(2 * prm.acc_cols);
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const long long n_mine = (prm.n_tiles > p) ? (prm.n_tiles - p + prm.P - 1) / prm.P : 0;
+  const __nv_bfloat16* Gm = prm.G + static_cast<long long>(m) * prm.worker_stride;
+  double row_sum = 0.0, row_diag = 0.0;
+
+  if (warp < kLoadWarps) {
+    // ---- loaders: 16-byte chunk c of the tile = row c / 32, chunk c % 32 of its 512 bytes ----
+    const int n_chunks = b * 32;
+    const int lag = prm.lag;
+    for (long long i = 0; i < n_mine; ++i) {
+      const int s = static_cast<int>(i % S);
+      const long long use = i / S;
+      if (use > 0) mbar_wait(empty_u32 + 8u * s, static_cast<uint32_t>((use - 1) & 1), abort_flag, prm.timeout_cycles);
+      const long long col0 = (p + i * prm.P) * kTileCols;
+      const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes;
+      for (int c = tid; c < n_chunks; c += kLoadWarps * 32) {
+        const int row = c >> 5, ch = c & 31;
+        const long long col = col0 + ch * 8;
+        const long long left = prm.d - col;                         // elements of this row from col on
+        const uint32_t bytes = left >= 8 ? 16u : (left > 0 ? static_cast<uint32_t>(left) * 2u : 0u);
+        const __nv_bfloat16* src = Gm + static_cast<long long>(row) * prm.row_stride + (left > 0 ? col : 0);
+        const uint32_t dst = stage + static_cast<uint32_t>(ch >> 3) * prm.kb_bytes + static_cast<uint32_t>(row) * 128u +
+                             (static_cast<uint32_t>((ch & 7) ^ (row & 7)) << 4);
+        cp_async_16(dst, src, bytes);                               // bytes past `bytes` are zero-filled
+      }
+      cp_async_commit();
+      if (i >= lag) {
+        cp_async_wait(lag);                                         // tile i - lag has landed
+        fence_async_smem();                                         // ... and is visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_u32 + 8u * static_cast<uint32_t>((i - lag) % S));
+      }
+    }
+    cp_async_wait(0);
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0)
+      for (long long i = (n_mine > lag ? n_mine - lag : 0); i < n_mine; ++i)
+        mbar_arrive(full_u32 + 8u * static_cast<uint32_t>(i % S));
+  } else if (warp == 8) {
+    // ---- MMA issue ----
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(prm.n_dim >> 3) << 17) |
+                             (8u << 24);                            // fp32 accumulate, bf16 x bf16, K-major, M = 128
+      for (long long i = 0; i < n_mine; ++i) {
+        const int s = static_cast<int>(i % S);
+        const long long fold = i / kFoldTiles;
+        const int buf = static_cast<int>(fold & 1);
+        const bool first = (i % kFoldTiles) == 0;
+        if (first && fold >= 2)
+          mbar_wait(accempty_u32 + 8u * buf, static_cast<uint32_t>((fold / 2 - 1) & 1), abort_flag, prm.timeout_cycles);
+        mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>((i / S) & 1), abort_flag, prm.timeout_cycles);
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.acc_cols);
+        const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes;
+#pragma unroll
+        for (int kb = 0; kb < 4; ++kb) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t desc = umma_desc(stage + static_cast<uint32_t>(kb) * prm.kb_bytes + static_cast<uint32_t>(k) * 32u);
+            umma_bf16(d_tmem, desc, desc, idesc, (first && kb == 0 && k == 0) ? 0u : 1u);
+          }
+        }
+        umma_commit(empty_u32 + 8u * s);                            // the stage may be refilled
+        if ((i % kFoldTiles) == kFoldTiles - 1 || i == n_mine - 1) umma_commit(accfull_u32 + 8u * buf);
+      }
+      umma_commit(done_u32);
+      volatile unsigned ignore = 0u;
+      mbar_wait(done_u32, 0u, &ignore, prm.timeout_cycles);         // no MMA in flight when TMEM is freed
+    }
+    __syncwarp();
+  } else if (warp < 8) {
+    // ---- accumulator read-back: this thread owns row i = 32 (warp % 4) + lane of K ----
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const long long n_folds = (n_mine + kFoldTiles - 1) / kFoldTiles;
+    for (long long f = 0; f < n_folds; ++f) {
+      const int buf = static_cast<int>(f & 1);
+      mbar_wait(accfull_u32 + 8u * buf, static_cast<uint32_t>((f / 2) & 1), abort_flag, prm.timeout_cycles);
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + static_cast<uint32_t>(buf * prm.acc_cols) + (static_cast<uint32_t>(q * 32) << 16);
+      float diag = 0.f;
+      for (int c0 = 0; c0 < prm.n_dim; c0 += 16) {
+        float v[16];
+        tmem_ld16(taddr + static_cast<uint32_t>(c0), v);
+        float part = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          part += (c0 + j < b) ? v[j] : 0.f;
+          diag = (c0 + j == row) ? v[j] : diag;
+        }
+        row_sum += static_cast<double>(part);
+      }
+      row_diag += static_cast<double>(diag);
+      tc_fence_before();
+      mbar_arrive(accempty_u32 + 8u * buf);
+    }
+  } else if (WANT_GBAR) {
+    // ---- column means on the CUDA cores: warp 9 + kb owns k-block kb; lane = (row phase, 16-byte chunk) ----
+    const int kb = warp - 9;
+    const int sub = lane >> 3, ch = lane & 7;
+    const float inv_b = 1.0f / static_cast<float>(b);
+    for (long long i = 0; i < n_mine; ++i) {
+      const int s = static_cast<int>(i % S);
+      mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>((i / S) & 1), abort_flag, prm.timeout_cycles);
+      const uint32_t base = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(kb) * prm.kb_bytes;
+      float cs[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) cs[j] = 0.f;
+      for (int r = sub; r < b; r += 4) {
+        const uint4 u = lds128(base + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>(ch ^ (r & 7)) << 4));
+        float x[8];
+        Vec<__nv_bfloat16>::unpack(u, x);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cs[j] += x[j];
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 8);
+        cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 16);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_u32 + 8u * s);
+      if (sub == 0) {
+        const long long col = (p + i * prm.P) * kTileCols + kb * 64 + ch * 8;
+        float* dst = prm.gbar_out + static_cast<long long>(m) * prm.d + col;
+        if (col + 8 <= prm.d && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+          *reinterpret_cast<float4*>(dst) = make_float4(cs[0] * inv_b, cs[1] * inv_b, cs[2] * inv_b, cs[3] * inv_b);
+          *reinterpret_cast<float4*>(dst + 4) = make_float4(cs[4] * inv_b, cs[5] * inv_b, cs[6] * inv_b, cs[7] * inv_b);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (col + j < prm.d) dst[j] = cs[j] * inv_b;
+        }
+      }
+    }
+  }
+
+  // ---- CTA epilogue: (e_r, V, N) from the row sums and the diagonal of K ----
+  if (warp >= 4 && warp < 8) {
+    const int row = (warp & 3) * 32 + lane;
+    red[row] = row_sum;
+    red[128 + row] = row_diag;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+  if (tid == 0) {
+    double total = 0.0, trace = 0.0;
+    for (int i = 0; i < b; ++i) {
+      total += red[i];
+      trace += red[128 + i];
+    }
+    red[256] = total;
+    red[257] = trace;
+  }
+  __syncthreads();
+  {
+    const double bd = static_cast<double>(b);
+    const double total = red[256], trace = red[257];
+    const double Ncta = total / (bd * bd);
+    double* out = prm.ws + (static_cast<size_t>(m) * prm.P + p) * (static_cast<size_t>(b) + 2);
+    for (int i = tid; i < b; i += blockDim.x) out[i] = red[i] / bd - Ncta;     // sum_j (g_ij - gbar_j) gbar_j
+    if (tid == 0) {
+      out[b] = trace - total / bd;                                             // sum_ij (g_ij - gbar_j)^2
+      out[b + 1] = Ncta;
+      if (*abort_flag) atomicOr(prm.flags, 1u);
+    }
+  }
+}
+
+struct UmmaGeom {
+  int rows_blk, n_dim, acc_cols, stages, lag;
+  unsigned kb_bytes, stage_bytes;
+  size_t smem;
+};
+
+bool umma_geometry(const Tuning& t, size_t smem_optin, long long b, UmmaGeom* g) {
+  if (b <= 32 || b > 128) return false;
+  g->rows_blk = static_cast<int>((b + 7) / 8 * 8);
+  g->n_dim = static_cast<int>((b + 15) / 16 * 16);
+  g->acc_cols = g->n_dim <= 64 ? 64 : 128;
+  g->kb_bytes = static_cast<unsigned>(g->rows_blk) * 128u;
+  g->stage_bytes = 4u * g->kb_bytes;
+  const size_t pad = static_cast<size_t>(128 - g->rows_blk) * 128;
+  const size_t fixed = 1024 + pad + static_cast<size_t>(kBarsU + 1) * 8 + 258 * sizeof(double) + 128;
+  int stages = static_cast<int>(t.stats_stages > 0 ? t.stats_stages : kMaxStagesU);
+  if (stages > kMaxStagesU) stages = kMaxStagesU;
+  while (stages > 2 && static_cast<size_t>(stages) * g->stage_bytes + fixed > smem_optin) --stages;
+  g->stages = stages;
+  g->smem = static_cast<size_t>(stages) * g->stage_bytes + fixed;
+  if (g->smem > smem_optin) return false;
+  // copy groups in flight per loader: all but one stage, at most 4 (the tensor core works on the oldest)
+  g->lag = stages - 1 > 4 ? 4 : stages - 1;
+  return true;
+}
+
+template <bool WANT_GBAR>
+int launch_umma_variant(abs_ctx* ctx, const UmmaParams& prm, dim3 grid, size_t smem, cudaStream_t stream) {
+  auto kern = abs_stats_umma_kernel<WANT_GBAR>;
+  ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  kern<<<grid, WANT_GBAR ? 416 : 288, smem, stream>>>(prm);
+  ABS_CUDA_TRY(ctx, cudaGetLastError());
+  return ABS_OK;
+}
+
+}  // namespace
+
+int plan_stats_umma(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out) {
+  UmmaGeom g;
+  if (dtype != ABS_BF16 || !umma_geometry(t, smem_optin, b, &g)) return ABS_ERR_UNSUPPORTED;
+  memset(out, 0, sizeof(*out));
+  out->route = 4;
+  out->lanes_per_row = 8;                    // a k-block row: 128 bytes
+  out->warps_per_box = kLoadWarps;
+  out->boxes_per_stage = 4;                  // k-blocks
+  out->stages = g.stages;
+  out->box_rows = g.rows_blk;
+  out->row_boxes = 1;
+  out->rows_per_thread = 0;
+  out->cluster_size = 1;
+  out->rows_per_cta = static_cast<int>(b);
+  out->stage_bytes = g.stage_bytes;
+  out->smem_bytes = g.smem;
+  return ABS_OK;
+}
+
+// Takes the call for bf16 rows with 32 < b <= 128 whose base and strides are multiples of 16 bytes.
+int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
+  if (a.dtype != ABS_BF16) return ABS_ERR_UNSUPPORTED;
+  UmmaGeom g;
+  if (!umma_geometry(ctx->tuning, ctx->smem_optin, a.b, &g)) return ABS_ERR_UNSUPPORTED;
+  const unsigned long long row_b = static_cast<unsigned long long>(a.row_stride) * 2;
+  const unsigned long long wrk_b = static_cast<unsigned long long>(a.M > 1 ? a.worker_stride : 0) * 2;
+  if ((reinterpret_cast<uintptr_t>(a.G) & 15u) || (row_b & 15u) || (wrk_b & 15u) || a.M > 65535)
+    return ABS_ERR_UNSUPPORTED;
+
+  const long long n_tiles = (a.d + kTileCols - 1) / kTileCols;
+  long long P = ctx->tuning.stats_ctas_per_worker > 0 ? ctx->tuning.stats_ctas_per_worker
+                                                      : static_cast<long long>(ctx->sm_count) / a.M;
+  if (P < 1) P = 1;
+  if (P > n_tiles) P = n_tiles;
+  if (P > 65535) P = 65535;
+  const size_t need = static_cast<size_t>(a.M) * P * (a.b + 2) * sizeof(double);
+  if (need > ctx->workspace_bytes)
+    return set_error(ctx, ABS_ERR_WORKSPACE, "abs_test_stats needs %zu workspace bytes, context has %zu", need,
+                     ctx->workspace_bytes);
+  UmmaParams prm;
+  prm.G = static_cast<const __nv_bfloat16*>(a.G);
+  prm.b = a.b;
+  prm.d = a.d;
+  prm.row_stride = a.row_stride;
+  prm.worker_stride = a.M > 1 ? a.worker_stride : 0;
+  prm.n_dim = g.n_dim;
+  prm.acc_cols = g.acc_cols;
+  prm.stages = g.stages;
+  prm.lag = g.lag;
+  prm.kb_bytes = g.kb_bytes;
+  prm.stage_bytes = g.stage_bytes;
+  prm.n_tiles = n_tiles;
+  prm.P = static_cast<int>(P);
+  prm.ws = static_cast<double*>(ctx->workspace);
+  prm.gbar_out = a.gbar_out;
+  prm.flags = ctx->flags;
+  prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
+  const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
+  const int rc = a.gbar_out != nullptr ? launch_umma_variant<true>(ctx, prm, grid, g.smem, a.stream)
+                                       : launch_umma_variant<false>(ctx, prm, grid, g.smem, a.stream);
+  if (rc != ABS_OK) return rc;
+  *P_out = static_cast<int>(P);
+  return ABS_OK;
+}
+
+}  // namespace absk

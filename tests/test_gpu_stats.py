@@ -160,6 +160,37 @@ def test_gram_and_tiled_kernels_agree_on_bf16(ctx, M, b, d):
                                atol=1e-6 * gbar_t.abs().max().item())
 
 
+@pytest.mark.parametrize("want_gbar", [False, True])
+@pytest.mark.parametrize("M,b,d,pad", [(1, 33, 2048, 0), (2, 40, 5003, 5), (1, 64, 9000, 0), (3, 100, 4104, 0),
+                                       (1, 128, 8200, 8), (1, 96, 300, 4), (1, 128, 300000, 0), (2, 72, 150001, 7),
+                                       (1, 48, 256, 0), (1, 127, 1025, 7)])
+def test_tcgen05_gram_kernel_matches_oracle_and_tiled_kernel(ctx, M, b, d, pad, want_gbar):
+    """bf16 input with 32 < b <= 128 and 16-byte aligned rows goes through the tcgen05 Gram kernel
+    (with and without the column-mean warps); the tiled kernel must give the same statistics, and
+    both must match the oracle, also with a ragged last tile and a last 16-byte chunk cut by d."""
+    assert pkg.plan_stats("bf16", b)["route"] == 4
+    G = make_G(170 + b, M, b, d, torch.bfloat16, sigma=2.0, pad=pad)
+    assert (G.stride(1) * 2) % 16 == 0 and G.data_ptr() % 16 == 0
+    tc, gbar_tc = run_gpu(ctx, G, want_gbar)
+    ctx.set_tuning("stats_no_gram", 1)
+    try:
+        tiled, gbar_t = run_gpu(ctx, G, want_gbar)
+    finally:
+        ctx.set_tuning("stats_no_gram", 0)
+    H = to_f64(G)
+    for m in range(M):
+        ref = orc.batch_test_stats(H[m])
+        check_record(tc[m], ref, 1e-3, b)
+        check_record(tiled[m], ref, 1e-3, b)
+        for key in ("gbar_sq", "var_norm", "sum_sq"):
+            assert tc[m][key] == pytest.approx(ref[key], rel=1e-5)
+    if want_gbar:
+        np.testing.assert_allclose(gbar_tc.cpu().numpy(), H.mean(axis=1), rtol=1e-5,
+                                   atol=1e-6 * float(np.abs(H).max()))
+        np.testing.assert_allclose(gbar_tc.cpu().numpy(), gbar_t.cpu().numpy(), rtol=1e-6,
+                                   atol=1e-6 * gbar_t.abs().max().item())
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("M,b,d", [(1, 512, 3000), (2, 700, 1300), (1, 1024, 2100), (1, 1500, 640), (1, 2048, 520),
                                    (1, 3000, 200), (1, 4096, 264)])

@@ -24,6 +24,15 @@ def check_plan(dtype, b, p):
     if p["route"] == 0:
         assert dtype == "bf16" and b <= 32 and p["box_rows"] == b
         return
+    if p["route"] == 4:
+        # tcgen05 Gram kernel: k-blocks of ceil8(b) rows x 128 bytes, each on a 1024-byte boundary
+        assert dtype == "bf16" and 32 < b <= 128
+        assert p["box_rows"] % 8 == 0 and b <= p["box_rows"] < b + 8
+        assert lpr == 8 and p["boxes_per_stage"] == 4
+        assert p["stage_bytes"] == 4 * p["box_rows"] * 128 and (p["stage_bytes"] // 4) % 1024 == 0
+        # the 128-row operand descriptor of the last k-block stays inside the allocation
+        assert p["stages"] * p["stage_bytes"] + (128 - p["box_rows"]) * 128 + 1024 <= p["smem_bytes"]
+        return
     groups = p["warps_per_box"] * 32 // lpr                  # row groups that share a box
     R = p["rows_per_thread"]
     assert R * groups >= p["rows_per_cta"]
@@ -52,6 +61,8 @@ def test_every_batch_size_gets_a_valid_plan(dtype):
         p = pkg.plan_stats(dtype, b)
         if dtype == "bf16" and b <= 32:
             assert p["route"] == 0
+        elif dtype == "bf16" and b <= 128:
+            assert p["route"] == 4
         elif b > 256:
             assert p["route"] == 1
         else:
@@ -76,3 +87,7 @@ def test_documented_shapes():
     assert (p["cluster_size"], p["rows_per_cta"], p["lanes_per_row"]) == (8, 512, 8)
     p = pkg.plan_stats("bf16", 16)
     assert (p["route"], p["boxes_per_stage"], p["lanes_per_row"]) == (0, 8, 32)
+    p = pkg.plan_stats("bf16", 128)
+    assert (p["route"], p["stages"], p["stage_bytes"]) == (4, 3, 65536)
+    p = pkg.plan_stats("bf16", 33)
+    assert (p["route"], p["stages"], p["box_rows"]) == (4, 8, 40)
