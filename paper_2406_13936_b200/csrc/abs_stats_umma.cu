@@ -6,7 +6,7 @@
 // The CUDA-core route needs about six instructions per bf16 element and stalls near 4 TB/s for
 // these batch sizes; a 128 x b x 16 tcgen05.mma takes the 4 KiB it consumes off the critical path.
 // Products of two bf16 values are exact in fp32; the tensor core adds them in fp32 over
-// kFoldTiles * 256 columns in TMEM, then four warps read the accumulator back (tcgen05.ld),
+// fold_tiles * 256 columns in TMEM, then four warps read the accumulator back (tcgen05.ld),
 // reduce each row to (K 1)_i and K_ii and add those to fp64 registers, which is where the
 // cancellation in c_i - N happens.  Two accumulators alternate, so the read-back overlaps the
 // next fold's MMAs.
@@ -32,7 +32,7 @@ namespace {
 
 constexpr int kLoadWarps = 4;
 constexpr int kTileCols = 256;       // columns per stage: four k-blocks of 64 (128-byte swizzle span)
-constexpr int kFoldTiles = 4;        // stages accumulated in TMEM before the fold into fp64
+constexpr int kFoldTilesDefault = 4;     // stages accumulated in TMEM before the fold into fp64
 constexpr int kMaxStagesU = 8;
 constexpr int kBarsU = 2 * kMaxStagesU + 5;
 
@@ -42,7 +42,7 @@ struct UmmaParams {
   int n_dim;              // ceil16(b): N of the MMA
   int acc_cols;           // TMEM columns per accumulator (n_dim rounded up to a power of two >= 32)
   int stages;
-  int lag;                // copy groups a loader keeps in flight
+  int fold_tiles;         // stages accumulated in TMEM before the fold into fp64
   unsigned kb_bytes;      // ceil8(b) * 128
   unsigned stage_bytes;   // 4 k-blocks
   long long n_tiles;
@@ -56,23 +56,25 @@ struct UmmaParams {
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait(int pending) {
-  switch (pending) {
-    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
-    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
-    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
-  }
-}
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// K-major operand, 128-byte swizzle: 8-row groups 1024 bytes apart; version 1 (sm_100).
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-  return static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+// Bounded wait for barriers that are expected to stay closed for a while: sleeps between polls so
+// that the waiting warps leave the issue slots to the loaders and the MMA thread.
+__device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity, volatile unsigned* abort_flag,
+                                                  long long limit, unsigned sleep_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (*abort_flag) return false;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag || clock64() - t0 > limit) {
+      *abort_flag = 1u;
+      return false;
+    }
+    __nanosleep(sleep_ns);
+  }
+  return true;
 }
 // D (fp32, TMEM) (+)= A (bf16, smem) * B^T (bf16, smem); issued by one thread.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
@@ -128,7 +130,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
 
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
-      mbar_init(full_u32 + 8u * s, kLoadWarps);
+      mbar_init(full_u32 + 8u * s, kLoadWarps * 32);
       mbar_init(empty_u32 + 8u * s, WANT_GBAR ? 5 : 1);
     }
     for (int k = 0; k < 2; ++k) {
@@ -156,65 +158,78 @@ abs_stats_umma_kernel(const UmmaParams prm) {
   double row_sum = 0.0, row_diag = 0.0;
 
   if (warp < kLoadWarps) {
-    // ---- loaders: 16-byte chunk c of the tile = row c / 32, chunk c % 32 of its 512 bytes ----
-    const int n_chunks = b * 32;
-    const int lag = prm.lag;
+    // ---- loaders: lane = 16-byte chunk of the tile row's 512 bytes, rows warp, warp + 4, ... ----
+    // The swizzle term depends on row % 8, which alternates between two values along a thread's rows.
+    const uint32_t kb_off = static_cast<uint32_t>(lane >> 3) * prm.kb_bytes + static_cast<uint32_t>(warp) * 128u;
+    const uint32_t swz0 = static_cast<uint32_t>((lane & 7) ^ warp) << 4;
+    const uint32_t swz1 = (static_cast<uint32_t>((lane & 7) ^ (warp + 4)) << 4) + 512u;
+    const long long step8 = 8 * prm.row_stride, step4 = 4 * prm.row_stride;
+    const __nv_bfloat16* row0 = Gm + static_cast<long long>(warp) * prm.row_stride;
+    long long col = static_cast<long long>(p) * kTileCols + lane * 8;
+    int s = 0;
+    uint32_t pass = 0;
     for (long long i = 0; i < n_mine; ++i) {
-      const int s = static_cast<int>(i % S);
-      const long long use = i / S;
-      if (use > 0) mbar_wait(empty_u32 + 8u * s, static_cast<uint32_t>((use - 1) & 1), abort_flag, prm.timeout_cycles);
-      const long long col0 = (p + i * prm.P) * kTileCols;
-      const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes;
-      for (int c = tid; c < n_chunks; c += kLoadWarps * 32) {
-        const int row = c >> 5, ch = c & 31;
-        const long long col = col0 + ch * 8;
-        const long long left = prm.d - col;                         // elements of this row from col on
-        const uint32_t bytes = left >= 8 ? 16u : (left > 0 ? static_cast<uint32_t>(left) * 2u : 0u);
-        const __nv_bfloat16* src = Gm + static_cast<long long>(row) * prm.row_stride + (left > 0 ? col : 0);
-        const uint32_t dst = stage + static_cast<uint32_t>(ch >> 3) * prm.kb_bytes + static_cast<uint32_t>(row) * 128u +
-                             (static_cast<uint32_t>((ch & 7) ^ (row & 7)) << 4);
-        cp_async_16(dst, src, bytes);                               // bytes past `bytes` are zero-filled
+      if (pass > 0) mbar_wait_backoff(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles, 64);
+      const long long left = prm.d - col;                           // elements of a row from this chunk on
+      const uint32_t bytes = left >= 8 ? 16u : (left > 0 ? static_cast<uint32_t>(left) * 2u : 0u);
+      const __nv_bfloat16* src = row0 + (left > 0 ? col : 0);
+      uint32_t dst = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + kb_off;
+      for (int row = warp; row < b; row += 8) {
+        cp_async_16(dst + swz0, src, bytes);                        // bytes past `bytes` are zero-filled
+        if (row + 4 < b) cp_async_16(dst + swz1, src + step4, bytes);
+        src += step8;
+        dst += 1024u;
       }
-      cp_async_commit();
-      if (i >= lag) {
-        cp_async_wait(lag);                                         // tile i - lag has landed
-        fence_async_smem();                                         // ... and is visible to the tensor core
-        __syncwarp();
-        if (lane == 0) mbar_arrive(full_u32 + 8u * static_cast<uint32_t>((i - lag) % S));
+      // one arrival on the stage's barrier once this thread's copies have landed; nothing here
+      // waits for them, so the loaders run a whole ring ahead of the tensor core
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_u32 + 8u * s) : "memory");
+      col += static_cast<long long>(prm.P) * kTileCols;
+      if (++s == S) {
+        s = 0;
+        ++pass;
       }
     }
-    cp_async_wait(0);
-    fence_async_smem();
-    __syncwarp();
-    if (lane == 0)
-      for (long long i = (n_mine > lag ? n_mine - lag : 0); i < n_mine; ++i)
-        mbar_arrive(full_u32 + 8u * static_cast<uint32_t>(i % S));
+    asm volatile("cp.async.wait_all;" ::: "memory");                // nothing in flight at exit
   } else if (warp == 8) {
     // ---- MMA issue ----
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(prm.n_dim >> 3) << 17) |
                              (8u << 24);                            // fp32 accumulate, bf16 x bf16, K-major, M = 128
+      // operand descriptor, K-major with 128-byte swizzle: start address / 16, 8-row groups 1024 bytes
+      // apart (64 << 32), descriptor version 1 (bit 46), swizzle mode 2 (bits 61-63)
+      const uint64_t desc_hi = (64ull << 32) | (1ull << 46) | (2ull << 61) | (1ull << 16);
+      const uint32_t kb16 = prm.kb_bytes >> 4;
+      int s = 0, fold_pos = 0;
+      uint32_t pass = 0, fold = 0;
       for (long long i = 0; i < n_mine; ++i) {
-        const int s = static_cast<int>(i % S);
-        const long long fold = i / kFoldTiles;
-        const int buf = static_cast<int>(fold & 1);
-        const bool first = (i % kFoldTiles) == 0;
-        if (first && fold >= 2)
-          mbar_wait(accempty_u32 + 8u * buf, static_cast<uint32_t>((fold / 2 - 1) & 1), abort_flag, prm.timeout_cycles);
-        mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>((i / S) & 1), abort_flag, prm.timeout_cycles);
+        const uint32_t buf = fold & 1u;
+        if (fold_pos == 0 && fold >= 2)
+          mbar_wait(accempty_u32 + 8u * buf, ((fold >> 1) - 1) & 1u, abort_flag, prm.timeout_cycles);
+        mbar_wait(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles);
+        fence_async_smem();                                         // the copies' writes, before the tensor core reads
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * prm.acc_cols);
-        const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes;
+        const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(prm.acc_cols);
+        const uint32_t lo = ((ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes) & 0x3ffffu) >> 4;
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const uint64_t desc = umma_desc(stage + static_cast<uint32_t>(kb) * prm.kb_bytes + static_cast<uint32_t>(k) * 32u);
-            umma_bf16(d_tmem, desc, desc, idesc, (first && kb == 0 && k == 0) ? 0u : 1u);
+            const uint64_t desc = desc_hi | static_cast<uint64_t>(lo + static_cast<uint32_t>(kb) * kb16 + 2u * k);
+            umma_bf16(d_tmem, desc, desc, idesc, (fold_pos == 0 && kb == 0 && k == 0) ? 0u : 1u);
           }
         }
         umma_commit(empty_u32 + 8u * s);                            // the stage may be refilled
-        if ((i % kFoldTiles) == kFoldTiles - 1 || i == n_mine - 1) umma_commit(accfull_u32 + 8u * buf);
+        if (fold_pos == prm.fold_tiles - 1 || i == n_mine - 1) {
+          umma_commit(accfull_u32 + 8u * buf);
+          fold_pos = 0;
+          ++fold;
+        } else {
+          ++fold_pos;
+        }
+        if (++s == S) {
+          s = 0;
+          ++pass;
+        }
       }
       umma_commit(done_u32);
       volatile unsigned ignore = 0u;
@@ -225,12 +240,12 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     // ---- accumulator read-back: this thread owns row i = 32 (warp % 4) + lane of K ----
     const int q = warp & 3;
     const int row = q * 32 + lane;
-    const long long n_folds = (n_mine + kFoldTiles - 1) / kFoldTiles;
+    const long long n_folds = (n_mine + prm.fold_tiles - 1) / prm.fold_tiles;
     for (long long f = 0; f < n_folds; ++f) {
-      const int buf = static_cast<int>(f & 1);
-      mbar_wait(accfull_u32 + 8u * buf, static_cast<uint32_t>((f / 2) & 1), abort_flag, prm.timeout_cycles);
+      const uint32_t buf = static_cast<uint32_t>(f) & 1u;
+      mbar_wait_backoff(accfull_u32 + 8u * buf, static_cast<uint32_t>(f >> 1) & 1u, abort_flag, prm.timeout_cycles, 256);
       tc_fence_after();
-      const uint32_t taddr = tmem_base + static_cast<uint32_t>(buf * prm.acc_cols) + (static_cast<uint32_t>(q * 32) << 16);
+      const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(prm.acc_cols) + (static_cast<uint32_t>(q * 32) << 16);
       float diag = 0.f;
       for (int c0 = 0; c0 < prm.n_dim; c0 += 16) {
         float v[16];
@@ -252,9 +267,11 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     const int kb = warp - 9;
     const int sub = lane >> 3, ch = lane & 7;
     const float inv_b = 1.0f / static_cast<float>(b);
+    long long col = static_cast<long long>(p) * kTileCols + kb * 64 + ch * 8;
+    int s = 0;
+    uint32_t pass = 0;
     for (long long i = 0; i < n_mine; ++i) {
-      const int s = static_cast<int>(i % S);
-      mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>((i / S) & 1), abort_flag, prm.timeout_cycles);
+      mbar_wait_backoff(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles, 32);
       const uint32_t base = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(kb) * prm.kb_bytes;
       float cs[8];
 #pragma unroll
@@ -274,7 +291,6 @@ abs_stats_umma_kernel(const UmmaParams prm) {
       __syncwarp();
       if (lane == 0) mbar_arrive(empty_u32 + 8u * s);
       if (sub == 0) {
-        const long long col = (p + i * prm.P) * kTileCols + kb * 64 + ch * 8;
         float* dst = prm.gbar_out + static_cast<long long>(m) * prm.d + col;
         if (col + 8 <= prm.d && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
           *reinterpret_cast<float4*>(dst) = make_float4(cs[0] * inv_b, cs[1] * inv_b, cs[2] * inv_b, cs[3] * inv_b);
@@ -284,6 +300,11 @@ abs_stats_umma_kernel(const UmmaParams prm) {
           for (int j = 0; j < 8; ++j)
             if (col + j < prm.d) dst[j] = cs[j] * inv_b;
         }
+      }
+      col += static_cast<long long>(prm.P) * kTileCols;
+      if (++s == S) {
+        s = 0;
+        ++pass;
       }
     }
   }
@@ -325,7 +346,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
 }
 
 struct UmmaGeom {
-  int rows_blk, n_dim, acc_cols, stages, lag;
+  int rows_blk, n_dim, acc_cols, stages;
   unsigned kb_bytes, stage_bytes;
   size_t smem;
 };
@@ -345,8 +366,6 @@ bool umma_geometry(const Tuning& t, size_t smem_optin, long long b, UmmaGeom* g)
   g->stages = stages;
   g->smem = static_cast<size_t>(stages) * g->stage_bytes + fixed;
   if (g->smem > smem_optin) return false;
-  // copy groups in flight per loader: all but one stage, at most 4 (the tensor core works on the oldest)
-  g->lag = stages - 1 > 4 ? 4 : stages - 1;
   return true;
 }
 
@@ -409,7 +428,8 @@ int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.n_dim = g.n_dim;
   prm.acc_cols = g.acc_cols;
   prm.stages = g.stages;
-  prm.lag = g.lag;
+  prm.fold_tiles = static_cast<int>(ctx->tuning.stats_flush_every > 0 ? (ctx->tuning.stats_flush_every > 64 ? 64 : ctx->tuning.stats_flush_every)
+                                                                      : kFoldTilesDefault);
   prm.kb_bytes = g.kb_bytes;
   prm.stage_bytes = g.stage_bytes;
   prm.n_tiles = n_tiles;
