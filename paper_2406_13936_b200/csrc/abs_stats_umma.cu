@@ -31,7 +31,7 @@ namespace absk {
 namespace {
 
 constexpr int kLoadWarps = 4;
-constexpr int kTileCols = 256;       // columns per stage: four k-blocks of 64 (128-byte swizzle span)
+constexpr int kSubCols = 256;        // columns of one row segment: four k-blocks of 64 (128-byte swizzle span)
 constexpr int kFoldTilesDefault = 4;     // stages accumulated in TMEM before the fold into fp64
 constexpr int kMaxStagesU = 8;
 constexpr int kBarsU = 2 * kMaxStagesU + 5;
@@ -39,11 +39,13 @@ constexpr int kBarsU = 2 * kMaxStagesU + 5;
 struct UmmaParams {
   const __nv_bfloat16* G;
   long long b, d, row_stride, worker_stride;   // strides in elements
-  int n_dim;              // ceil16(b): N of the MMA
+  int stack;              // column segments stacked as extra rows of the operand (1..3)
+  int rows_blk;           // ceil8(b): rows one segment takes in a k-block
+  int n_dim;              // ceil16(stack * rows_blk): N of the MMA
   int acc_cols;           // TMEM columns per accumulator (n_dim rounded up to a power of two >= 32)
   int stages;
   int fold_tiles;         // stages accumulated in TMEM before the fold into fp64
-  unsigned kb_bytes;      // ceil8(b) * 128
+  unsigned kb_bytes;      // stack * rows_blk * 128
   unsigned stage_bytes;   // 4 k-blocks
   long long n_tiles;
   int P;
@@ -121,7 +123,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);
   volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + kBarsU);
   unsigned* tmem_slot = const_cast<unsigned*>(abort_flag) + 1;
-  double* red = reinterpret_cast<double*>(bars + kBarsU + 1);     // [128] row sums, [128] diagonal, [2]
+  double* red = reinterpret_cast<double*>(bars + kBarsU + 1);     // [128] row sums, [128] diagonal, [2], [128] + [128] per row of G
   const uint32_t full_u32 = smem_u32(bars);
   const uint32_t empty_u32 = full_u32 + 8u * kMaxStagesU;
   const uint32_t accfull_u32 = empty_u32 + 8u * kMaxStagesU;      // 2
@@ -165,25 +167,30 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     const uint32_t swz1 = (static_cast<uint32_t>((lane & 7) ^ (warp + 4)) << 4) + 512u;
     const long long step8 = 8 * prm.row_stride, step4 = 4 * prm.row_stride;
     const __nv_bfloat16* row0 = Gm + static_cast<long long>(warp) * prm.row_stride;
-    long long col = static_cast<long long>(p) * kTileCols + lane * 8;
+    const long long tile_cols = static_cast<long long>(prm.stack) * kSubCols;
+    const uint32_t seg_bytes = static_cast<uint32_t>(prm.rows_blk) * 128u;
+    long long col0 = static_cast<long long>(p) * tile_cols + lane * 8;
     int s = 0;
     uint32_t pass = 0;
     for (long long i = 0; i < n_mine; ++i) {
       if (pass > 0) mbar_wait_backoff(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles, 64);
-      const long long left = prm.d - col;                           // elements of a row from this chunk on
-      const uint32_t bytes = left >= 8 ? 16u : (left > 0 ? static_cast<uint32_t>(left) * 2u : 0u);
-      const __nv_bfloat16* src = row0 + (left > 0 ? col : 0);
-      uint32_t dst = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + kb_off;
-      for (int row = warp; row < b; row += 8) {
-        cp_async_16(dst + swz0, src, bytes);                        // bytes past `bytes` are zero-filled
-        if (row + 4 < b) cp_async_16(dst + swz1, src + step4, bytes);
-        src += step8;
-        dst += 1024u;
+      for (int t = 0; t < prm.stack; ++t) {
+        const long long col = col0 + t * kSubCols;
+        const long long left = prm.d - col;                         // elements of a row from this chunk on
+        const uint32_t bytes = left >= 8 ? 16u : (left > 0 ? static_cast<uint32_t>(left) * 2u : 0u);
+        const __nv_bfloat16* src = row0 + (left > 0 ? col : 0);
+        uint32_t dst = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(t) * seg_bytes + kb_off;
+        for (int row = warp; row < b; row += 8) {
+          cp_async_16(dst + swz0, src, bytes);                      // bytes past `bytes` are zero-filled
+          if (row + 4 < b) cp_async_16(dst + swz1, src + step4, bytes);
+          src += step8;
+          dst += 1024u;
+        }
       }
       // one arrival on the stage's barrier once this thread's copies have landed; nothing here
       // waits for them, so the loaders run a whole ring ahead of the tensor core
       asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_u32 + 8u * s) : "memory");
-      col += static_cast<long long>(prm.P) * kTileCols;
+      col0 += static_cast<long long>(prm.P) * tile_cols;
       if (++s == S) {
         s = 0;
         ++pass;
@@ -237,9 +244,13 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     }
     __syncwarp();
   } else if (warp < 8) {
-    // ---- accumulator read-back: this thread owns row i = 32 (warp % 4) + lane of K ----
+    // ---- accumulator read-back: this thread owns TMEM lane r = 32 (warp % 4) + lane, which is row
+    // r % rows_blk of the Gram matrix of column segment r / rows_blk (columns c0 .. c0 + b of the lane) ----
     const int q = warp & 3;
     const int row = q * 32 + lane;
+    const int c_first = row / prm.rows_blk * prm.rows_blk;
+    const bool live = row < prm.stack * prm.rows_blk && row - c_first < b;
+    const int c_last = live ? c_first + b : 0;                      // columns [c_first, c_last) of this lane count
     const long long n_folds = (n_mine + prm.fold_tiles - 1) / prm.fold_tiles;
     for (long long f = 0; f < n_folds; ++f) {
       const uint32_t buf = static_cast<uint32_t>(f) & 1u;
@@ -253,7 +264,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
         float part = 0.f;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          part += (c0 + j < b) ? v[j] : 0.f;
+          part += (c0 + j >= c_first && c0 + j < c_last) ? v[j] : 0.f;
           diag = (c0 + j == row) ? v[j] : diag;
         }
         row_sum += static_cast<double>(part);
@@ -267,41 +278,46 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     const int kb = warp - 9;
     const int sub = lane >> 3, ch = lane & 7;
     const float inv_b = 1.0f / static_cast<float>(b);
-    long long col = static_cast<long long>(p) * kTileCols + kb * 64 + ch * 8;
+    const long long tile_cols = static_cast<long long>(prm.stack) * kSubCols;
+    long long col0 = static_cast<long long>(p) * tile_cols + kb * 64 + ch * 8;
     int s = 0;
     uint32_t pass = 0;
     for (long long i = 0; i < n_mine; ++i) {
       mbar_wait_backoff(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles, 32);
-      const uint32_t base = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(kb) * prm.kb_bytes;
-      float cs[8];
+      for (int t = 0; t < prm.stack; ++t) {
+        const long long col = col0 + t * kSubCols;
+        const uint32_t base = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes +
+                              static_cast<uint32_t>(kb) * prm.kb_bytes + static_cast<uint32_t>(t * prm.rows_blk) * 128u;
+        float cs[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) cs[j] = 0.f;
-      for (int r = sub; r < b; r += 4) {
-        const uint4 u = lds128(base + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>(ch ^ (r & 7)) << 4));
-        float x[8];
-        Vec<__nv_bfloat16>::unpack(u, x);
+        for (int j = 0; j < 8; ++j) cs[j] = 0.f;
+        for (int r = sub; r < b; r += 4) {
+          const uint4 u = lds128(base + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>(ch ^ (r & 7)) << 4));
+          float x[8];
+          Vec<__nv_bfloat16>::unpack(u, x);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) cs[j] += x[j];
-      }
+          for (int j = 0; j < 8; ++j) cs[j] += x[j];
+        }
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 8);
-        cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 16);
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(empty_u32 + 8u * s);
-      if (sub == 0) {
-        float* dst = prm.gbar_out + static_cast<long long>(m) * prm.d + col;
-        if (col + 8 <= prm.d && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
-          *reinterpret_cast<float4*>(dst) = make_float4(cs[0] * inv_b, cs[1] * inv_b, cs[2] * inv_b, cs[3] * inv_b);
-          *reinterpret_cast<float4*>(dst + 4) = make_float4(cs[4] * inv_b, cs[5] * inv_b, cs[6] * inv_b, cs[7] * inv_b);
-        } else {
+        for (int j = 0; j < 8; ++j) {
+          cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 8);
+          cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 16);
+        }
+        if (sub == 0) {
+          float* dst = prm.gbar_out + static_cast<long long>(m) * prm.d + col;
+          if (col + 8 <= prm.d && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+            *reinterpret_cast<float4*>(dst) = make_float4(cs[0] * inv_b, cs[1] * inv_b, cs[2] * inv_b, cs[3] * inv_b);
+            *reinterpret_cast<float4*>(dst + 4) = make_float4(cs[4] * inv_b, cs[5] * inv_b, cs[6] * inv_b, cs[7] * inv_b);
+          } else {
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (col + j < prm.d) dst[j] = cs[j] * inv_b;
+            for (int j = 0; j < 8; ++j)
+              if (col + j < prm.d) dst[j] = cs[j] * inv_b;
+          }
         }
       }
-      col += static_cast<long long>(prm.P) * kTileCols;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty_u32 + 8u * s);                // this warp's reads of the stage are done
+      col0 += static_cast<long long>(prm.P) * tile_cols;
       if (++s == S) {
         s = 0;
         ++pass;
@@ -321,11 +337,21 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
   }
+  if (tid < b) {                                  // the segments' Gram matrices add up to the tile's
+    double rs = 0.0, dg = 0.0;
+    for (int t = 0; t < prm.stack; ++t) {
+      rs += red[t * prm.rows_blk + tid];
+      dg += red[128 + t * prm.rows_blk + tid];
+    }
+    red[258 + tid] = rs;
+    red[386 + tid] = dg;
+  }
+  __syncthreads();
   if (tid == 0) {
     double total = 0.0, trace = 0.0;
     for (int i = 0; i < b; ++i) {
-      total += red[i];
-      trace += red[128 + i];
+      total += red[258 + i];
+      trace += red[386 + i];
     }
     red[256] = total;
     red[257] = trace;
@@ -336,7 +362,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     const double total = red[256], trace = red[257];
     const double Ncta = total / (bd * bd);
     double* out = prm.ws + (static_cast<size_t>(m) * prm.P + p) * (static_cast<size_t>(b) + 2);
-    for (int i = tid; i < b; i += blockDim.x) out[i] = red[i] / bd - Ncta;     // sum_j (g_ij - gbar_j) gbar_j
+    for (int i = tid; i < b; i += blockDim.x) out[i] = red[258 + i] / bd - Ncta;   // sum_j (g_ij - gbar_j) gbar_j
     if (tid == 0) {
       out[b] = trace - total / bd;                                             // sum_ij (g_ij - gbar_j)^2
       out[b + 1] = Ncta;
@@ -346,7 +372,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
 }
 
 struct UmmaGeom {
-  int rows_blk, n_dim, acc_cols, stages;
+  int rows_blk, stack, n_dim, acc_cols, stages;
   unsigned kb_bytes, stage_bytes;
   size_t smem;
 };
@@ -354,12 +380,13 @@ struct UmmaGeom {
 bool umma_geometry(const Tuning& t, size_t smem_optin, long long b, UmmaGeom* g) {
   if (b <= 32 || b > 128) return false;
   g->rows_blk = static_cast<int>((b + 7) / 8 * 8);
-  g->n_dim = static_cast<int>((b + 15) / 16 * 16);
+  g->stack = 128 / g->rows_blk;                   // 1 (b > 64), 2 (40 < b <= 64) or 3 (b <= 40)
+  g->n_dim = (g->stack * g->rows_blk + 15) / 16 * 16;
   g->acc_cols = g->n_dim <= 64 ? 64 : 128;
-  g->kb_bytes = static_cast<unsigned>(g->rows_blk) * 128u;
+  g->kb_bytes = static_cast<unsigned>(g->stack * g->rows_blk) * 128u;
   g->stage_bytes = 4u * g->kb_bytes;
-  const size_t pad = static_cast<size_t>(128 - g->rows_blk) * 128;
-  const size_t fixed = 1024 + pad + static_cast<size_t>(kBarsU + 1) * 8 + 258 * sizeof(double) + 128;
+  const size_t pad = static_cast<size_t>(128 - g->stack * g->rows_blk) * 128;
+  const size_t fixed = 1024 + pad + static_cast<size_t>(kBarsU + 1) * 8 + 514 * sizeof(double) + 128;
   int stages = static_cast<int>(t.stats_stages > 0 ? t.stats_stages : kMaxStagesU);
   if (stages > kMaxStagesU) stages = kMaxStagesU;
   while (stages > 2 && static_cast<size_t>(stages) * g->stage_bytes + fixed > smem_optin) --stages;
@@ -389,7 +416,7 @@ int plan_stats_umma(const Tuning& t, size_t smem_optin, abs_dtype dtype, long lo
   out->warps_per_box = kLoadWarps;
   out->boxes_per_stage = 4;                  // k-blocks
   out->stages = g.stages;
-  out->box_rows = g.rows_blk;
+  out->box_rows = g.stack * g.rows_blk;
   out->row_boxes = 1;
   out->rows_per_thread = 0;
   out->cluster_size = 1;
@@ -409,7 +436,8 @@ int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if ((reinterpret_cast<uintptr_t>(a.G) & 15u) || (row_b & 15u) || (wrk_b & 15u) || a.M > 65535)
     return ABS_ERR_UNSUPPORTED;
 
-  const long long n_tiles = (a.d + kTileCols - 1) / kTileCols;
+  const long long tile_cols = static_cast<long long>(g.stack) * kSubCols;
+  const long long n_tiles = (a.d + tile_cols - 1) / tile_cols;
   long long P = ctx->tuning.stats_ctas_per_worker > 0 ? ctx->tuning.stats_ctas_per_worker
                                                       : static_cast<long long>(ctx->sm_count) / a.M;
   if (P < 1) P = 1;
@@ -425,6 +453,8 @@ int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.d = a.d;
   prm.row_stride = a.row_stride;
   prm.worker_stride = a.M > 1 ? a.worker_stride : 0;
+  prm.stack = g.stack;
+  prm.rows_blk = g.rows_blk;
   prm.n_dim = g.n_dim;
   prm.acc_cols = g.acc_cols;
   prm.stages = g.stages;

@@ -25,9 +25,11 @@ def check_plan(dtype, b, p):
         assert dtype == "bf16" and b <= 32 and p["box_rows"] == b
         return
     if p["route"] == 4:
-        # tcgen05 Gram kernel: k-blocks of ceil8(b) rows x 128 bytes, each on a 1024-byte boundary
+        # tcgen05 Gram kernel: k-blocks of 1..3 column segments x ceil8(b) rows x 128 bytes, each k-block
+        # on a 1024-byte boundary, at most 128 operand rows
         assert dtype == "bf16" and 32 < b <= 128
-        assert p["box_rows"] % 8 == 0 and b <= p["box_rows"] < b + 8
+        rows_blk = (b + 7) // 8 * 8
+        assert p["box_rows"] == (128 // rows_blk) * rows_blk and p["rows_per_cta"] == b
         assert lpr == 8 and p["boxes_per_stage"] == 4
         assert p["stage_bytes"] == 4 * p["box_rows"] * 128 and (p["stage_bytes"] // 4) % 1024 == 0
         # the 128-row operand descriptor of the last k-block stays inside the allocation
@@ -90,4 +92,4 @@ def test_documented_shapes():
     p = pkg.plan_stats("bf16", 128)
     assert (p["route"], p["stages"], p["stage_bytes"]) == (4, 3, 65536)
     p = pkg.plan_stats("bf16", 33)
-    assert (p["route"], p["stages"], p["box_rows"]) == (4, 8, 40)
+    assert (p["route"], p["stages"], p["box_rows"]) == (4, 3, 120)
