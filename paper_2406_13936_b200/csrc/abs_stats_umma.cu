@@ -12,17 +12,26 @@
 // next fold's MMAs.
 //
 // Operands: both A and B are the same shared-memory tile (K-major, 128-byte swizzle): rows of G,
-// 64 columns per k-block, four k-blocks per stage.  A tensor-map copy into that layout is limited
-// to 128-byte box rows, which the copy engine serves at about two thirds of the HBM rate, so the
-// tile is filled by four loader warps with 16-byte cp.async copies (a warp covers 512 contiguous
-// bytes of one row) that apply the swizzle themselves.  A k-block holds ceil8(b) rows; the A
-// descriptor always spans 128 rows and the B descriptor ceil16(b), so both may run into the next
-// k-block: what they pick up there lands in rows / columns >= b of K, which nobody reads.
+// 64 columns per k-block, four k-blocks per row segment of 256 columns.  A tensor-map copy into
+// that layout is limited to 128-byte box rows, which the copy engine serves at about two thirds
+// of the HBM rate, so the tile is filled by four loader warps with 16-byte cp.async copies (a warp
+// covers 512 contiguous bytes of one row) that apply the swizzle themselves and signal the
+// stage's mbarrier through cp.async.mbarrier.arrive, so they never wait for their own copies.
+//
+// Measured here, an MMA of this shape costs about (128 + N) / 2 clocks whatever M and the
+// arithmetic are (the operands arrive at about 64 bytes per clock), i.e. about 100 clocks per 16
+// columns.  For b <= 64 that is slower than HBM delivers 16 columns, so two or three column
+// segments are stacked as extra operand rows: the tile [s * ceil8(b) rows] x [256 columns] holds
+// segment t in rows t * ceil8(b) ..., one MMA then covers 16 columns of every segment, and the
+// diagonal blocks of its s x s block result are the segments' Gram matrices (the off-diagonal
+// blocks are never read).  A k-block holds stack * ceil8(b) rows; the A descriptor always spans
+// 128 rows and the B descriptor ceil16(.), so both may run into the next k-block: what they pick
+// up there lands in rows / columns of the accumulator that nobody reads.
 //
 // Warp roles: 0-3 loaders, 4-7 accumulator read-back (warp w owns TMEM lanes 32 (w % 4) ..),
-// 8 MMA issue and TMEM allocation, 9-12 column means on the CUDA cores when gbar is wanted.
-// Every wait is bounded; a wait that runs out raises the CTA's abort flag, every role falls
-// through its loop, TMEM is freed and the records come back flagged ABS_STATUS_TIMEOUT.
+// 8 MMA issue (one elected lane) and TMEM allocation, 9-12 column means on the CUDA cores when
+// gbar is wanted.  Every wait is bounded; a wait that runs out raises the CTA's abort flag, every
+// role falls through its loop, TMEM is freed and the records come back flagged ABS_STATUS_TIMEOUT.
 #include <cuda_bf16.h>
 
 #include "abs_pipeline.cuh"
@@ -77,6 +86,16 @@ __device__ __forceinline__ bool mbar_wait_backoff(uint32_t bar, uint32_t parity,
     __nanosleep(sleep_ns);
   }
   return true;
+}
+// True in exactly one lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t is_leader;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(is_leader));
+  return is_leader != 0;
 }
 // D (fp32, TMEM) (+)= A (bf16, smem) * B^T (bf16, smem); issued by one thread.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
@@ -198,25 +217,27 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     }
     asm volatile("cp.async.wait_all;" ::: "memory");                // nothing in flight at exit
   } else if (warp == 8) {
-    // ---- MMA issue ----
-    if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(prm.n_dim >> 3) << 17) |
-                             (8u << 24);                            // fp32 accumulate, bf16 x bf16, K-major, M = 128
-      // operand descriptor, K-major with 128-byte swizzle: start address / 16, 8-row groups 1024 bytes
-      // apart (64 << 32), descriptor version 1 (bit 46), swizzle mode 2 (bits 61-63)
-      const uint64_t desc_hi = (64ull << 32) | (1ull << 46) | (2ull << 61) | (1ull << 16);
-      const uint32_t kb16 = prm.kb_bytes >> 4;
-      int s = 0, fold_pos = 0;
-      uint32_t pass = 0, fold = 0;
-      for (long long i = 0; i < n_mine; ++i) {
-        const uint32_t buf = fold & 1u;
-        if (fold_pos == 0 && fold >= 2)
-          mbar_wait(accempty_u32 + 8u * buf, ((fold >> 1) - 1) & 1u, abort_flag, prm.timeout_cycles);
-        mbar_wait(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles);
-        fence_async_smem();                                         // the copies' writes, before the tensor core reads
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(prm.acc_cols);
-        const uint32_t lo = ((ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes) & 0x3ffffu) >> 4;
+    // ---- MMA issue: the whole warp walks the loop (uniform control flow keeps the descriptors in
+    // uniform registers), one elected lane issues ----
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(prm.n_dim >> 3) << 17) |
+                           (8u << 24);                              // fp32 accumulate, bf16 x bf16, K-major, M = 128
+    // operand descriptor, K-major with 128-byte swizzle: start address / 16, 8-row groups 1024 bytes
+    // apart (64 << 32), descriptor version 1 (bit 46), swizzle mode 2 (bits 61-63)
+    const uint64_t desc_hi = (64ull << 32) | (1ull << 46) | (2ull << 61) | (1ull << 16);
+    const uint32_t kb16 = prm.kb_bytes >> 4;
+    int s = 0, fold_pos = 0;
+    uint32_t pass = 0, fold = 0;
+    for (long long i = 0; i < n_mine; ++i) {
+      const uint32_t buf = fold & 1u;
+      if (fold_pos == 0 && fold >= 2)
+        mbar_wait(accempty_u32 + 8u * buf, ((fold >> 1) - 1) & 1u, abort_flag, prm.timeout_cycles);
+      mbar_wait(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles);
+      fence_async_smem();                                           // the copies' writes, before the tensor core reads
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(prm.acc_cols);
+      const uint32_t lo = ((ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes) & 0x3ffffu) >> 4;
+      const bool last_of_fold = fold_pos == prm.fold_tiles - 1 || i == n_mine - 1;
+      if (elect_one()) {
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
 #pragma unroll
@@ -226,23 +247,24 @@ abs_stats_umma_kernel(const UmmaParams prm) {
           }
         }
         umma_commit(empty_u32 + 8u * s);                            // the stage may be refilled
-        if (fold_pos == prm.fold_tiles - 1 || i == n_mine - 1) {
-          umma_commit(accfull_u32 + 8u * buf);
-          fold_pos = 0;
-          ++fold;
-        } else {
-          ++fold_pos;
-        }
-        if (++s == S) {
-          s = 0;
-          ++pass;
-        }
+        if (last_of_fold) umma_commit(accfull_u32 + 8u * buf);
       }
-      umma_commit(done_u32);
-      volatile unsigned ignore = 0u;
-      mbar_wait(done_u32, 0u, &ignore, prm.timeout_cycles);         // no MMA in flight when TMEM is freed
+      __syncwarp();
+      if (last_of_fold) {
+        fold_pos = 0;
+        ++fold;
+      } else {
+        ++fold_pos;
+      }
+      if (++s == S) {
+        s = 0;
+        ++pass;
+      }
     }
+    if (elect_one()) umma_commit(done_u32);
     __syncwarp();
+    volatile unsigned ignore = 0u;
+    mbar_wait(done_u32, 0u, &ignore, prm.timeout_cycles);           // no MMA in flight when TMEM is freed
   } else if (warp < 8) {
     // ---- accumulator read-back: this thread owns TMEM lane r = 32 (warp % 4) + lane, which is row
     // r % rows_blk of the Gram matrix of column segment r / rows_blk (columns c0 .. c0 + b of the lane) ----
