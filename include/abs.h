@@ -85,7 +85,7 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_cluster_rows" (target rows per CTA of the cluster kernel, 16..512),
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
  * cluster when b > 256),
- * "stats_no_gram" (1 = do not use the tensor-core Gram kernels for bf16, b <= 128),
+ * "stats_no_gram" (1 = do not use the tensor-core Gram kernels for bf16, b <= 256),
  * "stats_ctas_per_sm" (1: one CTA per SM, 64 KiB buffers, up to 16 rows per
  * thread; 2: two CTAs per SM, 32 KiB buffers, up to 8 rows per thread).
  * Unknown key or out-of-range value: ABS_ERR_INVALID_ARG. */
@@ -135,7 +135,7 @@ int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long lon
  * aligned != 0 means base address and strides are multiples of 16 bytes.          */
 typedef struct {
   int route;              /* 0 Gram (bf16, b <= 32), 1 cluster, 2 tiled, 3 generic two-sweep,
-                             4 Gram on tcgen05 (bf16, 32 < b <= 128)                          */
+                             4 Gram on tcgen05 (bf16, 32 < b <= 256)                          */
   int lanes_per_row;      /* 16-byte vectors per tile row: a tile row has 16*lanes_per_row bytes */
   int warps_per_box;      /* consumer warps that share one box of rows                        */
   int boxes_per_stage;

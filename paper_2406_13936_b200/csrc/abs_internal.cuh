@@ -81,7 +81,7 @@ struct StatsLaunch {
 // (alignment, b too large); *P_out receives the number of partial records per worker.
 int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
 int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // bf16, b <= 32
-int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // bf16, 32 < b <= 128 (tcgen05)
+int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // bf16, 32 < b <= 256 (tcgen05)
 int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out);   // 256 < b <= 4096
 int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
 int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P);

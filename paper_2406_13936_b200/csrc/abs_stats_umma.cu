@@ -1,4 +1,4 @@
-// Gram-matrix statistics kernel for bf16 rows and 32 < b <= 128 on the tcgen05 tensor cores, sm_100a.
+// Gram-matrix statistics kernel for bf16 rows and 32 < b <= 256 on the tcgen05 tensor cores, sm_100a.
 //
 // As in the small-batch Gram kernel, K = G G^T carries everything the batch-size test needs
 // (Eq. batch_grad and Eq. def_var expanded):
@@ -28,6 +28,15 @@
 // 128 rows and the B descriptor ceil16(.), so both may run into the next k-block: what they pick
 // up there lands in rows / columns of the accumulator that nobody reads.
 //
+// 128 < b <= 256: the rows form two blocks of 128.  A tile is then 128 columns (two k-blocks, so that
+// three stages still fit), and each k-step issues two MMAs: rows 0..127 against all rows
+// (K00 | K01, N = ceil16(b)) and rows 128.. against rows 128.. (K11, N = ceil16(b) - 128).  K10 is
+// not computed: the row sums of rows >= 128 take its part from the column sums of K01, which the
+// read-back warps form with a halving butterfly of shuffles (16 per 16 columns).  Both
+// accumulators of a fold take 2 ceil16(b) - 128 TMEM columns, so they alternate with a second
+// pair only while ceil16(b) <= 192; above, the MMAs wait while a fold is read back, and folds are
+// twice as long.
+//
 // Warp roles: 0-3 loaders, 4-7 accumulator read-back (warp w owns TMEM lanes 32 (w % 4) ..),
 // 8 MMA issue (one elected lane) and TMEM allocation, 9-12 column means on the CUDA cores when
 // gbar is wanted.  Every wait is bounded; a wait that runs out raises the CTA's abort flag, every
@@ -40,22 +49,26 @@ namespace absk {
 namespace {
 
 constexpr int kLoadWarps = 4;
-constexpr int kSubCols = 256;        // columns of one row segment: four k-blocks of 64 (128-byte swizzle span)
-constexpr int kFoldTilesDefault = 4;     // stages accumulated in TMEM before the fold into fp64
+constexpr int kFoldCols = 1024;       // columns added up in fp32 (TMEM) before the fold into fp64
 constexpr int kMaxStagesU = 8;
 constexpr int kBarsU = 2 * kMaxStagesU + 5;
 
 struct UmmaParams {
   const __nv_bfloat16* G;
   long long b, d, row_stride, worker_stride;   // strides in elements
-  int stack;              // column segments stacked as extra rows of the operand (1..3)
+  int stack;              // column segments stacked as extra rows of the operand (1..3; 1 when b > 128)
   int rows_blk;           // ceil8(b): rows one segment takes in a k-block
-  int n_dim;              // ceil16(stack * rows_blk): N of the MMA
-  int acc_cols;           // TMEM columns per accumulator (n_dim rounded up to a power of two >= 32)
+  int nkb;                // k-blocks (64 columns each) per segment: 4, or 2 when b > 128
+  int n_dim;              // N of the MMA on rows 0..127: ceil16(stack * rows_blk)
+  int n1_dim;             // N of the MMA on rows 128..: n_dim - 128 (0 when b <= 128)
+  int nbuf;               // accumulator sets that alternate between folds (2, or 1 when they do not fit twice)
+  int buf_stride;         // TMEM columns from one accumulator set to the next
+  int acc1_off;           // TMEM column of the second row block's accumulator inside a set
+  int tmem_cols;          // TMEM columns allocated (a power of two)
   int stages;
   int fold_tiles;         // stages accumulated in TMEM before the fold into fp64
   unsigned kb_bytes;      // stack * rows_blk * 128
-  unsigned stage_bytes;   // 4 k-blocks
+  unsigned stage_bytes;   // nkb k-blocks
   long long n_tiles;
   int P;
   double* ws;
@@ -124,7 +137,34 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
   for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
 }
 
-template <bool WANT_GBAR>
+// Sum over the 32 lanes of a warp of each of 16 per-lane values with a halving butterfly (16
+// shuffles): afterwards every lane holds the total of value index 8 b4 + 4 b3 + 2 b2 + b1, where
+// b4..b1 are bits 4..1 of its lane number (lanes 2k and 2k+1 hold the same total).
+__device__ __forceinline__ float warp_sum_16_values(const float (&v)[16], int lane) {
+  float w[8], x[4], y[2];
+  const bool h16 = (lane & 16) != 0, h8 = (lane & 8) != 0, h4 = (lane & 4) != 0, h2 = (lane & 2) != 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w[i] = (h16 ? v[8 + i] : v[i]) + __shfl_xor_sync(0xffffffffu, h16 ? v[i] : v[8 + i], 16);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) x[i] = (h8 ? w[4 + i] : w[i]) + __shfl_xor_sync(0xffffffffu, h8 ? w[i] : w[4 + i], 8);
+#pragma unroll
+  for (int i = 0; i < 2; ++i) y[i] = (h4 ? x[2 + i] : x[i]) + __shfl_xor_sync(0xffffffffu, h4 ? x[i] : x[2 + i], 4);
+  float z = (h2 ? y[1] : y[0]) + __shfl_xor_sync(0xffffffffu, h2 ? y[0] : y[1], 2);
+  z += __shfl_xor_sync(0xffffffffu, z, 1);
+  return z;
+}
+
+// red[] layout (doubles) in the CTA's tail of shared memory
+constexpr int kRedRow = 0;        // [256] row sums per TMEM-lane owner (second row block at +128)
+constexpr int kRedDiag = 256;     // [256] diagonal entries
+constexpr int kRedCol = 512;      // [4][128] column sums of K01 per read-back warp
+constexpr int kRedTot = 1024;     // total, trace
+constexpr int kRedRs = 1026;      // [256] (K 1)_i per row of G
+constexpr int kRedDg = 1282;      // [256] K_ii per row of G
+constexpr int kRedDoubles = 1538;
+
+// MB: row blocks of 128 (1: b <= 128, 2: b <= 256)
+template <int MB, bool WANT_GBAR>
 __global__ void __launch_bounds__(WANT_GBAR ? 416 : 288, 1)
 abs_stats_umma_kernel(const UmmaParams prm) {
   extern __shared__ unsigned char smem_dyn[];
@@ -137,12 +177,13 @@ abs_stats_umma_kernel(const UmmaParams prm) {
   const uint32_t raw_u32 = smem_u32(smem_dyn);
   const uint32_t ring_u32 = (raw_u32 + 1023u) & ~1023u;
   unsigned char* ring = smem_dyn + (ring_u32 - raw_u32);
-  const uint32_t pad = (128u - prm.kb_bytes / 128u) * 128u;       // room the 128-row A descriptor may run into
+  // room the operand descriptors (128 * MB rows from the start of a k-block) may run into
+  const uint32_t pad = (static_cast<uint32_t>(128 * MB) - prm.kb_bytes / 128u) * 128u;
   unsigned char* tail = ring + static_cast<size_t>(S) * prm.stage_bytes + pad;
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);
   volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + kBarsU);
   unsigned* tmem_slot = const_cast<unsigned*>(abort_flag) + 1;
-  double* red = reinterpret_cast<double*>(bars + kBarsU + 1);     // [128] row sums, [128] diagonal, [2], [128] + [128] per row of G
+  double* red = reinterpret_cast<double*>(bars + kBarsU + 1);
   const uint32_t full_u32 = smem_u32(bars);
   const uint32_t empty_u32 = full_u32 + 8u * kMaxStagesU;
   const uint32_t accfull_u32 = empty_u32 + 8u * kMaxStagesU;      // 2
@@ -162,7 +203,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  const uint32_t tmem_cols = static_cast<uint32_t>(2 * prm.acc_cols);
+  const uint32_t tmem_cols = static_cast<uint32_t>(prm.tmem_cols);
   if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"(tmem_cols)
@@ -176,34 +217,44 @@ abs_stats_umma_kernel(const UmmaParams prm) {
 
   const long long n_mine = (prm.n_tiles > p) ? (prm.n_tiles - p + prm.P - 1) / prm.P : 0;
   const __nv_bfloat16* Gm = prm.G + static_cast<long long>(m) * prm.worker_stride;
-  double row_sum = 0.0, row_diag = 0.0;
+  const int seg_cols = prm.nkb * 64;                                // columns of one row segment
+  const long long tile_cols = static_cast<long long>(prm.stack) * seg_cols;
+  double row_sum[MB], row_diag[MB], col_sum[MB == 2 ? 8 : 1];
+#pragma unroll
+  for (int k = 0; k < MB; ++k) row_sum[k] = row_diag[k] = 0.0;
+#pragma unroll
+  for (int k = 0; k < (MB == 2 ? 8 : 1); ++k) col_sum[k] = 0.0;
 
   if (warp < kLoadWarps) {
-    // ---- loaders: lane = 16-byte chunk of the tile row's 512 bytes, rows warp, warp + 4, ... ----
-    // The swizzle term depends on row % 8, which alternates between two values along a thread's rows.
-    const uint32_t kb_off = static_cast<uint32_t>(lane >> 3) * prm.kb_bytes + static_cast<uint32_t>(warp) * 128u;
-    const uint32_t swz0 = static_cast<uint32_t>((lane & 7) ^ warp) << 4;
-    const uint32_t swz1 = (static_cast<uint32_t>((lane & 7) ^ (warp + 4)) << 4) + 512u;
-    const long long step8 = 8 * prm.row_stride, step4 = 4 * prm.row_stride;
-    const __nv_bfloat16* row0 = Gm + static_cast<long long>(warp) * prm.row_stride;
-    const long long tile_cols = static_cast<long long>(prm.stack) * kSubCols;
+    // ---- loaders: a row segment is nkb * 8 chunks of 16 bytes; a warp instruction covers one segment
+    // row (nkb = 4) or two (nkb = 2); a thread keeps its chunk and walks down the rows.  The swizzle
+    // term depends on row % 8, which takes at most two values along a thread's rows. ----
+    const int cpr = prm.nkb * 8;
+    const int rstep = kLoadWarps * (32 / cpr);                      // 4 or 8
+    const int r0 = warp * (32 / cpr) + lane / cpr;
+    const int ch = lane % cpr;
+    const uint32_t kb_off = static_cast<uint32_t>(ch >> 3) * prm.kb_bytes + static_cast<uint32_t>(r0) * 128u;
+    const uint32_t swz_a = static_cast<uint32_t>((ch & 7) ^ (r0 & 7)) << 4;
+    const uint32_t swz_b = (static_cast<uint32_t>((ch & 7) ^ ((r0 + rstep) & 7)) << 4) + static_cast<uint32_t>(rstep) * 128u;
+    const long long step_b = static_cast<long long>(rstep) * prm.row_stride, step_a = 2 * step_b;
+    const __nv_bfloat16* row0 = Gm + static_cast<long long>(r0) * prm.row_stride;
     const uint32_t seg_bytes = static_cast<uint32_t>(prm.rows_blk) * 128u;
-    long long col0 = static_cast<long long>(p) * tile_cols + lane * 8;
+    long long col0 = static_cast<long long>(p) * tile_cols + ch * 8;
     int s = 0;
     uint32_t pass = 0;
     for (long long i = 0; i < n_mine; ++i) {
       if (pass > 0) mbar_wait_backoff(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles, 64);
       for (int t = 0; t < prm.stack; ++t) {
-        const long long col = col0 + t * kSubCols;
+        const long long col = col0 + t * seg_cols;
         const long long left = prm.d - col;                         // elements of a row from this chunk on
         const uint32_t bytes = left >= 8 ? 16u : (left > 0 ? static_cast<uint32_t>(left) * 2u : 0u);
         const __nv_bfloat16* src = row0 + (left > 0 ? col : 0);
         uint32_t dst = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(t) * seg_bytes + kb_off;
-        for (int row = warp; row < b; row += 8) {
-          cp_async_16(dst + swz0, src, bytes);                      // bytes past `bytes` are zero-filled
-          if (row + 4 < b) cp_async_16(dst + swz1, src + step4, bytes);
-          src += step8;
-          dst += 1024u;
+        for (int row = r0; row < b; row += 2 * rstep) {
+          cp_async_16(dst + swz_a, src, bytes);                     // bytes past `bytes` are zero-filled
+          if (row + rstep < b) cp_async_16(dst + swz_b, src + step_b, bytes);
+          src += step_a;
+          dst += static_cast<uint32_t>(2 * rstep) * 128u;
         }
       }
       // one arrival on the stage's barrier once this thread's copies have landed; nothing here
@@ -219,8 +270,10 @@ abs_stats_umma_kernel(const UmmaParams prm) {
   } else if (warp == 8) {
     // ---- MMA issue: the whole warp walks the loop (uniform control flow keeps the descriptors in
     // uniform registers), one elected lane issues ----
-    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(prm.n_dim >> 3) << 17) |
-                           (8u << 24);                              // fp32 accumulate, bf16 x bf16, K-major, M = 128
+    // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N / 8 at bit 17, M / 16 = 8 at bit 24
+    const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | (8u << 24);
+    const uint32_t idesc0 = idesc_base | (static_cast<uint32_t>(prm.n_dim >> 3) << 17);
+    const uint32_t idesc1 = idesc_base | (static_cast<uint32_t>(prm.n1_dim >> 3) << 17);
     // operand descriptor, K-major with 128-byte swizzle: start address / 16, 8-row groups 1024 bytes
     // apart (64 << 32), descriptor version 1 (bit 46), swizzle mode 2 (bits 61-63)
     const uint64_t desc_hi = (64ull << 32) | (1ull << 46) | (2ull << 61) | (1ull << 16);
@@ -228,22 +281,27 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     int s = 0, fold_pos = 0;
     uint32_t pass = 0, fold = 0;
     for (long long i = 0; i < n_mine; ++i) {
-      const uint32_t buf = fold & 1u;
-      if (fold_pos == 0 && fold >= 2)
-        mbar_wait(accempty_u32 + 8u * buf, ((fold >> 1) - 1) & 1u, abort_flag, prm.timeout_cycles);
+      const uint32_t buf = prm.nbuf == 2 ? (fold & 1u) : 0u;
+      const uint32_t use = prm.nbuf == 2 ? (fold >> 1) : fold;      // how often this accumulator set was used before
+      if (fold_pos == 0 && use > 0)
+        mbar_wait(accempty_u32 + 8u * buf, (use - 1) & 1u, abort_flag, prm.timeout_cycles);
       mbar_wait(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles);
       fence_async_smem();                                           // the copies' writes, before the tensor core reads
       tc_fence_after();
-      const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(prm.acc_cols);
+      const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(prm.buf_stride);
       const uint32_t lo = ((ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes) & 0x3ffffu) >> 4;
       const bool last_of_fold = fold_pos == prm.fold_tiles - 1 || i == n_mine - 1;
       if (elect_one()) {
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
+        for (int kb = 0; kb < prm.nkb; ++kb) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
+            const uint32_t acc = (fold_pos == 0 && kb == 0 && k == 0) ? 0u : 1u;
             const uint64_t desc = desc_hi | static_cast<uint64_t>(lo + static_cast<uint32_t>(kb) * kb16 + 2u * k);
-            umma_bf16(d_tmem, desc, desc, idesc, (fold_pos == 0 && kb == 0 && k == 0) ? 0u : 1u);
+            umma_bf16(d_tmem, desc, desc, idesc0, acc);
+            if (MB == 2) {
+              const uint64_t desc1 = desc + 1024u;                  // rows 128..: 128 rows * 128 bytes / 16
+              umma_bf16(d_tmem + static_cast<uint32_t>(prm.acc1_off), desc1, desc1, idesc1, acc);
+            }
           }
         }
         umma_commit(empty_u32 + 8u * s);                            // the stage may be refilled
@@ -266,19 +324,23 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     volatile unsigned ignore = 0u;
     mbar_wait(done_u32, 0u, &ignore, prm.timeout_cycles);           // no MMA in flight when TMEM is freed
   } else if (warp < 8) {
-    // ---- accumulator read-back: this thread owns TMEM lane r = 32 (warp % 4) + lane, which is row
-    // r % rows_blk of the Gram matrix of column segment r / rows_blk (columns c0 .. c0 + b of the lane) ----
+    // ---- accumulator read-back: this thread owns TMEM lane r = 32 (warp % 4) + lane.
+    // MB = 1: lane r is row r % rows_blk of the Gram matrix of column segment r / rows_blk, whose
+    //         columns sit at [c_first, c_first + b) of the lane.
+    // MB = 2: lane r of the first accumulator is row r of (K00 | K01), lane r of the second is row
+    //         128 + r of K11 (its columns start at 128). ----
     const int q = warp & 3;
     const int row = q * 32 + lane;
-    const int c_first = row / prm.rows_blk * prm.rows_blk;
-    const bool live = row < prm.stack * prm.rows_blk && row - c_first < b;
+    const int c_first = MB == 1 ? row / prm.rows_blk * prm.rows_blk : 0;
+    const bool live = MB == 1 ? (row < prm.stack * prm.rows_blk && row - c_first < b) : true;
     const int c_last = live ? c_first + b : 0;                      // columns [c_first, c_last) of this lane count
     const long long n_folds = (n_mine + prm.fold_tiles - 1) / prm.fold_tiles;
     for (long long f = 0; f < n_folds; ++f) {
-      const uint32_t buf = static_cast<uint32_t>(f) & 1u;
-      mbar_wait_backoff(accfull_u32 + 8u * buf, static_cast<uint32_t>(f >> 1) & 1u, abort_flag, prm.timeout_cycles, 256);
+      const uint32_t buf = prm.nbuf == 2 ? (static_cast<uint32_t>(f) & 1u) : 0u;
+      const uint32_t use = prm.nbuf == 2 ? static_cast<uint32_t>(f >> 1) : static_cast<uint32_t>(f);
+      mbar_wait_backoff(accfull_u32 + 8u * buf, use & 1u, abort_flag, prm.timeout_cycles, 256);
       tc_fence_after();
-      const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(prm.acc_cols) + (static_cast<uint32_t>(q * 32) << 16);
+      const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(prm.buf_stride) + (static_cast<uint32_t>(q * 32) << 16);
       float diag = 0.f;
       for (int c0 = 0; c0 < prm.n_dim; c0 += 16) {
         float v[16];
@@ -286,46 +348,70 @@ abs_stats_umma_kernel(const UmmaParams prm) {
         float part = 0.f;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          part += (c0 + j >= c_first && c0 + j < c_last) ? v[j] : 0.f;
+          const bool in = c0 + j >= c_first && c0 + j < c_last;
+          part += in ? v[j] : 0.f;
           diag = (c0 + j == row) ? v[j] : diag;
+          if (MB == 2 && !in) v[j] = 0.f;                           // columns >= b hold whatever the operand ran into
         }
-        row_sum += static_cast<double>(part);
+        row_sum[0] += static_cast<double>(part);
+        if (MB == 2 && c0 >= 128) {
+          // column sums of K01 = row sums of K10: over this warp's 32 rows here, over the warps at the end
+          col_sum[(c0 - 128) >> 4] += static_cast<double>(warp_sum_16_values(v, lane));
+        }
       }
-      row_diag += static_cast<double>(diag);
+      row_diag[0] += static_cast<double>(diag);
+      if (MB == 2) {
+        float diag1 = 0.f;
+        for (int c0 = 0; c0 < prm.n1_dim; c0 += 16) {
+          float v[16];
+          tmem_ld16(taddr + static_cast<uint32_t>(prm.acc1_off + c0), v);
+          float part = 0.f;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            part += (128 + c0 + j < b) ? v[j] : 0.f;
+            diag1 = (c0 + j == row) ? v[j] : diag1;
+          }
+          row_sum[MB - 1] += static_cast<double>(part);
+        }
+        row_diag[MB - 1] += static_cast<double>(diag1);
+      }
       tc_fence_before();
       mbar_arrive(accempty_u32 + 8u * buf);
     }
   } else if (WANT_GBAR) {
-    // ---- column means on the CUDA cores: warp 9 + kb owns k-block kb; lane = (row phase, 16-byte chunk) ----
-    const int kb = warp - 9;
-    const int sub = lane >> 3, ch = lane & 7;
+    // ---- column means on the CUDA cores: the four warps split a segment's nkb * 8 chunks of 16
+    // bytes; lane = (row phase, chunk); the row phases are folded with shuffles ----
+    const int w = warp - 9;
+    const int cw = prm.nkb * 2;                                     // chunks per warp: 8 or 4
+    const int nph = 32 / cw;                                        // row phases: 4 or 8
+    const int rph = lane / cw;
+    const int gch = w * cw + lane % cw;                             // chunk of the segment
+    const int kb = gch >> 3, ch = gch & 7;
     const float inv_b = 1.0f / static_cast<float>(b);
-    const long long tile_cols = static_cast<long long>(prm.stack) * kSubCols;
-    long long col0 = static_cast<long long>(p) * tile_cols + kb * 64 + ch * 8;
+    long long col0 = static_cast<long long>(p) * tile_cols + gch * 8;
     int s = 0;
     uint32_t pass = 0;
     for (long long i = 0; i < n_mine; ++i) {
       mbar_wait_backoff(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles, 32);
       for (int t = 0; t < prm.stack; ++t) {
-        const long long col = col0 + t * kSubCols;
+        const long long col = col0 + t * seg_cols;
         const uint32_t base = ring_u32 + static_cast<uint32_t>(s) * prm.stage_bytes +
                               static_cast<uint32_t>(kb) * prm.kb_bytes + static_cast<uint32_t>(t * prm.rows_blk) * 128u;
         float cs[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) cs[j] = 0.f;
-        for (int r = sub; r < b; r += 4) {
+        for (int r = rph; r < b; r += nph) {
           const uint4 u = lds128(base + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>(ch ^ (r & 7)) << 4));
           float x[8];
           Vec<__nv_bfloat16>::unpack(u, x);
 #pragma unroll
           for (int j = 0; j < 8; ++j) cs[j] += x[j];
         }
+        for (int off = cw; off < 32; off <<= 1) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 8);
-          cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], 16);
+          for (int j = 0; j < 8; ++j) cs[j] += __shfl_xor_sync(0xffffffffu, cs[j], off);
         }
-        if (sub == 0) {
+        if (rph == 0) {
           float* dst = prm.gbar_out + static_cast<long long>(m) * prm.d + col;
           if (col + 8 <= prm.d && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
             *reinterpret_cast<float4*>(dst) = make_float4(cs[0] * inv_b, cs[1] * inv_b, cs[2] * inv_b, cs[3] * inv_b);
@@ -349,9 +435,18 @@ abs_stats_umma_kernel(const UmmaParams prm) {
 
   // ---- CTA epilogue: (e_r, V, N) from the row sums and the diagonal of K ----
   if (warp >= 4 && warp < 8) {
-    const int row = (warp & 3) * 32 + lane;
-    red[row] = row_sum;
-    red[128 + row] = row_diag;
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+#pragma unroll
+    for (int k = 0; k < MB; ++k) {
+      red[kRedRow + 128 * k + row] = row_sum[k];
+      red[kRedDiag + 128 * k + row] = row_diag[k];
+    }
+    if (MB == 2 && (lane & 1) == 0) {
+      const int c = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+#pragma unroll
+      for (int g = 0; g < 8; ++g) red[kRedCol + q * 128 + g * 16 + c] = col_sum[g];
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -359,34 +454,41 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
   }
-  if (tid < b) {                                  // the segments' Gram matrices add up to the tile's
+  if (tid < b) {
     double rs = 0.0, dg = 0.0;
-    for (int t = 0; t < prm.stack; ++t) {
-      rs += red[t * prm.rows_blk + tid];
-      dg += red[128 + t * prm.rows_blk + tid];
+    if (MB == 1) {                                  // the segments' Gram matrices add up to the tile's
+      for (int t = 0; t < prm.stack; ++t) {
+        rs += red[kRedRow + t * prm.rows_blk + tid];
+        dg += red[kRedDiag + t * prm.rows_blk + tid];
+      }
+    } else {
+      rs = red[kRedRow + tid];
+      dg = red[kRedDiag + tid];
+      if (tid >= 128)
+        for (int wq = 0; wq < 4; ++wq) rs += red[kRedCol + wq * 128 + tid - 128];
     }
-    red[258 + tid] = rs;
-    red[386 + tid] = dg;
+    red[kRedRs + tid] = rs;
+    red[kRedDg + tid] = dg;
   }
   __syncthreads();
   if (tid == 0) {
     double total = 0.0, trace = 0.0;
     for (int i = 0; i < b; ++i) {
-      total += red[258 + i];
-      trace += red[386 + i];
+      total += red[kRedRs + i];
+      trace += red[kRedDg + i];
     }
-    red[256] = total;
-    red[257] = trace;
+    red[kRedTot] = total;
+    red[kRedTot + 1] = trace;
   }
   __syncthreads();
   {
     const double bd = static_cast<double>(b);
-    const double total = red[256], trace = red[257];
+    const double total = red[kRedTot], trace = red[kRedTot + 1];
     const double Ncta = total / (bd * bd);
     double* out = prm.ws + (static_cast<size_t>(m) * prm.P + p) * (static_cast<size_t>(b) + 2);
-    for (int i = tid; i < b; i += blockDim.x) out[i] = red[258 + i] / bd - Ncta;   // sum_j (g_ij - gbar_j) gbar_j
+    for (int i = tid; i < b; i += blockDim.x) out[i] = red[kRedRs + i] / bd - Ncta;   // sum_j (g_ij - gbar_j) gbar_j
     if (tid == 0) {
-      out[b] = trace - total / bd;                                             // sum_ij (g_ij - gbar_j)^2
+      out[b] = trace - total / bd;                                                   // sum_ij (g_ij - gbar_j)^2
       out[b + 1] = Ncta;
       if (*abort_flag) atomicOr(prm.flags, 1u);
     }
@@ -394,33 +496,57 @@ abs_stats_umma_kernel(const UmmaParams prm) {
 }
 
 struct UmmaGeom {
-  int rows_blk, stack, n_dim, acc_cols, stages;
+  int mblocks, rows_blk, stack, nkb, n_dim, n1_dim, nbuf, buf_stride, acc1_off, tmem_cols, stages, fold_tiles;
   unsigned kb_bytes, stage_bytes;
   size_t smem;
 };
 
 bool umma_geometry(const Tuning& t, size_t smem_optin, long long b, UmmaGeom* g) {
-  if (b <= 32 || b > 128) return false;
+  if (b <= 32 || b > 256) return false;
   g->rows_blk = static_cast<int>((b + 7) / 8 * 8);
-  g->stack = 128 / g->rows_blk;                   // 1 (b > 64), 2 (40 < b <= 64) or 3 (b <= 40)
-  g->n_dim = (g->stack * g->rows_blk + 15) / 16 * 16;
-  g->acc_cols = g->n_dim <= 64 ? 64 : 128;
+  if (b <= 128) {
+    g->mblocks = 1;
+    g->nkb = 4;
+    g->stack = 128 / g->rows_blk;                 // 1 (b > 64), 2 (40 < b <= 64) or 3 (b <= 40)
+    g->n_dim = (g->stack * g->rows_blk + 15) / 16 * 16;
+    g->n1_dim = 0;
+    g->nbuf = 2;
+    g->buf_stride = g->n_dim <= 64 ? 64 : 128;
+    g->acc1_off = 0;
+    g->tmem_cols = 2 * g->buf_stride;
+  } else {
+    g->mblocks = 2;
+    g->nkb = 2;                                   // 128-column tiles, so that three stages of 256 rows fit
+    g->stack = 1;
+    g->n_dim = static_cast<int>((b + 15) / 16 * 16);
+    g->n1_dim = g->n_dim - 128;
+    g->nbuf = g->n_dim <= 192 ? 2 : 1;            // n_dim + n1_dim columns per set, 512 in all
+    g->buf_stride = 256;
+    g->acc1_off = g->nbuf == 2 ? 192 : 256;
+    g->tmem_cols = 512;
+  }
   g->kb_bytes = static_cast<unsigned>(g->stack * g->rows_blk) * 128u;
-  g->stage_bytes = 4u * g->kb_bytes;
-  const size_t pad = static_cast<size_t>(128 - g->stack * g->rows_blk) * 128;
-  const size_t fixed = 1024 + pad + static_cast<size_t>(kBarsU + 1) * 8 + 514 * sizeof(double) + 128;
+  g->stage_bytes = static_cast<unsigned>(g->nkb) * g->kb_bytes;
+  const size_t pad = static_cast<size_t>(128 * g->mblocks - g->stack * g->rows_blk) * 128;
+  const size_t fixed = 1024 + pad + static_cast<size_t>(kBarsU + 1) * 8 + kRedDoubles * sizeof(double) + 128;
   int stages = static_cast<int>(t.stats_stages > 0 ? t.stats_stages : kMaxStagesU);
   if (stages > kMaxStagesU) stages = kMaxStagesU;
   while (stages > 2 && static_cast<size_t>(stages) * g->stage_bytes + fixed > smem_optin) --stages;
   g->stages = stages;
   g->smem = static_cast<size_t>(stages) * g->stage_bytes + fixed;
   if (g->smem > smem_optin) return false;
+  // about kFoldCols columns are added up in fp32 before the fold into fp64; twice as many where the
+  // MMAs have to wait for the read-back
+  const int tile_cols = g->stack * g->nkb * 64;
+  int fold = (g->nbuf == 2 ? kFoldCols : 2 * kFoldCols) / tile_cols;
+  if (t.stats_flush_every > 0) fold = static_cast<int>(t.stats_flush_every > 64 ? 64 : t.stats_flush_every);
+  g->fold_tiles = fold < 1 ? 1 : fold;
   return true;
 }
 
-template <bool WANT_GBAR>
+template <int MB, bool WANT_GBAR>
 int launch_umma_variant(abs_ctx* ctx, const UmmaParams& prm, dim3 grid, size_t smem, cudaStream_t stream) {
-  auto kern = abs_stats_umma_kernel<WANT_GBAR>;
+  auto kern = abs_stats_umma_kernel<MB, WANT_GBAR>;
   ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   kern<<<grid, WANT_GBAR ? 416 : 288, smem, stream>>>(prm);
   ABS_CUDA_TRY(ctx, cudaGetLastError());
@@ -436,7 +562,7 @@ int plan_stats_umma(const Tuning& t, size_t smem_optin, abs_dtype dtype, long lo
   out->route = 4;
   out->lanes_per_row = 8;                    // a k-block row: 128 bytes
   out->warps_per_box = kLoadWarps;
-  out->boxes_per_stage = 4;                  // k-blocks
+  out->boxes_per_stage = g.nkb;              // k-blocks
   out->stages = g.stages;
   out->box_rows = g.stack * g.rows_blk;
   out->row_boxes = 1;
@@ -448,7 +574,7 @@ int plan_stats_umma(const Tuning& t, size_t smem_optin, abs_dtype dtype, long lo
   return ABS_OK;
 }
 
-// Takes the call for bf16 rows with 32 < b <= 128 whose base and strides are multiples of 16 bytes.
+// Takes the call for bf16 rows with 32 < b <= 256 whose base and strides are multiples of 16 bytes.
 int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if (a.dtype != ABS_BF16) return ABS_ERR_UNSUPPORTED;
   UmmaGeom g;
@@ -458,7 +584,7 @@ int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if ((reinterpret_cast<uintptr_t>(a.G) & 15u) || (row_b & 15u) || (wrk_b & 15u) || a.M > 65535)
     return ABS_ERR_UNSUPPORTED;
 
-  const long long tile_cols = static_cast<long long>(g.stack) * kSubCols;
+  const long long tile_cols = static_cast<long long>(g.stack) * g.nkb * 64;
   const long long n_tiles = (a.d + tile_cols - 1) / tile_cols;
   long long P = ctx->tuning.stats_ctas_per_worker > 0 ? ctx->tuning.stats_ctas_per_worker
                                                       : static_cast<long long>(ctx->sm_count) / a.M;
@@ -477,11 +603,15 @@ int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.worker_stride = a.M > 1 ? a.worker_stride : 0;
   prm.stack = g.stack;
   prm.rows_blk = g.rows_blk;
+  prm.nkb = g.nkb;
   prm.n_dim = g.n_dim;
-  prm.acc_cols = g.acc_cols;
+  prm.n1_dim = g.n1_dim;
+  prm.nbuf = g.nbuf;
+  prm.buf_stride = g.buf_stride;
+  prm.acc1_off = g.acc1_off;
+  prm.tmem_cols = g.tmem_cols;
   prm.stages = g.stages;
-  prm.fold_tiles = static_cast<int>(ctx->tuning.stats_flush_every > 0 ? (ctx->tuning.stats_flush_every > 64 ? 64 : ctx->tuning.stats_flush_every)
-                                                                      : kFoldTilesDefault);
+  prm.fold_tiles = g.fold_tiles;
   prm.kb_bytes = g.kb_bytes;
   prm.stage_bytes = g.stage_bytes;
   prm.n_tiles = n_tiles;
@@ -491,8 +621,14 @@ int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.flags = ctx->flags;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
-  const int rc = a.gbar_out != nullptr ? launch_umma_variant<true>(ctx, prm, grid, g.smem, a.stream)
-                                       : launch_umma_variant<false>(ctx, prm, grid, g.smem, a.stream);
+  const bool gb = a.gbar_out != nullptr;
+  int rc;
+  if (g.mblocks == 1)
+    rc = gb ? launch_umma_variant<1, true>(ctx, prm, grid, g.smem, a.stream)
+            : launch_umma_variant<1, false>(ctx, prm, grid, g.smem, a.stream);
+  else
+    rc = gb ? launch_umma_variant<2, true>(ctx, prm, grid, g.smem, a.stream)
+            : launch_umma_variant<2, false>(ctx, prm, grid, g.smem, a.stream);
   if (rc != ABS_OK) return rc;
   *P_out = static_cast<int>(P);
   return ABS_OK;

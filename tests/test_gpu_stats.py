@@ -163,9 +163,12 @@ def test_gram_and_tiled_kernels_agree_on_bf16(ctx, M, b, d):
 @pytest.mark.parametrize("want_gbar", [False, True])
 @pytest.mark.parametrize("M,b,d,pad", [(1, 33, 2048, 0), (2, 40, 5003, 5), (1, 64, 9000, 0), (3, 100, 4104, 0),
                                        (1, 128, 8200, 8), (1, 96, 300, 4), (1, 128, 300000, 0), (2, 72, 150001, 7),
-                                       (1, 48, 256, 0), (1, 127, 1025, 7)])
+                                       (1, 48, 256, 0), (1, 127, 1025, 7), (1, 50, 1, 7), (1, 33, 8, 0),
+                                       (4, 128, 40000, 0), (1, 65, 2000, 0), (5, 41, 7777, 7),
+                                       (1, 129, 3000, 0), (2, 136, 5003, 5), (1, 160, 40000, 0), (1, 192, 9000, 0),
+                                       (1, 200, 70001, 7), (3, 255, 2049, 7), (1, 256, 100000, 0), (1, 256, 128, 0)])
 def test_tcgen05_gram_kernel_matches_oracle_and_tiled_kernel(ctx, M, b, d, pad, want_gbar):
-    """bf16 input with 32 < b <= 128 and 16-byte aligned rows goes through the tcgen05 Gram kernel
+    """bf16 input with 32 < b <= 256 and 16-byte aligned rows goes through the tcgen05 Gram kernel
     (with and without the column-mean warps); the tiled kernel must give the same statistics, and
     both must match the oracle, also with a ragged last tile and a last 16-byte chunk cut by d."""
     assert pkg.plan_stats("bf16", b)["route"] == 4

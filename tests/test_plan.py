@@ -25,15 +25,21 @@ def check_plan(dtype, b, p):
         assert dtype == "bf16" and b <= 32 and p["box_rows"] == b
         return
     if p["route"] == 4:
-        # tcgen05 Gram kernel: k-blocks of 1..3 column segments x ceil8(b) rows x 128 bytes, each k-block
-        # on a 1024-byte boundary, at most 128 operand rows
-        assert dtype == "bf16" and 32 < b <= 128
+        # tcgen05 Gram kernel: k-blocks of 128-byte rows, each k-block on a 1024-byte boundary.
+        # b <= 128: 1..3 column segments of ceil8(b) rows stacked, at most 128 operand rows, 4 k-blocks
+        # per stage; b > 128: two row blocks of 128, 2 k-blocks per stage.
+        assert dtype == "bf16" and 32 < b <= 256
         rows_blk = (b + 7) // 8 * 8
-        assert p["box_rows"] == (128 // rows_blk) * rows_blk and p["rows_per_cta"] == b
-        assert lpr == 8 and p["boxes_per_stage"] == 4
-        assert p["stage_bytes"] == 4 * p["box_rows"] * 128 and (p["stage_bytes"] // 4) % 1024 == 0
-        # the 128-row operand descriptor of the last k-block stays inside the allocation
-        assert p["stages"] * p["stage_bytes"] + (128 - p["box_rows"]) * 128 + 1024 <= p["smem_bytes"]
+        mblocks = 1 if b <= 128 else 2
+        if mblocks == 1:
+            assert p["box_rows"] == (128 // rows_blk) * rows_blk and p["boxes_per_stage"] == 4
+        else:
+            assert p["box_rows"] == rows_blk and p["boxes_per_stage"] == 2
+        assert lpr == 8 and p["rows_per_cta"] == b
+        assert p["stage_bytes"] == p["boxes_per_stage"] * p["box_rows"] * 128
+        assert (p["stage_bytes"] // p["boxes_per_stage"]) % 1024 == 0
+        # the operand descriptors (128 rows per row block) of the last k-block stay inside the allocation
+        assert p["stages"] * p["stage_bytes"] + (128 * mblocks - p["box_rows"]) * 128 + 1024 <= p["smem_bytes"]
         return
     groups = p["warps_per_box"] * 32 // lpr                  # row groups that share a box
     R = p["rows_per_thread"]
@@ -63,7 +69,7 @@ def test_every_batch_size_gets_a_valid_plan(dtype):
         p = pkg.plan_stats(dtype, b)
         if dtype == "bf16" and b <= 32:
             assert p["route"] == 0
-        elif dtype == "bf16" and b <= 128:
+        elif dtype == "bf16" and b <= 256:
             assert p["route"] == 4
         elif b > 256:
             assert p["route"] == 1
@@ -93,3 +99,5 @@ def test_documented_shapes():
     assert (p["route"], p["stages"], p["stage_bytes"]) == (4, 3, 65536)
     p = pkg.plan_stats("bf16", 33)
     assert (p["route"], p["stages"], p["box_rows"]) == (4, 3, 120)
+    p = pkg.plan_stats("bf16", 256)
+    assert (p["route"], p["stages"], p["stage_bytes"], p["boxes_per_stage"]) == (4, 3, 65536, 2)
