@@ -49,7 +49,7 @@ namespace absk {
 namespace {
 
 constexpr int kLoadWarps = 4;
-constexpr int kFoldCols = 1024;       // columns added up in fp32 (TMEM) before the fold into fp64
+constexpr int kFoldCols = 4096;       // columns added up in fp32 (TMEM) before the fold into fp64
 constexpr int kMaxStagesU = 8;
 constexpr int kBarsU = 2 * kMaxStagesU + 5;
 
@@ -124,17 +124,24 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
+// 32 consecutive accumulator columns of this thread's TMEM lane: two loads in flight, one wait.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[2][16]) {
+  uint32_t r[32];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%32];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];\n\t"
       "tcgen05.wait::ld.sync.aligned;"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr), "r"(taddr + 16u)
       : "memory");
 #pragma unroll
-  for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+  for (int j = 0; j < 16; ++j) {
+    v[0][j] = __uint_as_float(r[j]);
+    v[1][j] = __uint_as_float(r[16 + j]);
+  }
 }
 
 // Sum over the 32 lanes of a warp of each of 16 per-lane values with a halving butterfly (16
@@ -342,34 +349,42 @@ abs_stats_umma_kernel(const UmmaParams prm) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(prm.buf_stride) + (static_cast<uint32_t>(q * 32) << 16);
       float diag = 0.f;
-      for (int c0 = 0; c0 < prm.n_dim; c0 += 16) {
-        float v[16];
-        tmem_ld16(taddr + static_cast<uint32_t>(c0), v);
-        float part = 0.f;
+      for (int c32 = 0; c32 < prm.n_dim; c32 += 32) {               // n_dim is a multiple of 16: the last pair may
+        float v[2][16];                                             // read 16 columns past it, inside the allocation
+        tmem_ld32(taddr + static_cast<uint32_t>(c32), v);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const bool in = c0 + j >= c_first && c0 + j < c_last;
-          part += in ? v[j] : 0.f;
-          diag = (c0 + j == row) ? v[j] : diag;
-          if (MB == 2 && !in) v[j] = 0.f;                           // columns >= b hold whatever the operand ran into
-        }
-        row_sum[0] += static_cast<double>(part);
-        if (MB == 2 && c0 >= 128) {
-          // column sums of K01 = row sums of K10: over this warp's 32 rows here, over the warps at the end
-          col_sum[(c0 - 128) >> 4] += static_cast<double>(warp_sum_16_values(v, lane));
+        for (int h = 0; h < 2; ++h) {
+          const int c0 = c32 + 16 * h;
+          float part = 0.f;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const bool in = c0 + j >= c_first && c0 + j < c_last;
+            part += in ? v[h][j] : 0.f;
+            diag = (c0 + j == row) ? v[h][j] : diag;
+            if (MB == 2 && !in) v[h][j] = 0.f;                      // columns >= b hold whatever the operand ran into
+          }
+          row_sum[0] += static_cast<double>(part);
+          if (MB == 2 && c0 >= 128 && c0 < prm.n_dim) {
+            // column sums of K01 = row sums of K10: over this warp's 32 rows here, over the warps at the end
+            col_sum[(c0 - 128) >> 4] += static_cast<double>(warp_sum_16_values(v[h], lane));
+          }
         }
       }
       row_diag[0] += static_cast<double>(diag);
       if (MB == 2) {
         float diag1 = 0.f;
-        for (int c0 = 0; c0 < prm.n1_dim; c0 += 16) {
-          float v[16];
-          tmem_ld16(taddr + static_cast<uint32_t>(prm.acc1_off + c0), v);
+        for (int c32 = 0; c32 < prm.n1_dim; c32 += 32) {
+          float v[2][16];
+          tmem_ld32(taddr + static_cast<uint32_t>(prm.acc1_off + c32), v);
           float part = 0.f;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            part += (128 + c0 + j < b) ? v[j] : 0.f;
-            diag1 = (c0 + j == row) ? v[j] : diag1;
+          for (int h = 0; h < 2; ++h) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int c = c32 + 16 * h + j;
+              part += (128 + c < b) ? v[h][j] : 0.f;
+              diag1 = (c == row) ? v[h][j] : diag1;
+            }
           }
           row_sum[MB - 1] += static_cast<double>(part);
         }
