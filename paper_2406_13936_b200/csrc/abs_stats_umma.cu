@@ -75,6 +75,7 @@ struct UmmaParams {
   float* gbar_out;
   unsigned* flags;
   long long timeout_cycles;
+  int drop_loads;         // fault injection for the bounded waits: the loaders issue nothing
 };
 
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
@@ -251,7 +252,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
     uint32_t pass = 0;
     for (long long i = 0; i < n_mine; ++i) {
       if (pass > 0) mbar_wait_backoff(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles, 64);
-      for (int t = 0; t < prm.stack; ++t) {
+      for (int t = 0; t < (prm.drop_loads ? 0 : prm.stack); ++t) {  // test hook: no copies, no arrival; the waits run out
         const long long col = col0 + t * seg_cols;
         const long long left = prm.d - col;                         // elements of a row from this chunk on
         const uint32_t bytes = left >= 8 ? 16u : (left > 0 ? static_cast<uint32_t>(left) * 2u : 0u);
@@ -266,7 +267,8 @@ abs_stats_umma_kernel(const UmmaParams prm) {
       }
       // one arrival on the stage's barrier once this thread's copies have landed; nothing here
       // waits for them, so the loaders run a whole ring ahead of the tensor core
-      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_u32 + 8u * s) : "memory");
+      if (!prm.drop_loads)
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full_u32 + 8u * s) : "memory");
       col0 += static_cast<long long>(prm.P) * tile_cols;
       if (++s == S) {
         s = 0;
@@ -635,6 +637,7 @@ int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
+  prm.drop_loads = ctx->tuning.stats_fault_drop_loads ? 1 : 0;
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
   const bool gb = a.gbar_out != nullptr;
   int rc;
