@@ -225,9 +225,9 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
                                  frac_of_peak=gbs / peak)
         del G
         torch.cuda.empty_cache()
-    # bf16 statistics with more rows per worker: the tcgen05 Gram kernel (32 < b <= 128)
+    # bf16 statistics with more rows per worker: the tcgen05 Gram kernel (32 < b <= 256)
     if torch.cuda.mem_get_info()[0] > 20e9:
-        for bb, dd in ((64, 22_400_000), (128, 11_200_000)):
+        for bb, dd in ((64, 22_400_000), (128, 11_200_000), (256, 11_200_000)):
             G = inputs.gaussian_rows(2, 1, bb, dd, 1.0, device="cuda", dtype=torch.bfloat16)
             stats = ctx.new_stats(1)
             sec = time_steps(torch, lambda i: ctx.abs_test_stats(G, stats), 10, 3)
@@ -301,6 +301,7 @@ PROFILE_CASES = {
     "stats_bf16_b16": dict(kind="stats", M=8, b=16, d=4_000_000, dtype="bf16"),
     "stats_bf16_b64": dict(kind="stats", M=1, b=64, d=8_000_000, dtype="bf16"),
     "stats_bf16_b128": dict(kind="stats", M=1, b=128, d=4_000_000, dtype="bf16"),
+    "stats_bf16_b256": dict(kind="stats", M=1, b=256, d=2_000_000, dtype="bf16"),
     "adamw": dict(kind="adamw", M=8, d=8_000_000),
     # full-size cases of the sweep, for timing only (not for multi-pass captures)
     "stats_f32_b64_d11m": dict(kind="stats", M=1, b=64, d=11_200_000, dtype="f32"),
