@@ -143,7 +143,159 @@ sgemm_kernel(const GemmArgs g) {
   }
 }
 
+// ---- the same GEMM for large operands: 128 x 128 tiles, 8 x 8 outputs per thread -------------
+// Operand tiles are fetched 16 bytes at a time along whichever index is contiguous in memory
+// (rows or k for A, k or columns for B), one 16-deep slice ahead of the arithmetic (registers ->
+// the other shared-memory buffer), so a slice costs one barrier.  Slices are summed in fp32 and
+// folded into fp64 as in sgemm_kernel; the results are bit-identical to it (same products, same
+// order of additions per output).
+constexpr int kBig = 128;
+
+// Four consecutive elements along the contiguous index starting at p; elements at or past `left`
+// (counted from p) read as zero.  `vec` says that p is 16-byte aligned.
+__device__ __forceinline__ float4 load4_guarded(const float* p, long long left, bool vec) {
+  if (left >= 4 && vec) return __ldg(reinterpret_cast<const float4*>(p));
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (left > 0) v.x = __ldg(p);
+  if (left > 1) v.y = __ldg(p + 1);
+  if (left > 2) v.z = __ldg(p + 2);
+  if (left > 3) v.w = __ldg(p + 3);
+  return v;
+}
+
+// A_KCONT: k is the contiguous index of A (a_cs == 1), else the row index is (a_rs == 1).
+// B_KCONT: k is the contiguous index of B (b_rs == 1), else the column index is (b_cs == 1).
+template <bool A_KCONT, bool B_KCONT>
+__global__ void __launch_bounds__(256, 1)
+sgemm_big_kernel(const GemmArgs g) {
+  __shared__ __align__(16) float As[2][kTileK][kBig + 4];
+  __shared__ __align__(16) float Bs[2][kTileK][kBig + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int z = blockIdx.z;
+  const long long r0 = static_cast<long long>(blockIdx.y) * kBig, c0 = static_cast<long long>(blockIdx.x) * kBig;
+  const float* A = g.A + z * g.a_bs;
+  const float* B = g.B + z * g.b_bs;
+  // 16-byte loads need an aligned base and a stride of the other index that keeps the alignment
+  const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && ((A_KCONT ? g.a_rs : g.a_cs) & 3) == 0;
+  const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && ((B_KCONT ? g.b_cs : g.b_rs) & 3) == 0;
+
+  // this thread's two 16-byte pieces of each operand tile (piece e = tid, tid + 256)
+  //   k contiguous:  e -> (index e / 4 of the tile, k quad e % 4)
+  //   else:          e -> (k = e / 32, quad e % 32 of the 128 rows / columns)
+  float4 ra[2], rb[2];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int e = tid + 256 * t;
+      if (A_KCONT) {
+        const long long r = r0 + (e >> 2);
+        const int k = k0 + 4 * (e & 3);
+        ra[t] = load4_guarded(A + r * g.a_rs + k, r < g.rows ? g.K - k : 0, a_vec);
+      } else {
+        const int k = k0 + (e >> 5);
+        const long long r = r0 + 4 * (e & 31);
+        ra[t] = load4_guarded(A + k * g.a_cs + r, k < g.K ? g.rows - r : 0, a_vec);
+      }
+      if (B_KCONT) {
+        const long long c = c0 + (e >> 2);
+        const int k = k0 + 4 * (e & 3);
+        rb[t] = load4_guarded(B + c * g.b_cs + k, c < g.cols ? g.K - k : 0, b_vec);
+      } else {
+        const int k = k0 + (e >> 5);
+        const long long c = c0 + 4 * (e & 31);
+        rb[t] = load4_guarded(B + k * g.b_rs + c, k < g.K ? g.cols - c : 0, b_vec);
+      }
+    }
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+      const int e = tid + 256 * t;
+      if (A_KCONT) {
+        const int r = e >> 2, k = 4 * (e & 3);
+        As[buf][k][r] = ra[t].x; As[buf][k + 1][r] = ra[t].y; As[buf][k + 2][r] = ra[t].z; As[buf][k + 3][r] = ra[t].w;
+      } else {
+        *reinterpret_cast<float4*>(&As[buf][e >> 5][4 * (e & 31)]) = ra[t];
+      }
+      if (B_KCONT) {
+        const int c = e >> 2, k = 4 * (e & 3);
+        Bs[buf][k][c] = rb[t].x; Bs[buf][k + 1][c] = rb[t].y; Bs[buf][k + 2][c] = rb[t].z; Bs[buf][k + 3][c] = rb[t].w;
+      } else {
+        *reinterpret_cast<float4*>(&Bs[buf][e >> 5][4 * (e & 31)]) = rb[t];
+      }
+    }
+  };
+
+  double dacc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) dacc[i][j] = 0.0;
+
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = 0; k0 < g.K; k0 += kTileK) {
+    const bool more = k0 + kTileK < g.K;
+    if (more) fetch(k0 + kTileK);
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+#pragma unroll
+    for (int k = 0; k < kTileK; ++k) {
+      // rows ty*4 .. +3 and 64 + ty*4 .. +3; columns tx*4 .. +3 and 64 + tx*4 .. +3
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][k][ty * 4]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[buf][k][64 + ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][k][tx * 4]);
+      const float4 b1 = *reinterpret_cast<const float4*>(&Bs[buf][k][64 + tx * 4]);
+      const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) dacc[i][j] += static_cast<double>(acc[i][j]);
+    if (more) stash(buf ^ 1);
+    __syncthreads();
+    buf ^= 1;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const long long r = r0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + i - 4);
+    if (r >= g.rows) continue;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const long long c = c0 + (j < 4 ? tx * 4 + j : 64 + tx * 4 + j - 4);
+      if (c >= g.cols) continue;
+      float v = static_cast<float>(g.mode == 0 ? dacc[i][j] * static_cast<double>(g.alpha) : dacc[i][j]);
+      if (g.mode == 0) {}
+      else if (g.mode == 1) v = fmaxf(static_cast<float>(dacc[i][j] + g.bias[z * g.bias_bs + c]), 0.f);
+      else if (g.mode == 2) v = static_cast<float>(dacc[i][j] + g.bias[z * g.bias_bs + c]);
+      else v = g.mask[z * g.mask_bs + r * g.mask_rs + c] > 0.f ? v : 0.f;
+      g.C[z * g.c_bs + r * g.c_rs + c] = v;
+    }
+  }
+}
+
 void launch_gemm(const GemmArgs& g, int batch, cudaStream_t st) {
+  // the large-tile kernel where a 128 x 128 tile is mostly used and both operands have a contiguous index
+  const bool a_ok = g.a_cs == 1 || g.a_rs == 1, b_ok = g.b_rs == 1 || g.b_cs == 1;
+  if (a_ok && b_ok && g.rows >= 96 && g.cols >= 96) {
+    const dim3 big((g.cols + kBig - 1) / kBig, (g.rows + kBig - 1) / kBig, batch);
+    const bool ak = g.a_cs == 1, bk = g.b_rs == 1;
+    if (ak && bk) sgemm_big_kernel<true, true><<<big, 256, 0, st>>>(g);
+    else if (ak) sgemm_big_kernel<true, false><<<big, 256, 0, st>>>(g);
+    else if (bk) sgemm_big_kernel<false, true><<<big, 256, 0, st>>>(g);
+    else sgemm_big_kernel<false, false><<<big, 256, 0, st>>>(g);
+    return;
+  }
   const dim3 grid((g.cols + kTile - 1) / kTile, (g.rows + kTile - 1) / kTile, batch);
   sgemm_kernel<<<grid, 256, 0, st>>>(g);
 }
@@ -178,16 +330,26 @@ __global__ void softmax_delta_kernel(float* __restrict__ scratch, long long per_
   for (int c = 0; c < n3; ++c) z[c] = z[c] / sum - (c == label ? 1.f : 0.f);
 }
 
-// db[o] = (1/b) sum_i D[i][o]; one thread per output unit and worker.
-__global__ void bias_grad_kernel(const float* __restrict__ scratch, long long per_worker, long long off, long long b,
-                                 int n, float* __restrict__ Gb, long long d, long long ob) {
-  const int m = blockIdx.y;
-  const int o = blockIdx.x * blockDim.x + threadIdx.x;
-  if (o >= n) return;
+// db[o] = (1/b) sum_i D[i][o].  A CTA covers 32 output units of one worker: warp w sums the rows
+// w, w + 32, ... of its 32 columns (128 contiguous bytes per row) in fp64, then the 32 partial sums
+// of a column are added in warp order, so the result does not depend on the launch.
+__global__ void __launch_bounds__(1024)
+bias_grad_kernel(const float* __restrict__ scratch, long long per_worker, long long off, long long b, int n,
+                 float* __restrict__ Gb, long long d, long long ob) {
+  __shared__ double part[32][33];
+  const int m = blockIdx.y, lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int o = blockIdx.x * 32 + lane;
   const float* D = scratch + m * per_worker + off;
   double acc = 0.0;
-  for (long long i = 0; i < b; ++i) acc += static_cast<double>(D[i * n + o]);
-  Gb[m * d + ob + o] = static_cast<float>(acc / static_cast<double>(b));
+  if (o < n)
+    for (long long i = w; i < b; i += 32) acc += static_cast<double>(D[i * n + o]);
+  part[w][lane] = acc;
+  __syncthreads();
+  if (w == 0 && o < n) {
+    double tot = 0.0;
+    for (int k = 0; k < 32; ++k) tot += part[k][lane];
+    Gb[m * d + ob + o] = static_cast<float>(tot / static_cast<double>(b));
+  }
 }
 
 // Row i of G: the flat gradient of sample i of one worker.  The weight segment of a layer is the
@@ -460,9 +622,9 @@ extern "C" int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* label
   g = GemmArgs{ws + s.sD1, 1, s.n1, pw, ws + s.sX, s.n0, 1, pw, Gb + s.oW1, s.n0, d, nullptr, 0, nullptr, 0, 0,
                s.n1, s.n0, static_cast<int>(b), inv_b, 0};
   launch_gemm(g, M, st);
-  bias_grad_kernel<<<dim3((s.n3 + 127) / 128, M), 128, 0, st>>>(ws, pw, s.sD3, b, s.n3, Gb, d, s.ob3);
-  bias_grad_kernel<<<dim3((s.n2 + 127) / 128, M), 128, 0, st>>>(ws, pw, s.sD2, b, s.n2, Gb, d, s.ob2);
-  bias_grad_kernel<<<dim3((s.n1 + 127) / 128, M), 128, 0, st>>>(ws, pw, s.sD1, b, s.n1, Gb, d, s.ob1);
+  bias_grad_kernel<<<dim3((s.n3 + 31) / 32, M), 1024, 0, st>>>(ws, pw, s.sD3, b, s.n3, Gb, d, s.ob3);
+  bias_grad_kernel<<<dim3((s.n2 + 31) / 32, M), 1024, 0, st>>>(ws, pw, s.sD2, b, s.n2, Gb, d, s.ob2);
+  bias_grad_kernel<<<dim3((s.n1 + 31) / 32, M), 1024, 0, st>>>(ws, pw, s.sD1, b, s.n1, Gb, d, s.ob1);
   const cudaError_t e = cudaGetLastError();
   if (prev != ctx->device) cudaSetDevice(prev);
   if (e != cudaSuccess) return set_error(ctx, ABS_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
