@@ -382,7 +382,10 @@ def test_mean_dominated_rows(ctx, b, d, offset, noise):
 
 @pytest.mark.parametrize("dtype,M,b,d,d0", [(torch.float32, 1, 256, 11_200_000, 100_003),
                                             (torch.float32, 1, 1024, 2_800_000, 50_003),
-                                            (torch.bfloat16, 8, 16, 124_439_808, 250_007)])
+                                            (torch.bfloat16, 8, 16, 124_439_808, 250_007),
+                                            (torch.bfloat16, 1, 64, 22_400_000, 100_003),
+                                            (torch.bfloat16, 8, 128, 2_000_000, 100_003),
+                                            (torch.bfloat16, 1, 256, 5_600_000, 50_003)])
 def test_full_size_launch_configuration(ctx, dtype, M, b, d, d0):
     # the benchmark's launch shape (same b, M, dtype; d as large as a test should hold), checked
     # through the column-periodic property that holds at any width
