@@ -349,6 +349,47 @@ def run_profile_case(args):
     ctx.close()
 
 
+def run_sweep(args):
+    """The statistics sweep: b in {64, 256, 1024} x d in {1 M, 11.2 M, 25.6 M}, fp32, M = 1, each case
+    abs_test_stats followed by abs_next_batch for the norm and the augmented inner-product test.
+    The variance of the rows does not change what is read, so the sweep runs sigma = 1 only.
+    Inputs under 1 GB rotate over 4 buffers so that L2 does not serve them; one JSON line."""
+    import torch
+    import paper_2406_13936_b200 as pkg
+    from paper_2406_13936_b200 import inputs
+    pkg.build.build()
+    ctx = pkg.Context(0)
+    peak, peak_kind = measured_peak()
+    cfgs = [pkg.make_test_cfg("norm", 1 << 20, eta=0.5), pkg.make_test_cfg("aug_ip", 1 << 20, theta=0.5, nu=0.5)]
+    table = []
+    for b in (64, 256, 1024):
+        for d in (1_000_000, 11_200_000, 25_600_000):
+            nbytes = 4 * b * d
+            if nbytes + (8 << 30) > torch.cuda.mem_get_info()[0]:
+                table.append(dict(b=b, d=d, note="does not fit on this device"))
+                continue
+            copies = 4 if nbytes < (1 << 30) else 1
+            Gs = [inputs.gaussian_rows(2 + k, 1, b, d, 1.0, device="cuda") for k in range(copies)]
+            stats = ctx.new_stats(1)
+            b_cur = torch.tensor([b], dtype=torch.int64, device="cuda")
+            b_next = torch.zeros(1, dtype=torch.int64, device="cuda")
+
+            def step(i):
+                ctx.abs_test_stats(Gs[i % copies], stats)
+                for cfg in cfgs:
+                    ctx.abs_next_batch(stats, cfg, b_cur, b_next)
+
+            sec = time_steps(torch, step, args.steps, args.warmup)
+            table.append(dict(b=b, d=d, GB=nbytes / 1e9, ms=sec * 1e3, GBps=nbytes / sec / 1e9,
+                              frac_of_peak=nbytes / sec / 1e9 / peak, frac_of_nominal_8TBps=nbytes / sec / 8e12,
+                              buffers=copies, b_next=int(b_next.item())))
+            del Gs
+            torch.cuda.empty_cache()
+    print(json.dumps(dict(sweep="stats fp32 M=1, abs_test_stats + 2 x abs_next_batch per step", steps=args.steps,
+                          warmup=args.warmup, peak_GBps=peak, peak_kind=peak_kind, cases=table)))
+    ctx.close()
+
+
 def run_ours(args):
     import torch
     import paper_2406_13936_b200 as pkg
@@ -489,10 +530,13 @@ def main():
     ap.add_argument("--case", default=None, choices=sorted(PROFILE_CASES),
                     help="run only a few launches of one kernel on a small case (for profiler captures)")
     ap.add_argument("--shape", default=None, help="M,b,d,f32|bf16: time abs_test_stats on that shape only")
+    ap.add_argument("--sweep", action="store_true", help="time the nine fp32 (b, d) cases of the statistics sweep")
     ap.add_argument("--tune", action="append", default=[], help="key=value passed to abs_set_tuning (with --case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
-    if args.case or args.shape:
+    if args.sweep:
+        run_sweep(args)
+    elif args.case or args.shape:
         run_profile_case(args)
     elif args.impl == "reference":
         run_reference(args)

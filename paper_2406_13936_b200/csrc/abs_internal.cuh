@@ -62,6 +62,34 @@ int set_error(abs_ctx* ctx, int code, const char* fmt, ...);
                              cudaGetErrorString(e__));                                   \
   } while (0)
 
+// ---- programmatic dependent launch ---------------------------------------------------------
+// The small kernels that follow a statistics kernel in the stream (finalisation, batch-size
+// update) are launched with the programmatic-serialisation attribute: their launch overlaps the
+// tail of the kernel before them, and they call pdl_wait() before they touch anything it wrote
+// (the wait returns when that kernel has completed and its writes are visible).  The kernels
+// before them call pdl_launch_dependents() once they are resident.  Both are no-ops in a kernel
+// launched the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                             Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- statistics kernels (abs_stats_tiled.cu, abs_stats_generic.cu) ---------------------
 // Layout of the partial-sum workspace written by both statistics kernels:
 //   ws[(m * P + p) * (b + 2) + r]      r < b : sum over the CTA's columns of (g_rj - gbar_j) gbar_j

@@ -26,6 +26,8 @@ abs_next_batch_kernel(const abs_stats* __restrict__ stats, int M, abs_test_cfg c
   __shared__ long long red[kThreads / 32];
   const int tid = threadIdx.x;
   long long T = 0;
+  pdl_wait();                    // the records (and b_cur) written by the kernels before
+  pdl_launch_dependents();
   if (tid < M) {
     const abs_stats s = stats[tid];
     const bool usable = (s.status & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) == 0u &&
@@ -76,8 +78,8 @@ extern "C" int abs_next_batch(abs_ctx* ctx, const abs_stats* stats, int M, const
   int prev = -1;
   ABS_CUDA_TRY(ctx, cudaGetDevice(&prev));
   if (prev != ctx->device) ABS_CUDA_TRY(ctx, cudaSetDevice(ctx->device));
-  abs_next_batch_kernel<<<1, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(stats, M, *cfg, b_cur, T_out, b_next);
-  const cudaError_t e = cudaGetLastError();
+  const cudaError_t e = launch_dependent(abs_next_batch_kernel, dim3(1), dim3(kThreads), 0,
+                                         static_cast<cudaStream_t>(stream), stats, M, *cfg, b_cur, T_out, b_next);
   if (prev != ctx->device) cudaSetDevice(prev);
   if (e != cudaSuccess) return set_error(ctx, ABS_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
   return ABS_OK;

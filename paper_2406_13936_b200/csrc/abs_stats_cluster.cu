@@ -128,6 +128,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
   }
   for (int i = tid; i < RC; i += kThreadsC) e_acc[i] = 0.0;
   cluster_sync_all();      // every CTA's barriers exist before anybody signals them
+  pdl_launch_dependents(); // the finalisation kernel may be scheduled; it waits for this grid to complete
   if (tid == 0)
     for (long long i = 0; i < S && i < n_mine; ++i) issue_load(i);
 

@@ -41,6 +41,7 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
   const T* Gm = G + static_cast<long long>(m) * worker_stride;
   double* out = ws + (static_cast<size_t>(m) * P + p) * (static_cast<size_t>(b) + 2);
   const float inv_b = 1.0f / static_cast<float>(b);
+  pdl_launch_dependents();      // the finalisation kernel may be scheduled; it waits for this grid to complete
 
   for (long long r = tid; r < b; r += kThreads) out[r] = 0.0;
   __syncthreads();
@@ -129,6 +130,8 @@ abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, uns
   const int m = blockIdx.x;
   const size_t rec = static_cast<size_t>(b) + 2;
   const double* base = ws + static_cast<size_t>(m) * P * rec;
+  pdl_wait();                    // the statistics kernel's partial records
+  pdl_launch_dependents();
 
   // Rows are spread over the threads; when b < 1024 several threads share a row and split the P
   // records between them (record p goes to thread group p mod tpr), then the groups' sums are
@@ -241,9 +244,8 @@ int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
 }
 
 int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P) {
-  abs_stats_finalize_kernel<<<a.M, kFinalThreads, 0, a.stream>>>(static_cast<const double*>(ctx->workspace), a.b, P,
-                                                               ctx->flags, a.stats_out);
-  ABS_CUDA_TRY(ctx, cudaGetLastError());
+  ABS_CUDA_TRY(ctx, launch_dependent(abs_stats_finalize_kernel, dim3(a.M), dim3(kFinalThreads), 0, a.stream,
+                                     static_cast<const double*>(ctx->workspace), a.b, P, ctx->flags, a.stats_out));
   return ABS_OK;
 }
 

@@ -88,6 +88,7 @@ abs_stats_gram_kernel(const __grid_constant__ CUtensorMap tmap, const GramParams
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
+  pdl_launch_dependents();      // the finalisation kernel may be scheduled; it waits for this grid to complete
 
   const long long n_mine = (prm.n_iters > p) ? (prm.n_iters - p + prm.P - 1) / prm.P : 0;
 

@@ -94,6 +94,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
   }
   for (int i = tid; i < prm.bx * b; i += kThreads) e_acc[i] = 0.0;
   __syncthreads();
+  pdl_launch_dependents();      // the finalisation kernel may be scheduled; it waits for this grid to complete
 
   // iterations of this CTA: it = p, p + P, ... < n_iters
   const long long n_mine = (prm.n_iters > p) ? (prm.n_iters - p + prm.P - 1) / prm.P : 0;

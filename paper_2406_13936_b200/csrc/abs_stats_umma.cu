@@ -222,6 +222,7 @@ abs_stats_umma_kernel(const UmmaParams prm) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_launch_dependents();      // the finalisation kernel may be scheduled; it waits for this grid to complete
 
   const long long n_mine = (prm.n_tiles > p) ? (prm.n_tiles - p + prm.P - 1) / prm.P : 0;
   const __nv_bfloat16* Gm = prm.G + static_cast<long long>(m) * prm.worker_stride;
