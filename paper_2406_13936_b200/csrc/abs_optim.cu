@@ -110,6 +110,7 @@ template <typename Rule, typename V>
 __global__ void __launch_bounds__(kThreads)
 local_step_kernel(const Rule rule, const StepArgs a) {
   const long long step = static_cast<long long>(gridDim.x) * kThreads;
+  pdl_wait();      // launched as a programmatic dependent: the gradient of the kernels before is complete now
   for (long long j = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; j < a.n; j += step) {
     V acc = zero4<V>();
     for (int m0 = 0; m0 < a.M; m0 += kChunk) {
@@ -165,7 +166,13 @@ int launch_step(abs_ctx* ctx, const Rule& rule, float* X, float* S0, float* S1, 
     a.n = nvec; a.offset = 0;
     long long blocks = (nvec + kThreads - 1) / kThreads;
     if (blocks > max_blocks) blocks = max_blocks;
-    local_step_kernel<Rule, float4><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(rule, a);
+    // small steps are bound by launch latency: let the launch overlap the kernel before (the kernel
+    // waits for it before it reads); large steps gain nothing from that and are launched the plain way
+    if (blocks < max_blocks)
+      ABS_CUDA_TRY(ctx, launch_dependent(local_step_kernel<Rule, float4>, dim3(static_cast<unsigned>(blocks)),
+                                         dim3(kThreads), 0, stream, rule, a));
+    else
+      local_step_kernel<Rule, float4><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(rule, a);
     ABS_CUDA_TRY(ctx, cudaGetLastError());
   }
   const long long tail = d - nvec * 4;
@@ -173,8 +180,8 @@ int launch_step(abs_ctx* ctx, const Rule& rule, float* X, float* S0, float* S1, 
     a.n = tail; a.offset = nvec * 4;
     long long blocks = (tail + kThreads - 1) / kThreads;
     if (blocks > max_blocks) blocks = max_blocks;
-    local_step_kernel<Rule, float><<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(rule, a);
-    ABS_CUDA_TRY(ctx, cudaGetLastError());
+    ABS_CUDA_TRY(ctx, launch_dependent(local_step_kernel<Rule, float>, dim3(static_cast<unsigned>(blocks)),
+                                       dim3(kThreads), 0, stream, rule, a));
   }
   return ABS_OK;
 }
