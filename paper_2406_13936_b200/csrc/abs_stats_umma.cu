@@ -5,8 +5,8 @@
 //   N = 1^T K 1 / b^2,  c_i = (K 1)_i / b,  sum_i ||g_i - gbar||^2 = tr K - 1^T K 1 / b.
 // The CUDA-core route needs about six instructions per bf16 element and stalls near 4 TB/s for
 // these batch sizes; a 128 x b x 16 tcgen05.mma takes the 4 KiB it consumes off the critical path.
-// Products of two bf16 values are exact in fp32; the tensor core adds them in fp32 over
-// fold_tiles * 256 columns in TMEM, then four warps read the accumulator back (tcgen05.ld),
+// Products of two bf16 values are exact in fp32; the tensor core adds them in fp32 over about
+// 4096 columns in TMEM (a fold), then four warps read the accumulator back (tcgen05.ld),
 // reduce each row to (K 1)_i and K_ii and add those to fp64 registers, which is where the
 // cancellation in c_i - N happens.  Two accumulators alternate, so the read-back overlaps the
 // next fold's MMAs.
