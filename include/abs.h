@@ -72,16 +72,18 @@ int abs_destroy(abs_ctx* ctx);
  * last failing abs_create on this thread. */
 const char* abs_last_error(const abs_ctx* ctx);
 
-/* Optional tuning of the tiled statistics kernel; 0 restores the automatic
+/* Optional tuning of the statistics kernels; 0 restores the automatic
  * choice.  key: "stats_stages" (2..8 tile buffers), "stats_ctas_per_worker",
  * "stats_force_generic" (1 = always use the alignment-free kernel),
- * "stats_flush_every" (tiles between fp64 flushes of the per-row sums),
+ * "stats_flush_every" (tiles between fp64 flushes of the per-row sums; for the
+ * tcgen05 kernel: tiles added up in its fp32 accumulators before the fold into
+ * fp64, at most 64),
  * "stats_stage_kb" (upper bound on one tile buffer, 4..200 KiB),
  * "stats_timeout_cycles" (SM clock cycles a wait for a tile copy may last before
  * the record is flagged ABS_STATUS_TIMEOUT; default about two seconds),
- * "stats_fault_drop_loads" (fault injection for tests: the loaders of the tiled and
- * of the tcgen05 kernel issue no copies, so every wait runs out and the records come back flagged
- * ABS_STATUS_TIMEOUT; nothing traps or hangs),
+ * "stats_fault_drop_loads" (fault injection for tests: the loaders of the tiled
+ * and of the tcgen05 kernel issue no copies, so every wait runs out and the
+ * records come back flagged ABS_STATUS_TIMEOUT; nothing traps or hangs),
  * "stats_cluster_rows" (target rows per CTA of the cluster kernel, 16..512),
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
  * cluster when b > 256),
