@@ -121,12 +121,14 @@ typedef struct {
  *                receives the batch gradients; may be NULL
  *   stats_out    [M] records
  * G is read exactly once from HBM when its base address and both strides are
- * multiples of 16 bytes and b <= 4096 (bf16 input with b <= 32 goes through a
- * tensor-core Gram-matrix kernel, b > 256 through a kernel that splits the rows
- * over a thread-block cluster, everything else through the tiled kernel);
- * otherwise an alignment-free kernel that reads it twice is used.  The result does not depend on which kernel ran beyond
- * floating-point rounding.  Accumulation: fp32 within a tile, fp64 across tiles;
- * the reduction order is fixed, so repeated calls give bit-identical records.
+ * multiples of 16 bytes and b <= 4096 (bf16 input with b <= 256 goes through
+ * tensor-core Gram-matrix kernels, other input with b > 256 through a kernel
+ * that splits the rows over a thread-block cluster, everything else through the
+ * tiled kernel); otherwise an alignment-free kernel that reads it twice is used.
+ * The result does not depend on which kernel ran beyond floating-point rounding.
+ * Accumulation: fp32 within a tile (the Gram kernels: exact bf16 products added
+ * in fp32 over at most 8192 columns), fp64 across tiles; the reduction order is
+ * fixed, so repeated calls give bit-identical records.
  * Errors: ABS_ERR_INVALID_ARG, ABS_ERR_WORKSPACE, ABS_ERR_CUDA.               */
 int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long long b, long long d,
                    long long row_stride, long long worker_stride,
