@@ -175,6 +175,8 @@ def test_tcgen05_gram_kernel_matches_oracle_and_tiled_kernel(ctx, M, b, d, pad, 
     G = make_G(170 + b, M, b, d, torch.bfloat16, sigma=2.0, pad=pad)
     assert (G.stride(1) * 2) % 16 == 0 and G.data_ptr() % 16 == 0
     tc, gbar_tc = run_gpu(ctx, G, want_gbar)
+    again, _ = run_gpu(ctx, G, want_gbar)
+    assert again == tc                                      # fixed order of additions: bit-identical records
     ctx.set_tuning("stats_no_gram", 1)
     try:
         tiled, gbar_t = run_gpu(ctx, G, want_gbar)
