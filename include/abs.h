@@ -138,7 +138,7 @@ int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long lon
  * statistics kernels, exposed for inspection and for tests that need no GPU.
  * aligned != 0 means base address and strides are multiples of 16 bytes.          */
 typedef struct {
-  int route;              /* 0 Gram (bf16, b <= 32), 1 cluster, 2 tiled, 3 generic two-sweep,
+  int route;              /* 0 Gram (bf16, 7 <= b <= 32), 1 cluster, 2 tiled, 3 generic two-sweep,
                              4 Gram on tcgen05 (bf16, 32 < b <= 256)                          */
   int lanes_per_row;      /* 16-byte vectors per tile row: a tile row has 16*lanes_per_row bytes */
   int warps_per_box;      /* consumer warps that share one box of rows                        */

@@ -56,6 +56,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+      : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -158,6 +166,29 @@ inline int encode_g_tensor_map(abs_ctx* ctx, const StatsLaunch& a, long long box
       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS)
     return set_error(ctx, ABS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r));
+  return ABS_OK;
+}
+
+// 4-D map over the same G for very small batches: a row is cut into segments of 256 elements
+// (the widest box a tensor map allows), and one box takes `segs` consecutive segments of each of
+// box_rows rows: [1][box_rows][segs][256].  In shared memory a box row is then segs * 256 elements
+// long, so one copy moves what several 3-D boxes would.  Needs d to be a multiple of 256.
+constexpr int kSegElems = 256;
+inline int encode_g_segment_map(abs_ctx* ctx, const StatsLaunch& a, int segs, int box_rows, CUtensorMap* tmap) {
+  const int es = a.dtype == ABS_F32 ? 4 : 2;
+  const cuuint64_t gdim[4] = {static_cast<cuuint64_t>(kSegElems), static_cast<cuuint64_t>(a.d / kSegElems),
+                              static_cast<cuuint64_t>(a.b), static_cast<cuuint64_t>(a.M)};
+  const cuuint64_t gstr[3] = {static_cast<cuuint64_t>(kSegElems) * es, static_cast<cuuint64_t>(a.row_stride) * es,
+                              static_cast<cuuint64_t>(a.M > 1 ? a.worker_stride : a.b * a.row_stride) * es};
+  const cuuint32_t box[4] = {static_cast<cuuint32_t>(kSegElems), static_cast<cuuint32_t>(segs),
+                             static_cast<cuuint32_t>(box_rows), 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUresult r = encode_tiled_fn()(
+      tmap, a.dtype == ABS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+      const_cast<void*>(a.G), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return set_error(ctx, ABS_ERR_CUDA, "cuTensorMapEncodeTiled (segments) failed with code %d", static_cast<int>(r));
   return ABS_OK;
 }
 

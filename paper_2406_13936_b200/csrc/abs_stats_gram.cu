@@ -22,6 +22,9 @@ namespace absk {
 namespace {
 
 constexpr int kWarpsC = 8;                    // consumer warps
+// A warp spends about 1300 clocks of MMA issue on a box of 256 columns however few rows it has, so
+// below 7 rows the tiled kernel (a few instructions per element) is faster: 6.2 against 3.5 TB/s at b = 4.
+constexpr int kMinRows = 7;
 constexpr int kThreadsG = kWarpsC * 32 + 32;
 // box width in columns: 512-byte rows for one 16-row block, 256-byte rows for two
 __host__ __device__ constexpr int box_cols_for(int nb) { return nb == 1 ? 256 : 128; }
@@ -37,6 +40,10 @@ struct GramParams {
   float* gbar_out;
   unsigned* flags;
   long long timeout_cycles;
+  // b < 8 and d a multiple of 256: one copy per stage through the segment map; a tile row then holds
+  // the 8 boxes side by side (row_pitch = 8 * 512 bytes, box q starts q * 512 bytes into the row)
+  int segment_map;
+  unsigned row_pitch, box_stride;
 };
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
@@ -79,7 +86,13 @@ abs_stats_gram_kernel(const __grid_constant__ CUtensorMap tmap, const GramParams
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // Rows b..BP-1 of every box are never written by the loads (the box has b rows): zero them once.
-  if (b < BP) {
+  if (b < BP && prm.segment_map) {
+    const int pad_words = (BP - b) * static_cast<int>(prm.row_pitch / 4);        // rows b.. of every stage
+    for (int st = 0; st < S; ++st) {
+      unsigned* dst = reinterpret_cast<unsigned*>(stage_mem + static_cast<size_t>(st) * prm.stage_bytes + b * prm.row_pitch);
+      for (int i = tid; i < pad_words; i += kThreadsG) dst[i] = 0u;
+    }
+  } else if (b < BP) {
     const int pad_words = (BP - b) * (kRowBytes / 4);
     for (int box = 0; box < S * kWarpsC; ++box) {
       unsigned* dst = reinterpret_cast<unsigned*>(stage_mem + static_cast<size_t>(box) * prm.box_bytes + b * kRowBytes);
@@ -102,18 +115,26 @@ abs_stats_gram_kernel(const __grid_constant__ CUtensorMap tmap, const GramParams
 
   if (warp == kWarpsC) {
     if (lane == 0) {
-      for (long long i = 0; i < n_mine; ++i) {
-        const int s = static_cast<int>(i % S);
-        const long long use = i / S;
-        if (use > 0)
-          mbar_wait(empty_u32 + 8u * s, static_cast<uint32_t>((use - 1) & 1), abort_flag, prm.timeout_cycles);
+      // s = i % S and the pass number i / S are carried along instead of divided out per tile
+      int s = 0;
+      uint32_t pass = 0;
+      long long x0 = static_cast<long long>(p) * kWarpsC * kBoxCols;
+      const long long x_step = static_cast<long long>(prm.P) * kWarpsC * kBoxCols;
+      for (long long i = 0; i < n_mine; ++i, x0 += x_step) {
+        if (pass > 0) mbar_wait(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles);
         const uint32_t full = full_u32 + 8u * s;
         mbar_expect_tx(full, static_cast<uint32_t>(kWarpsC) * static_cast<uint32_t>(b) * kRowBytes);
-        const long long it = p + i * prm.P;
-        for (int q = 0; q < kWarpsC; ++q) {
-          const long long x = (it * kWarpsC + q) * kBoxCols;
-          tma_load_3d(stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(q) * prm.box_bytes,
-                      &tmap, static_cast<int>(x), 0, m, full);
+        if (prm.segment_map) {        // a copy costs about 100 clocks plus 8 per row: one for the whole stage
+          tma_load_4d(stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes, &tmap, 0, static_cast<int>(x0 / kSegElems), 0, m,
+                      full);
+        } else {
+          for (int q = 0; q < kWarpsC; ++q)
+            tma_load_3d(stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(q) * prm.box_bytes,
+                        &tmap, static_cast<int>(x0 + q * kBoxCols), 0, m, full);
+        }
+        if (++s == S) {
+          s = 0;
+          ++pass;
         }
       }
       for (int s = 0; s < S && s < n_mine; ++s) {    // leave no copy in flight
@@ -124,13 +145,17 @@ abs_stats_gram_kernel(const __grid_constant__ CUtensorMap tmap, const GramParams
     }
   } else {
     const int r = lane >> 2, t = lane & 3;
-    const uint32_t lane_off = static_cast<uint32_t>(r) * kRowBytes + static_cast<uint32_t>(t) * 16u;
+    const uint32_t pitch = prm.row_pitch;
+    const uint32_t lane_off = static_cast<uint32_t>(r) * pitch + static_cast<uint32_t>(t) * 16u;
     const float inv_b = 1.0f / static_cast<float>(b);
+    int s = -1;
+    uint32_t parity = 1u;
     for (long long i = 0; i < n_mine; ++i) {
-      const int s = static_cast<int>(i % S);
-      mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>((i / S) & 1), abort_flag, prm.timeout_cycles);
+      if (++s == S) s = 0;                        // s = i % S, parity = (i / S) & 1 without dividing
+      if (s == 0) parity ^= 1u;
+      mbar_wait(full_u32 + 8u * s, parity, abort_flag, prm.timeout_cycles);
       const uint32_t base = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes +
-                            static_cast<uint32_t>(warp) * prm.box_bytes;
+                            static_cast<uint32_t>(warp) * prm.box_stride;
       float acc[NPAIR][2][4];
 #pragma unroll
       for (int q = 0; q < NPAIR; ++q)
@@ -144,8 +169,8 @@ abs_stats_gram_kernel(const __grid_constant__ CUtensorMap tmap, const GramParams
         uint4 lo[NB], hi[NB];
 #pragma unroll
         for (int I = 0; I < NB; ++I) {
-          lo[I] = lds128(base + lane_off + static_cast<uint32_t>(I * 16) * kRowBytes + ch * 64);
-          hi[I] = lds128(base + lane_off + static_cast<uint32_t>(I * 16 + 8) * kRowBytes + ch * 64);
+          lo[I] = lds128(base + lane_off + static_cast<uint32_t>(I * 16) * pitch + ch * 64);
+          hi[I] = lds128(base + lane_off + static_cast<uint32_t>(I * 16 + 8) * pitch + ch * 64);
         }
 #pragma unroll
         for (int I = 0; I < NB; ++I) {
@@ -169,7 +194,7 @@ abs_stats_gram_kernel(const __grid_constant__ CUtensorMap tmap, const GramParams
 #pragma unroll
         for (int j = 0; j < 8; ++j) cs[j] = 0.f;
         for (int row = 0; row < b; ++row) {
-          const uint4 u = lds128(base + static_cast<uint32_t>(row) * kRowBytes + lane * 16);
+          const uint4 u = lds128(base + static_cast<uint32_t>(row) * pitch + lane * 16);
           cs[0] += __uint_as_float(u.x << 16);
           cs[1] += __uint_as_float(u.x & 0xffff0000u);
           cs[2] += __uint_as_float(u.y << 16);
@@ -280,7 +305,7 @@ int launch_gram_variant(abs_ctx* ctx, const CUtensorMap& tmap, const GramParams&
 }  // namespace
 
 int plan_stats_gram(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out) {
-  if (dtype != ABS_BF16 || b < 2 || b > 32) return ABS_ERR_UNSUPPORTED;
+  if (dtype != ABS_BF16 || b < kMinRows || b > 32) return ABS_ERR_UNSUPPORTED;
   const int NB = b <= 16 ? 1 : 2;
   const unsigned box_bytes = static_cast<unsigned>(16 * NB) * static_cast<unsigned>(box_cols_for(NB)) * 2u;
   int stages = static_cast<int>(t.stats_stages > 0 ? t.stats_stages : 3);
@@ -302,7 +327,7 @@ int plan_stats_gram(const Tuning& t, size_t smem_optin, abs_dtype dtype, long lo
 }
 
 int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
-  if (a.dtype != ABS_BF16 || a.b > 32 || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
+  if (a.dtype != ABS_BF16 || a.b < kMinRows || a.b > 32 || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
   const int NB = a.b <= 16 ? 1 : 2;
   const int BP = 16 * NB;
   const int kBoxCols = box_cols_for(NB);
@@ -331,8 +356,12 @@ int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if (need > ctx->workspace_bytes)
     return set_error(ctx, ABS_ERR_WORKSPACE, "abs_test_stats needs %zu workspace bytes, context has %zu", need,
                      ctx->workspace_bytes);
+  // fewer than 8 rows: the copy engine's cost per copy (about 100 clocks) shows; the segment map
+  // brings a whole stage in one copy, if the rows can be cut into segments of 256 elements
+  const bool segment_map = NB == 1 && a.b < 8 && a.d % kSegElems == 0 && kBoxCols == kSegElems;
   CUtensorMap tmap;
-  int rc = encode_g_tensor_map(ctx, a, kBoxCols, static_cast<int>(a.b), &tmap);
+  int rc = segment_map ? encode_g_segment_map(ctx, a, kWarpsC, static_cast<int>(a.b), &tmap)
+                       : encode_g_tensor_map(ctx, a, kBoxCols, static_cast<int>(a.b), &tmap);
   if (rc != ABS_OK) return rc;
 
   GramParams prm;
@@ -347,6 +376,9 @@ int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
+  prm.segment_map = segment_map ? 1 : 0;
+  prm.row_pitch = segment_map ? kWarpsC * kRowBytes : kRowBytes;
+  prm.box_stride = segment_map ? kRowBytes : box_bytes;
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
   const size_t smem = smem_for(stages);
   const bool gb = a.gbar_out != nullptr;

@@ -47,6 +47,8 @@ struct TiledParams {
   unsigned* flags;
   long long timeout_cycles;
   int drop_loads;        // fault injection for the bounded waits: the loader issues nothing
+  int boxes_per_copy;    // neighbouring boxes that one copy brings in as one tile row: 1; 2, 4 or 8 for very small batches
+  int segment_map;       // the tensor map is the 4-D segment map (x counted in segments of 256 elements)
 };
 
 // ---- the kernel ----------------------------------------------------------------------------
@@ -105,22 +107,39 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
     // ------------------------------ producer ------------------------------
     if (lane == 0) {
       const int box_cols = lpr * VE;
-      for (long long i = 0; i < n_mine; ++i) {
-        const int s = static_cast<int>(i % S);
-        const long long use = i / S;
-        if (use > 0)
-          mbar_wait(empty_u32 + 8u * s, static_cast<uint32_t>((use - 1) & 1), abort_flag, prm.timeout_cycles);
+      // s = i % S and the pass number i / S are carried along: a 64-bit division per tile is most
+      // of the work when a tile is a few KiB (very small batches)
+      int s = 0;
+      uint32_t pass = 0;
+      long long x0 = static_cast<long long>(p) * prm.bx * box_cols;           // first column of the stage
+      const long long x_step = static_cast<long long>(prm.P) * prm.bx * box_cols;
+      for (long long i = 0; i < n_mine; ++i, x0 += x_step) {
+        const int s_now = s;
+        const uint32_t pass_now = pass;
+        if (++s == S) {
+          s = 0;
+          ++pass;
+        }
+        if (pass_now > 0)
+          mbar_wait(empty_u32 + 8u * s_now, (pass_now - 1) & 1u, abort_flag, prm.timeout_cycles);
         if (prm.drop_loads) continue;     // test hook: the consumers' waits must run out, not hang
-        const uint32_t full = full_u32 + 8u * s;
+        const uint32_t full = full_u32 + 8u * s_now;
         mbar_expect_tx(full, prm.stage_bytes);
-        const long long it = p + i * prm.P;
-        for (int q = 0; q < prm.bx; ++q) {
-          const long long x = (it * prm.bx + q) * box_cols;
+        // a copy costs the copy engine about 100 clocks plus 8 per row, so boxes of a few rows are
+        // brought in several at a time: one copy whose rows are boxes_per_copy boxes long, which
+        // as many consumer warps share side by side
+        const int q_step = prm.boxes_per_copy;
+        for (int q = 0; q < prm.bx; q += q_step) {
+          const long long x = x0 + static_cast<long long>(q) * box_cols;
           const uint32_t dst0 =
-              stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + static_cast<uint32_t>(q) * prm.box_bytes;
-          for (int rb = 0; rb < prm.n_row_boxes; ++rb)
-            tma_load_3d(dst0 + static_cast<uint32_t>(rb * prm.box_rows) * row_bytes, &tmap, static_cast<int>(x),
-                        rb * prm.box_rows, m, full);
+              stage_u32 + static_cast<uint32_t>(s_now) * prm.stage_bytes + static_cast<uint32_t>(q) * prm.box_bytes;
+          if (prm.segment_map) {
+            tma_load_4d(dst0, &tmap, 0, static_cast<int>(x / kSegElems), 0, m, full);
+          } else {
+            for (int rb = 0; rb < prm.n_row_boxes; ++rb)
+              tma_load_3d(dst0 + static_cast<uint32_t>(rb * prm.box_rows) * row_bytes * q_step, &tmap, static_cast<int>(x),
+                          rb * prm.box_rows, m, full);
+          }
         }
       }
       // Leave no copy in flight: every armed phase of every buffer must have completed
@@ -144,9 +163,13 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
     // In the register-resident variants RMAX is exactly ceil(b / RG): every thread owns rows
     // 0..RMAX-2 of its group and only the last one can fall past the batch.
     const bool last_ok = n_rows_mine >= RMAX;
-    const unsigned row_step = static_cast<unsigned>(RG) * row_bytes;
-    const uint32_t my_off = static_cast<uint32_t>(q) * prm.box_bytes + static_cast<uint32_t>(rg) * row_bytes +
-                            static_cast<uint32_t>(cv) * 16u;
+    // boxes_per_copy > 1: box q is one of the boxes that lie side by side in a longer tile row
+    const int bpc = prm.boxes_per_copy;
+    const unsigned row_pitch = static_cast<unsigned>(bpc) * row_bytes;
+    const uint32_t box_off = static_cast<uint32_t>(q / bpc) * static_cast<uint32_t>(bpc) * prm.box_bytes +
+                             static_cast<uint32_t>(q % bpc) * row_bytes;
+    const unsigned row_step = static_cast<unsigned>(RG) * row_pitch;
+    const uint32_t my_off = box_off + static_cast<uint32_t>(rg) * row_pitch + static_cast<uint32_t>(cv) * 16u;
     const float inv_b = 1.0f / static_cast<float>(b);
     const bool first_rg = (rg == 0);
     double* e_mine = e_acc + static_cast<size_t>(q) * b;
@@ -156,13 +179,15 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
     for (int k = 0; k < RMAX; ++k) e[k] = 0.f;
     int since_flush = 0;
 
+    int s = -1;
+    uint32_t parity = 1u;
     for (long long i = 0; i < n_mine; ++i) {
-      const int s = static_cast<int>(i % S);
-      const uint32_t parity = static_cast<uint32_t>((i / S) & 1);
+      if (++s == S) s = 0;                        // s = i % S, parity = (i / S) & 1 without dividing
+      if (s == 0) parity ^= 1u;
       mbar_wait(full_u32 + 8u * s, parity, abort_flag, prm.timeout_cycles);
       const uint32_t base = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + my_off;
-      const uint32_t base0 = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes +
-                             static_cast<uint32_t>(q) * prm.box_bytes + static_cast<uint32_t>(cv) * 16u;   // row 0
+      const uint32_t base0 = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes + box_off +
+                             static_cast<uint32_t>(cv) * 16u;   // row 0
 
       // sweep 1: column sums over this thread's rows
       uint4 v[KEEP ? RMAX : 1];
@@ -304,7 +329,7 @@ abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledPara
 // ---- host side -----------------------------------------------------------------------------
 struct TileChoice {
   int lpr_log2, rs_log2, bx, stages, box_rows, n_row_boxes, rmax;
-  bool keep, full;
+  bool keep, full, small_rows;
   unsigned box_bytes, stage_bytes;
   size_t smem_bytes;
 };
@@ -355,6 +380,8 @@ bool choose_tile(long long b, int ve, size_t smem_optin, long long want_stages, 
       c->keep = (pass == 0);
       c->rmax = pass == 0 ? static_cast<int>(R) : 32;
       c->full = (b % RG == 0) && (pass == 0 ? (R == 2 || R == 4 || R == 8 || R == 16) : R == 32);
+      // boxes of fewer than 8 rows, one per consumer warp: candidates for sharing a copy
+      c->small_rows = (b < 8 && lpr == 32 && rs_log2 == 0 && n_row_boxes == 1);
       c->box_bytes = static_cast<unsigned>(rows_pad * lpr * 16);
       c->stage_bytes = static_cast<unsigned>(stage);
       c->smem_bytes = stages * stage + extras_bytes(lpr, ve, bx, b, stages) + 128;
@@ -462,8 +489,19 @@ int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
                      ctx->workspace_bytes);
 
   CUtensorMap tmap;
+  int boxes_per_copy = 1, segment_map = 0;
   {
-    const int rc = encode_g_tensor_map(ctx, a, box_cols, c.box_rows, &tmap);
+    // Very small batches: all boxes of a stage in one copy through the segment map when d allows it,
+    // else (4-byte elements) two boxes per copy, the widest a plain box can be.
+    if (c.small_rows && a.d % kSegElems == 0) {
+      boxes_per_copy = c.bx;
+      segment_map = 1;
+    } else if (c.small_rows && ve == 4) {
+      boxes_per_copy = 2;
+    }
+    const int rc = segment_map
+                       ? encode_g_segment_map(ctx, a, static_cast<int>(boxes_per_copy * box_cols / kSegElems), c.box_rows, &tmap)
+                       : encode_g_tensor_map(ctx, a, boxes_per_copy * box_cols, c.box_rows, &tmap);
     if (rc != ABS_OK) return rc;
   }
 
@@ -485,6 +523,8 @@ int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.drop_loads = ctx->tuning.stats_fault_drop_loads ? 1 : 0;
+  prm.boxes_per_copy = boxes_per_copy;
+  prm.segment_map = segment_map;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
 
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));

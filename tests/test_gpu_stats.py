@@ -74,6 +74,8 @@ SHAPES = [
     (1, 33, 3000), (2, 64, 2500), (1, 100, 1531), (1, 128, 5000), (1, 129, 777), (1, 256, 4099),
     (1, 257, 1200), (1, 300, 900), (1, 512, 1100), (1, 1000, 515), (1, 1024, 700), (1, 2048, 300),
     (1, 4096, 130), (8, 16, 20000), (1, 64, 70001),
+    # fewer than 8 rows: several boxes per copy (segment map when d is a multiple of 256, else pairs)
+    (1, 2, 256), (2, 3, 1024), (1, 4, 70144), (3, 7, 2560), (1, 5, 256000), (1, 4, 1000), (2, 6, 4104), (8, 2, 51200),
 ]
 
 

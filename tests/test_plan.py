@@ -22,7 +22,7 @@ def check_plan(dtype, b, p):
     if p["boxes_per_stage"] > 1:
         assert (p["stage_bytes"] // p["boxes_per_stage"]) % 128 == 0
     if p["route"] == 0:
-        assert dtype == "bf16" and b <= 32 and p["box_rows"] == b
+        assert dtype == "bf16" and 7 <= b <= 32 and p["box_rows"] == b
         return
     if p["route"] == 4:
         # tcgen05 Gram kernel: k-blocks of 128-byte rows, each k-block on a 1024-byte boundary.
@@ -67,9 +67,9 @@ def check_plan(dtype, b, p):
 def test_every_batch_size_gets_a_valid_plan(dtype):
     for b in range(2, 4097):
         p = pkg.plan_stats(dtype, b)
-        if dtype == "bf16" and b <= 32:
+        if dtype == "bf16" and 7 <= b <= 32:
             assert p["route"] == 0
-        elif dtype == "bf16" and b <= 256:
+        elif dtype == "bf16" and 32 < b <= 256:
             assert p["route"] == 4
         elif b > 256:
             assert p["route"] == 1
