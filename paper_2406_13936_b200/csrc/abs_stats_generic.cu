@@ -27,7 +27,11 @@ __device__ __forceinline__ double warp_sum_d(double v) {
   return v;
 }
 
-template <typename T>
+// E_SMEM: the per-row sums e_r live in (dynamic) shared memory until the end, which is possible up
+// to kGenericSmemRows rows; beyond, they are updated in the CTA's workspace record strip by strip.
+constexpr int kGenericSmemRows = 4096;
+
+template <typename T, bool E_SMEM>
 __global__ void __launch_bounds__(kThreads)
 abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long long row_stride,
                          long long worker_stride, long long n_strips, int P, double* __restrict__ ws,
@@ -35,15 +39,17 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
   __shared__ float colpart[kWarps][kStrip];
   __shared__ float gbar_s[kStrip];
   __shared__ double red[2 * kWarps];
+  extern __shared__ double e_rows[];            // [b] when E_SMEM
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m = blockIdx.y, p = blockIdx.x;
   const T* Gm = G + static_cast<long long>(m) * worker_stride;
   double* out = ws + (static_cast<size_t>(m) * P + p) * (static_cast<size_t>(b) + 2);
+  double* e_acc = E_SMEM ? e_rows : out;        // one warp owns a row: a single writer either way
   const float inv_b = 1.0f / static_cast<float>(b);
   pdl_launch_dependents();      // the finalisation kernel may be scheduled; it waits for this grid to complete
 
-  for (long long r = tid; r < b; r += kThreads) out[r] = 0.0;
+  for (long long r = tid; r < b; r += kThreads) e_acc[r] = 0.0;
   __syncthreads();
 
   double vacc = 0.0, nacc = 0.0;
@@ -95,7 +101,7 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
       }
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) el += __shfl_xor_sync(0xffffffffu, el, off);
-      if (lane == 0) out[r] += static_cast<double>(el);
+      if (lane == 0) e_acc[r] += static_cast<double>(el);
     }
     vacc += static_cast<double>(vl);
     __syncthreads();
@@ -108,6 +114,8 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
     red[kWarps + warp] = nacc;
   }
   __syncthreads();
+  if (E_SMEM)
+    for (long long r = tid; r < b; r += kThreads) out[r] = e_rows[r];
   if (tid == 0) {
     double vs = 0.0, ns = 0.0;
     for (int w = 0; w < kWarps; ++w) {
@@ -230,14 +238,18 @@ int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
                      static_cast<size_t>(a.M) * P * rec, ctx->workspace_bytes);
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));
   double* ws = static_cast<double*>(ctx->workspace);
-  if (a.dtype == ABS_F32)
-    abs_stats_generic_kernel<float><<<grid, kThreads, 0, a.stream>>>(
-        static_cast<const float*>(a.G), a.b, a.d, a.row_stride, a.worker_stride, n_strips, static_cast<int>(P), ws,
-        a.gbar_out);
-  else
-    abs_stats_generic_kernel<__nv_bfloat16><<<grid, kThreads, 0, a.stream>>>(
-        static_cast<const __nv_bfloat16*>(a.G), a.b, a.d, a.row_stride, a.worker_stride, n_strips,
-        static_cast<int>(P), ws, a.gbar_out);
+  const bool e_smem = a.b <= kGenericSmemRows;
+  const size_t smem = e_smem ? static_cast<size_t>(a.b) * sizeof(double) : 0;
+#define ABS_GENERIC_LAUNCH(T, E)                                                                                 \
+  abs_stats_generic_kernel<T, E><<<grid, kThreads, smem, a.stream>>>(static_cast<const T*>(a.G), a.b, a.d,       \
+                                                                     a.row_stride, a.worker_stride, n_strips,    \
+                                                                     static_cast<int>(P), ws, a.gbar_out)
+  if (a.dtype == ABS_F32) {
+    if (e_smem) ABS_GENERIC_LAUNCH(float, true); else ABS_GENERIC_LAUNCH(float, false);
+  } else {
+    if (e_smem) ABS_GENERIC_LAUNCH(__nv_bfloat16, true); else ABS_GENERIC_LAUNCH(__nv_bfloat16, false);
+  }
+#undef ABS_GENERIC_LAUNCH
   ABS_CUDA_TRY(ctx, cudaGetLastError());
   *P_out = static_cast<int>(P);
   return ABS_OK;
