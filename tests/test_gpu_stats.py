@@ -434,6 +434,48 @@ def test_worker_gradient_estimator(ctx, M, b_local, d):
         assert b_local * rec["var_norm"] == pytest.approx(4.0 * d, rel=0.1)
 
 
+# ------------------------------------------------------------------ stream capture
+@pytest.mark.parametrize("dtype,b", [(torch.float32, 256), (torch.float32, 1024), (torch.bfloat16, 16),
+                                     (torch.bfloat16, 128)])
+def test_a_step_can_be_captured_in_a_cuda_graph(ctx, dtype, b):
+    """The calls only enqueue work (no allocation, no synchronisation), so a statistics + batch-size
+    + optimiser step can be captured once and replayed: the replays give the eager results bit for bit."""
+    M, d = 2, 20480
+    G = make_G(55, M, b, d, dtype)
+    cfg = pkg.make_test_cfg("aug_ip", 1 << 20, theta=0.5, nu=0.5)
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+
+    def fresh():
+        X = torch.linspace(-1.0, 1.0, M * d, device="cuda").reshape(M, d).contiguous()
+        return dict(X=X, m1=torch.zeros_like(X), m2=torch.zeros_like(X), gbar=torch.zeros((M, d), device="cuda"),
+                    stats=ctx.new_stats(M), b_cur=torch.tensor([b], dtype=torch.int64, device="cuda"),
+                    b_next=torch.zeros(1, dtype=torch.int64, device="cuda"))
+
+    def step(st, t):
+        ctx.abs_test_stats(G, st["stats"], st["gbar"])
+        ctx.abs_next_batch(st["stats"], cfg, st["b_cur"], st["b_next"])
+        ctx.local_adamw_step(st["X"], st["m1"], st["m2"], st["gbar"], pkg.make_adamw_cfg(step=t, **hp), average_after=1)
+
+    eager = fresh()
+    step(eager, 1)
+    torch.cuda.synchronize()
+    cap = fresh()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(cap, 1)                                   # warm-up outside the capture (function attributes)
+        torch.cuda.synchronize()
+        replay = fresh()
+        with torch.cuda.graph(graph, stream=side):
+            step(replay, 1)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert pkg.stats_to_dicts(replay["stats"]) == pkg.stats_to_dicts(eager["stats"])
+    assert int(replay["b_next"].item()) == int(eager["b_next"].item())
+    assert torch.equal(replay["X"], eager["X"]) and torch.equal(replay["m2"], eager["m2"])
+
+
 # ------------------------------------------------------------------ bounded waits
 @pytest.mark.parametrize("dtype,b", [(torch.float32, 40), (torch.bfloat16, 72), (torch.bfloat16, 200)])
 def test_wait_that_runs_out_is_reported_and_the_context_stays_usable(ctx, dtype, b):
