@@ -261,6 +261,7 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
         del G
         torch.cuda.empty_cache()
     out["rounds_logreg"] = end_to_end_rounds(torch, pkg, inputs, ctx, "logreg")
+    out["rounds_logreg_fused"] = logreg_rounds_fused(torch, pkg, inputs, ctx)
     out["rounds_mlp"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp")
     out["rounds_mlp_fused_stats"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp_fused")
     return out
@@ -305,6 +306,41 @@ def end_to_end_rounds(torch, pkg, inputs, ctx, which):
     sec = time.perf_counter() - t0
     return dict(rounds=rounds, rounds_per_s=rounds / sec, seconds=sec, M=M, H=H, b_first=history[0],
                 b_last=history[-1], rounds_until_cap=next((i for i, v in enumerate(history) if v >= b_max), None))
+
+
+def logreg_rounds_fused(torch, pkg, inputs, ctx):
+    """The logistic configuration with all 50 rounds in one cooperative launch (abs_logreg_rounds_fused:
+    parameters in shared memory, batch size on the device, no per-sample gradient matrix), and with one
+    launch per round; CUDA-event time of the launches, after one untimed run."""
+    n, d, M, H, lr, b0, b_max, rounds = 65536, 256, 4, 8, 0.1, 16, 1024, 50
+    A, y = inputs.logreg_dataset(1, n, d, device="cuda")
+    cfg = pkg.make_test_cfg("norm", b_max, eta=0.5)
+    idx = inputs.batch_indices(11, (rounds, H, M, b_max), n, device="cuda")
+    stats = ctx.new_stats(rounds * M)
+    hist = torch.zeros(rounds + 1, dtype=torch.int64, device="cuda")
+    out = dict(rounds=rounds, M=M, H=H)
+    for mode in ("one_launch", "launch_per_round"):
+        best = None
+        for rep in range(4):
+            X = torch.zeros((M, d), device="cuda")
+            b_dev = torch.tensor([b0], dtype=torch.int64, device="cuda")
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            if mode == "one_launch":
+                ctx.abs_logreg_rounds_fused(A, y, idx, X, H, lr, cfg, stats, b_dev, b_hist=hist)
+            else:
+                for k in range(rounds):
+                    ctx.abs_logreg_rounds_fused(A, y, idx[k:k + 1], X, H, lr, cfg, stats[k * M:(k + 1) * M], b_dev)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            if rep > 0:
+                best = ms if best is None else min(best, ms)
+        out[mode] = dict(rounds_per_s=rounds / (best * 1e-3), us_per_round=best * 1e3 / rounds)
+    h = hist.tolist()
+    out.update(b_first=h[0], b_last=h[-1], rounds_until_cap=next((i for i, v in enumerate(h) if v >= b_max), None))
+    return out
 
 
 PROFILE_CASES = {

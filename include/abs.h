@@ -322,6 +322,26 @@ int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, long long n, 
                      float lr, const abs_test_cfg* cfg, float* G_scratch, float* Gb_scratch,
                      abs_stats* stats, long long* T_out, long long* b_dev, void* stream);
 
+/* `rounds` communication rounds of the same method in ONE cooperative launch
+ * (Algorithm 2's structure, Algorithm 1's per-sample statistic once per round,
+ * Section 4.3; b <- min(b_max, max{b, max_m T_m})): the parameters stay in shared
+ * memory, the batch size stays on the device from round to round, the per-sample
+ * gradient matrix is never written, and there is one grid-wide barrier per local
+ * step.  For small problems, where abs_logreg_round is bound by launch latency.
+ *   idx [rounds][H][M][idx_stride] int32 with idx_stride >= cfg->b_max (indices
+ *   outside [0, n) are clamped);  X [M][d] in place (replica stride d);
+ *   stats [rounds][M] records of each round's test;  T_out [rounds][M] or NULL;
+ *   b_hist [rounds + 1] or NULL: the batch size each round ran with, then the last
+ *   update;  b_dev: the starting size on entry (raised to 2, capped at b_max), the
+ *   size after the last round on exit.
+ * Needs d <= 1024, d % 4 == 0, M <= 64 and 16-byte aligned A and X, else
+ * ABS_ERR_UNSUPPORTED; scratch comes from the context's workspace
+ * (ABS_ERR_WORKSPACE if it is too small).  Only enqueues.                          */
+int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
+                            const int* idx, long long idx_stride, int rounds, float* X, int M, int H,
+                            float lr, const abs_test_cfg* cfg, abs_stats* stats, long long* T_out,
+                            long long* b_hist, long long* b_dev, void* stream);
+
 /* Three-layer ReLU MLP with softmax cross-entropy (the second synthetic problem).
  * dims = {n0, n1, n2, n3} layer widths.  One replica's parameters are a flat fp32
  * vector W1 [n1][n0], b1 [n1], W2 [n2][n1], b2 [n2], W3 [n3][n2], b3 [n3] (each W

@@ -71,6 +71,10 @@ EXPORTS = {
                          ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                          ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p, ctypes.c_void_p,
                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_logreg_rounds_fused": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
+                                ctypes.c_longlong, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_void_p,
+                                ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p,
+                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "abs_mlp_param_count": [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_longlong)],
     "abs_mlp_scratch_bytes": [ctypes.c_int, ctypes.c_longlong, ctypes.POINTER(ctypes.c_int),
                               ctypes.POINTER(ctypes.c_size_t)],
@@ -285,6 +289,24 @@ class Context:
                                                int(H), int(b), float(lr), ctypes.byref(cfg), _ptr(G_scratch),
                                                _ptr(Gb_scratch), _ptr(stats), _ptr(T_out), _ptr(b_dev),
                                                _stream(stream)), "abs_logreg_round")
+
+    def abs_logreg_rounds_fused(self, A, y, idx, X, H, lr, cfg, stats, b_dev, T_out=None, b_hist=None, stream=None):
+        """idx [rounds, H, M, >= cfg.b_max] int32 (contiguous but for the last stride); stats [rounds*M, 7] from
+        new_stats(rounds * M); T_out [rounds, M] and b_hist [rounds + 1] int64 or None; b_dev int64 device tensor."""
+        n, d = A.shape
+        M = X.shape[0]
+        rounds = idx.shape[0]
+        if idx.dim() != 4 or idx.shape[1] != H or idx.shape[2] != M or idx.stride(3) != 1 or \
+                idx.stride(1) != M * idx.stride(2) or idx.stride(0) != H * idx.stride(1):
+            raise ValueError("idx must be [rounds, H, M, stride] with the first three dimensions packed")
+        if stats.shape[0] < rounds * M:
+            raise ValueError("stats needs rounds * M records")
+        if not (A.is_contiguous() and X.is_contiguous()):
+            raise ValueError("A and X must be contiguous")
+        self._check(self._lib.abs_logreg_rounds_fused(self._h, _ptr(A), _ptr(y), n, d, _ptr(idx), idx.stride(2),
+                                                      int(rounds), _ptr(X), M, int(H), float(lr), ctypes.byref(cfg),
+                                                      _ptr(stats), _ptr(T_out), _ptr(b_hist), _ptr(b_dev),
+                                                      _stream(stream)), "abs_logreg_rounds_fused")
 
     def mlp_param_count(self, dims):
         out = ctypes.c_longlong()

@@ -90,6 +90,64 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
 }
 #endif
 
+// ---- decisions shared by the kernels that turn sums into records and records into sizes -----
+#ifdef __CUDACC__
+__device__ __forceinline__ double safe_ratio(double num, double den) {
+  if (num == 0.0) return 0.0;            // 0/x and 0/0 count as 0
+  if (den == 0.0) return INFINITY;       // x/0 counts as +infinity
+  return num / den;
+}
+__device__ __forceinline__ long long ceil_saturating(double x) {
+  if (!(x < 4611686018427387904.0)) return 1ll << 62;   // also catches NaN
+  return static_cast<long long>(ceil(x));
+}
+
+// T of one worker (Eq. norm_test, Eq. test_stat; the augmented inner-product test takes the
+// larger of its two ceilings).  All arithmetic that decides the integer is fp64, in the order
+// scale * (variance / (constant^2 * N [* N])).  A record that cannot be used gives 0.
+__device__ __forceinline__ long long test_size_from_record(const abs_stats& s, const abs_test_cfg& cfg) {
+  const bool usable = (s.status & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) == 0u &&
+                      (cfg.kind == ABS_TEST_NORM || (s.status & ABS_STATUS_NORM_ONLY) == 0u);
+  if (!usable) return 0;
+  const double scale = cfg.row_weight / cfg.divisor;
+  const double N = s.gbar_sq;
+  if (cfg.kind == ABS_TEST_NORM) return ceil_saturating(scale * safe_ratio(s.var_norm, cfg.eta * cfg.eta * N));
+  const long long t_ip = ceil_saturating(scale * safe_ratio(s.var_ip, cfg.theta * cfg.theta * N * N));
+  const long long t_orth = ceil_saturating(scale * safe_ratio(s.var_orth, cfg.nu * cfg.nu * N));
+  return t_ip > t_orth ? t_ip : t_orth;
+}
+
+// The record of one worker from its four sums (Eq. def_var): V = sum_i ||g_i - gbar||^2,
+// N = ||gbar||^2, s_e = sum_i e_i and s_ee = sum_i e_i^2 with e_i = <g_i - gbar, gbar>.
+__device__ __forceinline__ abs_stats record_from_sums(double V, double N, double s_e, double s_ee, long long b,
+                                                      bool timed_out) {
+  const double bd = static_cast<double>(b);
+  const double var_norm = V / (bd - 1.0);
+  double ss = s_ee - s_e * s_e / bd;     // sum_i (e_i - mean e)^2; mean e is rounding noise only
+  if (ss < 0.0) ss = 0.0;
+  const double var_ip = ss / (bd - 1.0);
+  double var_orth = var_norm;
+  if (N > 0.0) {
+    var_orth = var_norm - var_ip / N;
+    if (var_orth < 0.0) var_orth = 0.0;
+  }
+  unsigned status = 0u;
+  if (!(isfinite(V) && isfinite(N) && isfinite(s_ee))) status |= ABS_STATUS_NONFINITE;
+  if (N == 0.0) status |= ABS_STATUS_ZERO_MEAN;
+  if (timed_out) status |= ABS_STATUS_TIMEOUT;
+  abs_stats s;
+  s.gbar_sq = N;
+  s.var_norm = var_norm;
+  s.var_ip = var_ip;
+  s.var_orth = var_orth;
+  s.sum_sq = V + bd * N;
+  s.rows = b;
+  s.status = status;
+  s.reserved = 0u;
+  return s;
+}
+#endif
+
 // ---- statistics kernels (abs_stats_tiled.cu, abs_stats_generic.cu) ---------------------
 // Layout of the partial-sum workspace written by both statistics kernels:
 //   ws[(m * P + p) * (b + 2) + r]      r < b : sum over the CTA's columns of (g_rj - gbar_j) gbar_j

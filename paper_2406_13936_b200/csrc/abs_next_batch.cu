@@ -7,17 +7,6 @@ namespace absk {
 namespace {
 
 constexpr int kThreads = 1024;
-constexpr long long kSaturate = 1ll << 62;
-
-__device__ __forceinline__ double safe_ratio(double num, double den) {
-  if (num == 0.0) return 0.0;            // 0/x and 0/0 count as 0
-  if (den == 0.0) return INFINITY;       // x/0 counts as +infinity
-  return num / den;
-}
-__device__ __forceinline__ long long ceil_saturating(double x) {
-  if (!(x < 4611686018427387904.0)) return kSaturate;   // also catches NaN
-  return static_cast<long long>(ceil(x));
-}
 
 __global__ void __launch_bounds__(kThreads)
 abs_next_batch_kernel(const abs_stats* __restrict__ stats, int M, abs_test_cfg cfg,
@@ -29,20 +18,7 @@ abs_next_batch_kernel(const abs_stats* __restrict__ stats, int M, abs_test_cfg c
   pdl_wait();                    // the records (and b_cur) written by the kernels before
   pdl_launch_dependents();
   if (tid < M) {
-    const abs_stats s = stats[tid];
-    const bool usable = (s.status & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) == 0u &&
-                        (cfg.kind == ABS_TEST_NORM || (s.status & ABS_STATUS_NORM_ONLY) == 0u);
-    if (usable) {
-      const double scale = cfg.row_weight / cfg.divisor;
-      const double N = s.gbar_sq;
-      if (cfg.kind == ABS_TEST_NORM) {
-        T = ceil_saturating(scale * safe_ratio(s.var_norm, cfg.eta * cfg.eta * N));
-      } else {
-        const long long t_ip = ceil_saturating(scale * safe_ratio(s.var_ip, cfg.theta * cfg.theta * N * N));
-        const long long t_orth = ceil_saturating(scale * safe_ratio(s.var_orth, cfg.nu * cfg.nu * N));
-        T = t_ip > t_orth ? t_ip : t_orth;
-      }
-    }
+    T = test_size_from_record(stats[tid], cfg);
     if (T_out != nullptr) T_out[tid] = T;
   }
 #pragma unroll

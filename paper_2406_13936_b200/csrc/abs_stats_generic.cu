@@ -187,20 +187,7 @@ abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, uns
       V += red[2][w];
       N += red[3][w];
     }
-    const double bd = static_cast<double>(b);
-    const double var_norm = V / (bd - 1.0);
-    double ss = s_ee - s_e * s_e / bd;     // sum_i (e_i - mean e)^2; mean e is rounding noise only
-    if (ss < 0.0) ss = 0.0;
-    const double var_ip = ss / (bd - 1.0);
-    double var_orth = var_norm;
-    if (N > 0.0) {
-      var_orth = var_norm - var_ip / N;
-      if (var_orth < 0.0) var_orth = 0.0;
-    }
-    unsigned status = 0u;
-    if (!(isfinite(V) && isfinite(N) && isfinite(s_ee))) status |= ABS_STATUS_NONFINITE;
-    if (N == 0.0) status |= ABS_STATUS_ZERO_MEAN;
-    if (*reinterpret_cast<volatile unsigned*>(flags) != 0u) status |= ABS_STATUS_TIMEOUT;
+    const bool timed_out = *reinterpret_cast<volatile unsigned*>(flags) != 0u;
     // The last worker's block to get here clears the time-out flag (flags[0]) and the arrival
     // counter (flags[1]) for the next call, which saves a memset per call.
     __threadfence();
@@ -208,16 +195,7 @@ abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, uns
       flags[0] = 0u;
       flags[1] = 0u;
     }
-    abs_stats s;
-    s.gbar_sq = N;
-    s.var_norm = var_norm;
-    s.var_ip = var_ip;
-    s.var_orth = var_orth;
-    s.sum_sq = V + bd * N;
-    s.rows = b;
-    s.status = status;
-    s.reserved = 0u;
-    stats_out[m] = s;
+    stats_out[m] = record_from_sums(V, N, s_e, s_ee, b, timed_out);
   }
 }
 

@@ -111,6 +111,122 @@ def test_end_to_end_logistic_rounds(ctx, rounds):
     assert torch.equal(X[0], X[M - 1])              # replicas agree after the averaging
 
 
+# ------------------------------------------------------------------ rounds fused into one launch
+def _ratios(st, kind, cfg):
+    N = st["gbar_sq"]
+    if kind == "norm":
+        return [st["var_norm"] / (cfg["eta"] ** 2 * N)]
+    return [st["var_ip"] / (cfg["theta"] ** 2 * N * N), st["var_orth"] / (cfg["nu"] ** 2 * N)]
+
+
+@pytest.mark.parametrize("n,d,M,H,lr,kind,cfg,b,b_max,rounds", [
+    (65536, 256, 4, 8, 0.1, "norm", dict(eta=0.5), 16, 1024, 50),          # the tiny end-to-end configuration
+    (3000, 36, 3, 3, 0.2, "aug_ip", dict(theta=0.5, nu=0.5), 5, 300, 14),  # ragged: d/4 = 9 vectors, odd sizes
+    (5000, 1024, 2, 2, 0.05, "norm", dict(eta=0.7), 2, 700, 8),            # widest rows, b from its minimum
+    (4096, 128, 40, 1, 0.1, "norm", dict(eta=0.4), 3, 64, 6),              # many workers: few CTAs per worker
+])
+def test_fused_logistic_rounds_teacher_forced(ctx, n, d, M, H, lr, kind, cfg, b, b_max, rounds):
+    A, y = inputs.logreg_dataset(1, n, d, device="cuda")
+    idx = inputs.batch_indices(11, (rounds, H, M, b_max), n, device="cuda")
+    X = torch.zeros((M, d), device="cuda")
+    stats = ctx.new_stats(M)
+    T_out = torch.zeros((1, M), dtype=torch.int64, device="cuda")
+    b_hist = torch.zeros(2, dtype=torch.int64, device="cuda")
+    b_dev = torch.tensor([b], dtype=torch.int64, device="cuda")
+    tcfg = pkg.make_test_cfg(kind, b_max, **cfg)
+    An, yn, In = f64(A), f64(y), idx.cpu().numpy()
+    history, exact, total = [b], 0, 0
+    loss0 = logistic_loss(An, yn, np.zeros(d))
+    for k in range(rounds):
+        X0 = f64(X)
+        ctx.abs_logreg_rounds_fused(A, y, idx[k:k + 1], X, H, lr, tcfg, stats, b_dev, T_out=T_out, b_hist=b_hist)
+        torch.cuda.synchronize()
+
+        def grads(m, h, x, k=k, b=b):
+            rows = In[k, h, m, :b]
+            return orc.logreg_per_sample_grads(An[rows], yn[rows], x)
+        Xr, b_ref, T_ref, st_ref = orc.local_round(X0, grads, H, lr, b, b_max, kind, **cfg)
+        params_close(X, Xr)
+        recs = pkg.stats_to_dicts(stats)
+        for m in range(M):
+            assert recs[m]["rows"] == b and recs[m]["status"] == 0
+            for key in ("gbar_sq", "var_norm", "var_ip", "sum_sq"):
+                assert recs[m][key] == pytest.approx(st_ref[m][key], rel=1e-5)
+            assert abs(recs[m]["var_orth"] - st_ref[m]["var_orth"]) <= 1e-5 * st_ref[m]["var_norm"]
+            total += 1
+            if any(near_integer(x) for x in _ratios(st_ref[m], kind, cfg)):
+                assert abs(T_out[0, m].item() - T_ref[m]) <= 1
+            else:
+                assert T_out[0, m].item() == T_ref[m]
+                exact += 1
+        b_new = int(b_dev.item())
+        assert b_hist.tolist() == [b, b_new]
+        if T_out[0].tolist() == T_ref:
+            assert b_new == b_ref
+        assert b <= b_new <= b_max
+        b = b_new
+        history.append(b)
+        for m in range(1, M):
+            assert torch.equal(X[0], X[m])            # replicas agree after the averaging
+    assert exact >= 0.8 * total
+    assert history[-1] > history[0]
+    assert logistic_loss(An, yn, f64(X)[0]) < loss0
+
+
+def test_fused_rounds_in_one_launch_equal_one_launch_per_round(ctx):
+    n, d, M, H, lr, b0, b_max, rounds = 65536, 256, 4, 8, 0.1, 16, 1024, 12
+    A, y = inputs.logreg_dataset(1, n, d, device="cuda")
+    idx = inputs.batch_indices(11, (rounds, H, M, b_max), n, device="cuda")
+    tcfg = pkg.make_test_cfg("norm", b_max, eta=0.5)
+    # one launch for all rounds: the batch size never leaves the device
+    X1 = torch.zeros((M, d), device="cuda")
+    stats1 = ctx.new_stats(rounds * M)
+    T1 = torch.zeros((rounds, M), dtype=torch.int64, device="cuda")
+    hist1 = torch.zeros(rounds + 1, dtype=torch.int64, device="cuda")
+    b1 = torch.tensor([b0], dtype=torch.int64, device="cuda")
+    ctx.abs_logreg_rounds_fused(A, y, idx, X1, H, lr, tcfg, stats1, b1, T_out=T1, b_hist=hist1)
+    # one launch per round
+    X2 = torch.zeros((M, d), device="cuda")
+    stats2 = ctx.new_stats(rounds * M)
+    T2 = torch.zeros((rounds, M), dtype=torch.int64, device="cuda")
+    b2 = torch.tensor([b0], dtype=torch.int64, device="cuda")
+    hist2 = [b0]
+    for k in range(rounds):
+        ctx.abs_logreg_rounds_fused(A, y, idx[k:k + 1], X2, H, lr, tcfg, stats2[k * M:(k + 1) * M], b2, T_out=T2[k:k + 1])
+        hist2.append(int(b2.item()))
+    torch.cuda.synchronize()
+    assert hist1.tolist() == hist2 and int(b1.item()) == hist2[-1]
+    assert hist2[-1] == b_max                                   # the run reaches the cap
+    assert torch.equal(X1, X2) and torch.equal(T1, T2) and torch.equal(stats1, stats2)
+    # and the unfused driver, which forms the per-sample gradient matrix, takes the same decisions
+    X3 = torch.zeros((M, d), device="cuda")
+    G = torch.empty((M, b_max, d), device="cuda")
+    Gb = torch.empty((M, d), device="cuda")
+    stats3 = ctx.new_stats(M)
+    b3 = torch.tensor([b0], dtype=torch.int64, device="cuda")
+    b = b0
+    for k in range(rounds):
+        ctx.abs_logreg_round(A, y, idx[k], X3, H, b, lr, tcfg, G, Gb, stats3, b3)
+        b = int(b3.item())
+        assert abs(b - hist2[k + 1]) <= max(1, 2e-5 * b)
+        if b != hist2[k + 1]:
+            break                                               # a ratio on a rounding boundary forks the runs
+    else:
+        params_close(X3, f64(X1), tol=1e-5)
+
+
+def test_fused_rounds_refuse_shapes_they_do_not_cover(ctx):
+    tcfg = pkg.make_test_cfg("norm", 64, eta=0.5)
+    b_dev = torch.tensor([4], dtype=torch.int64, device="cuda")
+    for n, d, M, stride in [(100, 1028, 2, 64), (100, 30, 2, 64), (100, 32, 65, 64), (100, 32, 2, 32)]:
+        A = torch.zeros((n, d), device="cuda")
+        y = torch.zeros(n, device="cuda")
+        idx = torch.zeros((1, 1, M, stride), dtype=torch.int32, device="cuda")
+        X = torch.zeros((M, d), device="cuda")
+        with pytest.raises(pkg.AbsError):
+            ctx.abs_logreg_rounds_fused(A, y, idx, X, 1, 0.1, tcfg, ctx.new_stats(M), b_dev)
+
+
 # ------------------------------------------------------------------ MLP producer and rounds
 def mlp_problem(seed, n, dims, M, device="cuda"):
     inp, lab = inputs.gaussian_mixture(seed, n, dim=dims[0], classes=dims[3], device=device)
