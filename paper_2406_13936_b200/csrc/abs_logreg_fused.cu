@@ -2,31 +2,34 @@
 // (Algorithm 2's structure with Algorithm 1's per-sample statistic once per round, Section 4.3).
 //
 // The round driver abs_logreg_round enqueues about four small kernels per local step; for a
-// problem of a few hundred parameters every one of them is pure launch latency.  Here a grid of
-// M x P resident CTAs (P CTAs per worker, all co-resident: cooperative launch) keeps the
-// parameters of its worker in shared memory and walks through the steps with one grid-wide
-// barrier per local step:
+// problem of a few hundred parameters every one of them is pure launch latency.  Here each
+// worker is ONE thread-block cluster of P CTAs (P = 16, 8, ... - the largest that leaves all M
+// clusters co-resident), every CTA keeps the worker's parameters in shared memory, and a local
+// step needs nothing outside the cluster:
 //
 //   phase A   every warp takes samples of the step's batch: z = <a_i, x>, r_i = sigmoid(z) - y_i,
-//             and adds r_i a_i to its partial batch gradient; one partial per CTA goes to global
-//             memory
-//   barrier
-//   phase B   every CTA of the worker adds the P partials in a fixed order -> gbar (Eq. batch_grad)
-//             and takes the step x <- x - lr gbar (Eq. local_sgd_alt); all CTAs of a worker do the
-//             same arithmetic, so their copies of x stay bit-identical
+//             and adds r_i a_i to its partial batch gradient; the CTA's partial is stored into
+//             the shared memory of every CTA of the cluster (distributed shared memory)
+//   cluster barrier
+//   phase B   every CTA of the worker adds the P partials it received in a fixed order -> gbar
+//             (Eq. batch_grad), then takes the step x <- x - lr gbar (Eq. local_sgd_alt); all
+//             CTAs of a worker do the same arithmetic, so their copies of x stay bit-identical
 //   last step of a round, between B and the update:
 //   phase C   the CTA's samples again (from L1/L2): sum_i ||g_i - gbar||^2, e_i = <g_i - gbar, gbar>
-//             (Eq. def_var, centred), partial sums per CTA in fp64
-//   barrier
+//             (Eq. def_var, centred), partial sums per CTA in fp64, to global memory
+//   grid barrier (the only one of the round: the workers meet here)
 //   phase D   model averaging over the M workers (Eq. local_sgd_alt, second line), the records,
 //             T per worker, b <- min(b_max, max(b, max_m T_m)) (Algorithm 1) - computed by every
 //             CTA from the same numbers, so the next round's batch size needs no further barrier
 //             and never leaves the device.
 //
-// The per-sample gradient matrix is never written.  Data written by one CTA and read by another
-// inside the launch goes through L2 only (st.cg / ld.cg); buffers are reused no sooner than two
-// barriers later.  Every CTA executes the same sequence of barriers: the trip counts depend only
-// on (rounds, H) and on b, which all CTAs derive from the same values.
+// The per-sample gradient matrix is never written.  The received partials alternate between two
+// buffers by step, so one cluster barrier per step is enough: a buffer is rewritten two steps
+// later, after a barrier that its reader reaches only when it has finished reading.  No CTA
+// leaves while a peer may still store into it: a grid barrier follows the last cluster barrier.
+// Data that crosses clusters inside the launch goes through L2 only (st.cg / ld.cg) and is
+// reused no sooner than a grid barrier later.  Every CTA executes the same sequence of barriers:
+// the trip counts depend only on (rounds, H) and on b, which all CTAs derive from the same values.
 #include <cooperative_groups.h>
 
 #include "abs_internal.cuh"
@@ -40,7 +43,7 @@ constexpr int kFW = 8;                     // warps per CTA
 constexpr int kFThreads = kFW * 32;
 constexpr int kMaxWorkersFused = 64;
 constexpr int kMaxDimFused = 1024;
-constexpr int kMaxCtasPerWorker = 32;
+constexpr int kMaxCtasPerWorker = 16;        // = the largest cluster (16 needs the non-portable opt-in)
 
 struct FusedParams {
   const float* A;
@@ -57,16 +60,10 @@ struct FusedParams {
   long long* T_out;
   long long* b_hist;
   long long* b_dev;
-  float* partial;   // [2][M][P][d]   partial batch gradients, two buffers alternate by step
   double* S;        // [M][P][4]      V, sum e, sum e^2, N
   float* Xpre;      // [M][d]         parameters before the averaging
 };
 
-__device__ __forceinline__ float warp_sum_f(float v) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  return v;
-}
 __device__ __forceinline__ double warp_sum_dd(double v) {
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
@@ -85,15 +82,21 @@ __device__ __forceinline__ float residual(float z, float label) {
   return p - label;
 }
 
+__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
 // KV: 16-byte column vectors per lane (slot k of a lane is vector k*32 + lane of the row).
 template <int KV>
 __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const FusedParams prm) {
+  constexpr int U = 16 / KV;               // samples a warp keeps in flight (16 row vectors in registers)
   cg::grid_group grid = cg::this_grid();
   extern __shared__ __align__(16) float smem_f[];
   const int d = prm.d, DV = d >> 2;
   float4* x4 = reinterpret_cast<float4*>(smem_f);              // [DV] parameters of this worker
   float4* g4 = x4 + DV;                                         // [DV] batch gradient of the step
   float4* wacc4 = g4 + DV;                                      // [kFW][DV] per-warp partial sums
+  float4* inbox4 = wacc4 + kFW * DV;                            // [2][P][DV] the partial batch gradients of all
+                                                                // CTAs of the cluster, written by their owners
+  cg::cluster_group cluster = cg::this_cluster();
   __shared__ double red[kFW][3];
   __shared__ double N_s;
   __shared__ long long T_s[kMaxWorkersFused];
@@ -114,76 +117,87 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
   if (blockIdx.x == 0 && tid == 0 && prm.b_hist != nullptr) prm.b_hist[0] = b;
   __syncthreads();
 
-  // Row index and label of the warp's t-th sample of the step are fetched by lane t % 32 ahead
-  // of the loop over the samples, so that the loop's loads do not wait for an index first.
+  // Sample i of a step belongs to CTA i % P and there to warp (i / P) % 8.  The row index of the
+  // warp's t-th sample is fetched by lane t % 32 ahead of the loop over the samples; for the
+  // first 32 samples of a warp (all of them unless b > 256 P) that load is issued a whole local
+  // step earlier, and the rows themselves are prefetched before the grid barrier, so that after
+  // the barrier nothing waits for memory that does not depend on the new parameters.
   const long long first = p + static_cast<long long>(P) * warp;     // this warp's first sample
   const long long hop = static_cast<long long>(P) * kFW;
+  auto clamp_row = [&](int raw) -> long long {                       // indices outside the data are clamped
+    return raw < 0 ? 0 : (raw >= prm.n ? prm.n - 1 : static_cast<long long>(raw));
+  };
+  auto fetch_row = [&](const int* idx_step, long long t) { return clamp_row(idx_step[first + t * hop]); };
+  const int lines_per_row = (d * 4 + 127) >> 7;
+  long long chunk0_row = 0;                                          // row of sample `lane` of the current step
 
   for (int r = 0; r < prm.rounds; ++r) {
     const int Pa = static_cast<int>(b < P ? b : P);                 // CTAs of a worker that have samples
     const long long n_mine = b > first ? (b - first + hop - 1) / hop : 0;
     const float inv_b = 1.0f / static_cast<float>(b);
+    chunk0_row = lane < n_mine ? fetch_row(prm.idx + (static_cast<long long>(r) * prm.H * M + m) * prm.idx_stride, lane) : 0;
     for (int h = 0; h < prm.H; ++h) {
       const long long gstep = static_cast<long long>(r) * prm.H + h;
       const bool last = h == prm.H - 1;
       const int* idx_m = prm.idx + (gstep * M + m) * prm.idx_stride;
-      float4* part4 = reinterpret_cast<float4*>(prm.partial) + (gstep & 1) * static_cast<long long>(M) * P * DV;
+      float4* part4 = inbox4 + (gstep & 1) * static_cast<long long>(P) * DV;
 
       // ---- phase A: partial batch gradient of this CTA ------------------------------------
       float4 acc[KV];
 #pragma unroll
       for (int k = 0; k < KV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      // the row indices of the NEXT local step's first chunk: the load is issued here and used after
+      // this step's samples, so it costs nothing
+      // (the value is not touched before the samples of this step are done: an instruction that
+      // used it here would make the warp wait for the load)
+      int ahead_raw = 0;
+      if (!last && lane < n_mine) ahead_raw = (idx_m + static_cast<long long>(M) * prm.idx_stride)[first + lane * hop];
       for (long long t0 = 0; t0 < n_mine; t0 += 32) {
         const int cnt = static_cast<int>(n_mine - t0 < 32 ? n_mine - t0 : 32);
-        long long my_row = 0;
-        float my_label = 0.f;
-        if (lane < cnt) {
-          long long row = idx_m[first + (t0 + lane) * hop];
-          row = row < 0 ? 0 : (row >= prm.n ? prm.n - 1 : row);     // indices outside the data are clamped
-          my_row = row;
-          my_label = prm.y[row];
-        }
-        for (int t = 0; t < cnt; t += 2) {
-          const bool two = t + 1 < cnt;
-          const long long row0 = __shfl_sync(0xffffffffu, my_row, t);
-          const long long row1 = __shfl_sync(0xffffffffu, my_row, two ? t + 1 : t);
-          const float lab0 = __shfl_sync(0xffffffffu, my_label, t);
-          const float lab1 = __shfl_sync(0xffffffffu, my_label, two ? t + 1 : t);
-          float4 a0[KV], a1[KV];
-          float z0 = 0.f, z1 = 0.f;
+        long long my_row = chunk0_row;
+        if (t0 > 0 && lane < cnt) my_row = fetch_row(idx_m, t0 + lane);
+        for (int t = 0; t < cnt; t += U) {
+          // U samples in flight: all their loads are issued before anything is reduced.  A slot past
+          // the end repeats sample t with weight 0.
+          long long rows[U];
+          float lab[U], z[U];
+          float4 a[U][KV];
 #pragma unroll
-          for (int k = 0; k < KV; ++k) {
-            const int j = k * 32 + lane;
-            if (j < DV) {
-              a0[k] = __ldg(A4 + row0 * DV + j);
-              a1[k] = __ldg(A4 + row1 * DV + j);
-            } else {
-              a0[k] = a1[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int u = 0; u < U; ++u) rows[u] = __shfl_sync(0xffffffffu, my_row, t + u < cnt ? t + u : t);
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            lab[u] = __ldg(prm.y + rows[u]);                                  // one address per warp
+#pragma unroll
+            for (int k = 0; k < KV; ++k) {
+              const int j = k * 32 + lane;
+              a[u][k] = j < DV ? __ldg(A4 + rows[u] * DV + j) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+            z[u] = 0.f;
           }
 #pragma unroll
           for (int k = 0; k < KV; ++k) {
             const int j = k * 32 + lane;
             if (j < DV) {
               const float4 xv = x4[j];
-              z0 = dot4(a0[k], xv, z0);
-              z1 = dot4(a1[k], xv, z1);
+#pragma unroll
+              for (int u = 0; u < U; ++u) z[u] = dot4(a[u][k], xv, z[u]);
             }
           }
-          z0 = warp_sum_f(z0);
-          z1 = warp_sum_f(z1);
-          const float r0 = residual(z0, lab0);
-          const float r1 = two ? residual(z1, lab1) : 0.f;
 #pragma unroll
-          for (int k = 0; k < KV; ++k) {
-            acc[k].x = fmaf(r0, a0[k].x, acc[k].x);
-            acc[k].y = fmaf(r0, a0[k].y, acc[k].y);
-            acc[k].z = fmaf(r0, a0[k].z, acc[k].z);
-            acc[k].w = fmaf(r0, a0[k].w, acc[k].w);
-            acc[k].x = fmaf(r1, a1[k].x, acc[k].x);
-            acc[k].y = fmaf(r1, a1[k].y, acc[k].y);
-            acc[k].z = fmaf(r1, a1[k].z, acc[k].z);
-            acc[k].w = fmaf(r1, a1[k].w, acc[k].w);
+          for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) z[u] += __shfl_xor_sync(0xffffffffu, z[u], off);
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            const float rr = t + u < cnt ? residual(z[u], lab[u]) : 0.f;
+#pragma unroll
+            for (int k = 0; k < KV; ++k) {
+              acc[k].x = fmaf(rr, a[u][k].x, acc[k].x);
+              acc[k].y = fmaf(rr, a[u][k].y, acc[k].y);
+              acc[k].z = fmaf(rr, a[u][k].z, acc[k].z);
+              acc[k].w = fmaf(rr, a[u][k].w, acc[k].w);
+            }
           }
         }
       }
@@ -192,19 +206,36 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
         const int j = k * 32 + lane;
         if (j < DV) wacc4[warp * DV + j] = acc[k];
       }
+      if (!last) {
+        // the next step's rows on their way into L1 while the barrier is crossed
+        const long long ahead_row = clamp_row(ahead_raw);
+        const int cnt0 = static_cast<int>(n_mine < 32 ? n_mine : 32);
+        const int total = cnt0 * lines_per_row;
+        for (int q0 = 0; q0 < total; q0 += 32) {
+          const int q = q0 + lane, t = q / lines_per_row;
+          const long long row = __shfl_sync(0xffffffffu, ahead_row, t < cnt0 ? t : 0);
+          if (q < total) prefetch_l1(reinterpret_cast<const char*>(prm.A + row * d) + (q - t * lines_per_row) * 128);
+        }
+        chunk0_row = ahead_row;
+      }
       __syncthreads();
       if (p < Pa) {
-        for (int j = tid; j < DV; j += kFThreads) {
+        // Every thread group adds the warps' sums (all groups get the same bits) and stores the
+        // result into the inboxes of the peers it serves: remote stores are posted, the barrier's
+        // release/acquire makes them visible, and phase B then reads local shared memory only.
+        const int groups = kFThreads / DV >= kFW ? kFW : (kFThreads / DV > 0 ? kFThreads / DV : 1);
+        const int grp = tid / DV, j = tid - grp * DV;
+        if (grp < groups) {
           float4 s = wacc4[j];
 #pragma unroll
           for (int w = 1; w < kFW; ++w) {
             const float4 v = wacc4[w * DV + j];
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
           }
-          __stcg(part4 + (static_cast<long long>(m) * P + p) * DV + j, s);
+          for (int q = grp; q < P; q += groups) cluster.map_shared_rank(part4, q)[p * DV + j] = s;
         }
       }
-      grid.sync();
+      cluster.sync();
 
       // ---- phase B: batch gradient of the worker; the step unless statistics come first -----
       // The P partials are split over thread groups (group q takes partials q, q + groups, ...),
@@ -214,10 +245,9 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
         const int grp = tid / DV, j = tid - grp * DV;
         if (grp < groups) {
           float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-          const float4* src = part4 + static_cast<long long>(m) * P * DV + j;
 #pragma unroll 4
           for (int q = grp; q < Pa; q += groups) {
-            const float4 v = __ldcg(src + static_cast<long long>(q) * DV);
+            const float4 v = part4[q * DV + j];
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
           }
           wacc4[grp * DV + j] = s;
@@ -253,46 +283,72 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
       double V = 0.0, se = 0.0, see = 0.0;
       for (long long t0 = 0; t0 < n_mine; t0 += 32) {
         const int cnt = static_cast<int>(n_mine - t0 < 32 ? n_mine - t0 : 32);
-        long long my_row = 0;
-        float my_label = 0.f;
-        if (lane < cnt) {
-          long long row = idx_m[first + (t0 + lane) * hop];
-          row = row < 0 ? 0 : (row >= prm.n ? prm.n - 1 : row);
-          my_row = row;
-          my_label = prm.y[row];
-        }
-        for (int t = 0; t < cnt; ++t) {
-          const long long row = __shfl_sync(0xffffffffu, my_row, t);
-          const float lab = __shfl_sync(0xffffffffu, my_label, t);
-          float4 a[KV];
-          float z = 0.f;
+        long long my_row = chunk0_row;
+        if (t0 > 0 && lane < cnt) my_row = fetch_row(idx_m, t0 + lane);
+        for (int t = 0; t < cnt; t += U) {
+          long long rows[U];
+          float lab[U], z[U], s1[U], s2[U];
+          float4 a[U][KV];
+#pragma unroll
+          for (int u = 0; u < U; ++u) rows[u] = __shfl_sync(0xffffffffu, my_row, t + u < cnt ? t + u : t);
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            lab[u] = __ldg(prm.y + rows[u]);
+#pragma unroll
+            for (int k = 0; k < KV; ++k) {
+              const int j = k * 32 + lane;
+              a[u][k] = j < DV ? __ldg(A4 + rows[u] * DV + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            z[u] = s1[u] = s2[u] = 0.f;
+          }
 #pragma unroll
           for (int k = 0; k < KV; ++k) {
             const int j = k * 32 + lane;
             if (j < DV) {
-              a[k] = __ldg(A4 + row * DV + j);
-              z = dot4(a[k], x4[j], z);
+              const float4 xv = x4[j];
+#pragma unroll
+              for (int u = 0; u < U; ++u) z[u] = dot4(a[u][k], xv, z[u]);
             }
           }
-          z = warp_sum_f(z);
-          const float rr = residual(z, lab);
-          float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) z[u] += __shfl_xor_sync(0xffffffffu, z[u], off);
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u) z[u] = residual(z[u], lab[u]);           // from here on z holds r_i
 #pragma unroll
           for (int k = 0; k < KV; ++k) {
             const int j = k * 32 + lane;
             if (j < DV) {
               const float4 gv = g4[j];
-              const float tx = fmaf(rr, a[k].x, -gv.x), ty = fmaf(rr, a[k].y, -gv.y);
-              const float tz = fmaf(rr, a[k].z, -gv.z), tw = fmaf(rr, a[k].w, -gv.w);
-              s1 = fmaf(tx, tx, s1); s1 = fmaf(ty, ty, s1); s1 = fmaf(tz, tz, s1); s1 = fmaf(tw, tw, s1);
-              s2 = fmaf(tx, gv.x, s2); s2 = fmaf(ty, gv.y, s2); s2 = fmaf(tz, gv.z, s2); s2 = fmaf(tw, gv.w, s2);
+#pragma unroll
+              for (int u = 0; u < U; ++u) {
+                const float tx = fmaf(z[u], a[u][k].x, -gv.x), ty = fmaf(z[u], a[u][k].y, -gv.y);
+                const float tz = fmaf(z[u], a[u][k].z, -gv.z), tw = fmaf(z[u], a[u][k].w, -gv.w);
+                s1[u] = fmaf(tx, tx, s1[u]); s1[u] = fmaf(ty, ty, s1[u]);
+                s1[u] = fmaf(tz, tz, s1[u]); s1[u] = fmaf(tw, tw, s1[u]);
+                s2[u] = fmaf(tx, gv.x, s2[u]); s2[u] = fmaf(ty, gv.y, s2[u]);
+                s2[u] = fmaf(tz, gv.z, s2[u]); s2[u] = fmaf(tw, gv.w, s2[u]);
+              }
             }
           }
-          s1 = warp_sum_f(s1);
-          s2 = warp_sum_f(s2);
-          V += static_cast<double>(s1);
-          se += static_cast<double>(s2);
-          see += static_cast<double>(s2) * static_cast<double>(s2);
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              s1[u] += __shfl_xor_sync(0xffffffffu, s1[u], off);
+              s2[u] += __shfl_xor_sync(0xffffffffu, s2[u], off);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            if (t + u < cnt) {
+              V += static_cast<double>(s1[u]);
+              se += static_cast<double>(s2[u]);
+              see += static_cast<double>(s2[u]) * static_cast<double>(s2[u]);
+            }
+          }
         }
       }
       if (lane == 0) {
@@ -326,31 +382,56 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
       grid.sync();
 
       // ---- phase D: averaging, records, next batch size ---------------------------------------
-      const float inv_M = 1.0f / static_cast<float>(M);
-      for (int j = tid; j < DV; j += kFThreads) {
-        float4 s = __ldcg(Xpre4 + j);
-        for (int w = 1; w < M; ++w) {
-          const float4 v = __ldcg(Xpre4 + static_cast<long long>(w) * DV + j);
-          s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      // The loads of this phase come from L2 and nothing else is left to overlap them with, so
+      // they are spread over the threads and issued together: the records by one warp per worker
+      // (lane q reads the sums of CTA q; the shuffle tree adds them in a fixed order), the
+      // parameters by thread groups that split the workers and are added in group order.
+      for (int w = warp; w < M; w += kFW) {
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, nn = 0.0;
+        if (lane < Pa) {
+          const double* src = prm.S + (static_cast<long long>(w) * P + lane) * 4;
+          a0 = __ldcg(src + 0);
+          a1 = __ldcg(src + 1);
+          a2 = __ldcg(src + 2);
+          nn = __ldcg(src + 3);
         }
-        s.x *= inv_M; s.y *= inv_M; s.z *= inv_M; s.w *= inv_M;
-        x4[j] = s;
-        if (p == 0 && r == prm.rounds - 1) X4[static_cast<long long>(m) * DV + j] = s;
+        a0 = warp_sum_dd(a0);
+        a1 = warp_sum_dd(a1);
+        a2 = warp_sum_dd(a2);
+        nn = __shfl_sync(0xffffffffu, nn, 0);
+        if (lane == 0) {
+          const abs_stats rec = record_from_sums(a0, nn, a1, a2, b, false);
+          const long long T = test_size_from_record(rec, prm.cfg);
+          T_s[w] = T;
+          if (blockIdx.x == 0) {
+            prm.stats[static_cast<long long>(r) * M + w] = rec;
+            if (prm.T_out != nullptr) prm.T_out[static_cast<long long>(r) * M + w] = T;
+          }
+        }
       }
-      if (tid < M) {
-        const double* src = prm.S + static_cast<long long>(tid) * P * 4;
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0;
-        for (int q = 0; q < Pa; ++q) {
-          a0 += __ldcg(src + q * 4 + 0);
-          a1 += __ldcg(src + q * 4 + 1);
-          a2 += __ldcg(src + q * 4 + 2);
+      {
+        const float inv_M = 1.0f / static_cast<float>(M);
+        const int groups = kFThreads / DV >= kFW ? kFW : (kFThreads / DV > 0 ? kFThreads / DV : 1);
+        const int grp = tid / DV, j = tid - grp * DV;
+        if (grp < groups) {
+          float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+          for (int w = grp; w < M; w += groups) {
+            const float4 v = __ldcg(Xpre4 + static_cast<long long>(w) * DV + j);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+          }
+          wacc4[grp * DV + j] = s;
         }
-        const abs_stats rec = record_from_sums(a0, __ldcg(src + 3), a1, a2, b, false);
-        const long long T = test_size_from_record(rec, prm.cfg);
-        T_s[tid] = T;
-        if (blockIdx.x == 0) {
-          prm.stats[static_cast<long long>(r) * M + tid] = rec;
-          if (prm.T_out != nullptr) prm.T_out[static_cast<long long>(r) * M + tid] = T;
+        __syncthreads();
+        for (int jj = tid; jj < DV; jj += kFThreads) {
+          float4 s = wacc4[jj];
+          for (int q = 1; q < groups; ++q) {
+            const float4 v = wacc4[q * DV + jj];
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+          }
+          s.x *= inv_M; s.y *= inv_M; s.z *= inv_M; s.w *= inv_M;
+          x4[jj] = s;
+          if (p == 0 && r == prm.rounds - 1) X4[static_cast<long long>(m) * DV + jj] = s;
         }
       }
       __syncthreads();
@@ -416,34 +497,57 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
 
   const int DV = static_cast<int>(d / 4);
   KernelFn kernel = pick_kernel(DV);
-  const size_t smem = static_cast<size_t>(2 + kFW) * d * sizeof(float);
-  int per_sm = 0;
-  ABS_CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kFThreads, smem));
-  const long long resident = static_cast<long long>(per_sm) * ctx->sm_count;
-  long long P = resident / M;
-  if (P > kMaxCtasPerWorker) P = kMaxCtasPerWorker;
-  if (P < 1) return set_error(ctx, ABS_ERR_UNSUPPORTED, "%d workers do not fit a co-resident grid (%lld CTAs)", M, resident);
+  const size_t smem_fixed = static_cast<size_t>(2 + kFW) * d * sizeof(float);   // + 2 P d floats of inboxes
 
-  // scratch in the context's workspace: partial gradients, statistics partials, pre-average parameters
-  const size_t partial_bytes = 2ull * M * P * d * sizeof(float);
+  // One cluster per worker: the largest cluster size that leaves all M clusters co-resident.
+  cudaLaunchConfig_t lc = {};
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeClusterDimension;
+  attrs[1].id = cudaLaunchAttributeCooperative;
+  attrs[1].val.cooperative = 1;
+  lc.blockDim = dim3(kFThreads);
+  lc.stream = static_cast<cudaStream_t>(stream);
+  lc.attrs = attrs;
+  lc.numAttrs = 2;
+  ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel),
+                                         cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  int P = 0;
+  for (int cand = kMaxCtasPerWorker; cand >= 1 && P == 0; cand >>= 1) {
+    const size_t smem = smem_fixed + 2ull * cand * d * sizeof(float);
+    if (smem + 1024 > ctx->smem_optin) continue;      // 1 KiB for the static shared variables
+    ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel),
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    lc.dynamicSmemBytes = smem;
+    attrs[0].val.clusterDim.x = static_cast<unsigned>(cand);
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    lc.gridDim = dim3(static_cast<unsigned>(M * cand));
+    int clusters = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, reinterpret_cast<const void*>(kernel), &lc);
+    if (e != cudaSuccess) {
+      cudaGetLastError();        // this cluster size is not available on the device: try the next
+      continue;
+    }
+    if (clusters >= M) P = cand;
+  }
+  if (P == 0) return set_error(ctx, ABS_ERR_UNSUPPORTED, "%d workers do not fit a co-resident grid", M);
+
+  // scratch in the context's workspace: statistics partials, pre-average parameters
   const size_t S_bytes = static_cast<size_t>(M) * P * 4 * sizeof(double);
   const size_t xpre_bytes = static_cast<size_t>(M) * d * sizeof(float);
-  if (partial_bytes + S_bytes + xpre_bytes > ctx->workspace_bytes)
+  if (S_bytes + xpre_bytes > ctx->workspace_bytes)
     return set_error(ctx, ABS_ERR_WORKSPACE, "workspace of %zu bytes is too small (%zu needed)", ctx->workspace_bytes,
-                     partial_bytes + S_bytes + xpre_bytes);
+                     S_bytes + xpre_bytes);
   unsigned char* ws = static_cast<unsigned char*>(ctx->workspace);
 
   FusedParams prm;
   prm.A = A; prm.y = y; prm.n = n; prm.d = static_cast<int>(d);
   prm.idx = idx; prm.idx_stride = idx_stride;
-  prm.rounds = rounds; prm.M = M; prm.H = H; prm.P = static_cast<int>(P);
+  prm.rounds = rounds; prm.M = M; prm.H = H; prm.P = P;
   prm.lr = lr; prm.cfg = *cfg;
   prm.X = X; prm.stats = stats; prm.T_out = T_out; prm.b_hist = b_hist; prm.b_dev = b_dev;
-  prm.partial = reinterpret_cast<float*>(ws);
-  prm.S = reinterpret_cast<double*>(ws + partial_bytes);
-  prm.Xpre = reinterpret_cast<float*>(ws + partial_bytes + S_bytes);
-  void* args[] = {&prm};
-  ABS_CUDA_TRY(ctx, cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kernel), dim3(static_cast<unsigned>(M * P)),
-                                                dim3(kFThreads), args, smem, static_cast<cudaStream_t>(stream)));
+  prm.S = reinterpret_cast<double*>(ws);
+  prm.Xpre = reinterpret_cast<float*>(ws + S_bytes);
+  ABS_CUDA_TRY(ctx, cudaLaunchKernelEx(&lc, kernel, prm));
   return ABS_OK;
 }
