@@ -5,12 +5,13 @@
 // problem of a few hundred parameters every one of them is pure launch latency.  Here each
 // worker is ONE thread-block cluster of P CTAs (P = 16, 8, ... - the largest that leaves all M
 // clusters co-resident), every CTA keeps the worker's parameters in shared memory, and a local
-// step needs nothing outside the cluster:
+// step needs nothing outside the cluster's shared memory:
 //
 //   phase A   every warp takes samples of the step's batch: z = <a_i, x>, r_i = sigmoid(z) - y_i,
-//             and adds r_i a_i to its partial batch gradient; the CTA's partial is stored into
-//             the shared memory of every CTA of the cluster (distributed shared memory)
-//   cluster barrier
+//             and adds r_i a_i to its partial batch gradient; the CTA's partial goes into the
+//             shared memory of every CTA of the cluster by one bulk copy per peer
+//             (cp.async.bulk shared::cta -> shared::cluster) that signals the peer's mbarrier
+//   wait      on the CTA's own mbarrier until the partials of all peers have arrived (bounded)
 //   phase B   every CTA of the worker adds the P partials it received in a fixed order -> gbar
 //             (Eq. batch_grad), then takes the step x <- x - lr gbar (Eq. local_sgd_alt); all
 //             CTAs of a worker do the same arithmetic, so their copies of x stay bit-identical
@@ -23,16 +24,19 @@
 //             CTA from the same numbers, so the next round's batch size needs no further barrier
 //             and never leaves the device.
 //
-// The per-sample gradient matrix is never written.  The received partials alternate between two
-// buffers by step, so one cluster barrier per step is enough: a buffer is rewritten two steps
-// later, after a barrier that its reader reaches only when it has finished reading.  No CTA
-// leaves while a peer may still store into it: a grid barrier follows the last cluster barrier.
+// The per-sample gradient matrix is never written.  A local step has no cluster-wide barrier:
+// the received partials (and the copies' source) alternate between two buffers by step, and a
+// peer can only send the partial of step h + 2 after it has received this CTA's partial of step
+// h + 1, which is sent after the buffer of step h has been read.  A wait that runs out raises a
+// flag, all later waits of the CTA return at once, the barriers that follow are still reached,
+// and the round's records carry ABS_STATUS_TIMEOUT.  No CTA leaves while a peer may still copy
+// into it: a grid barrier follows the last exchange.
 // Data that crosses clusters inside the launch goes through L2 only (st.cg / ld.cg) and is
 // reused no sooner than a grid barrier later.  Every CTA executes the same sequence of barriers:
 // the trip counts depend only on (rounds, H) and on b, which all CTAs derive from the same values.
 #include <cooperative_groups.h>
 
-#include "abs_internal.cuh"
+#include "abs_pipeline.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -60,6 +64,9 @@ struct FusedParams {
   long long* T_out;
   long long* b_hist;
   long long* b_dev;
+  unsigned* flag;   // device word, zero at launch: set when a wait for the peers' partials ran out
+  long long timeout_cycles;
+  int drop_copies;  // test hook: the partials are not sent, so the waits run out
   double* S;        // [M][P][4]      V, sum e, sum e^2, N
   float* Xpre;      // [M][d]         parameters before the averaging
 };
@@ -96,7 +103,11 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
   float4* wacc4 = g4 + DV;                                      // [kFW][DV] per-warp partial sums
   float4* inbox4 = wacc4 + kFW * DV;                            // [2][P][DV] the partial batch gradients of all
                                                                 // CTAs of the cluster, written by their owners
-  cg::cluster_group cluster = cg::this_cluster();
+  float4* outbox4 = inbox4 + 2 * prm.P * DV;                    // [2][DV] this CTA's partial, source of the copies
+  __shared__ __align__(8) unsigned long long xbar[2];           // "all partials of the step have arrived"
+  __shared__ unsigned abort_s;
+  volatile unsigned* abort_flag = &abort_s;
+  const uint32_t xbar_u32 = smem_u32(xbar);
   __shared__ double red[kFW][3];
   __shared__ double N_s;
   __shared__ long long T_s[kMaxWorkersFused];
@@ -115,7 +126,14 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
   if (b > prm.cfg.b_max) b = prm.cfg.b_max;
   if (b < 2) b = 2;                        // the variance needs two rows
   if (blockIdx.x == 0 && tid == 0 && prm.b_hist != nullptr) prm.b_hist[0] = b;
-  __syncthreads();
+  if (tid == 0) {
+    mbar_init(xbar_u32, 1);
+    mbar_init(xbar_u32 + 8u, 1);
+    abort_s = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  cg::this_cluster().sync();               // every CTA's barriers exist before a peer signals them
 
   // Sample i of a step belongs to CTA i % P and there to warp (i / P) % 8.  The row index of the
   // warp's t-th sample is fetched by lane t % 32 ahead of the loop over the samples; for the
@@ -219,23 +237,38 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
         chunk0_row = ahead_row;
       }
       __syncthreads();
+      // The CTA's partial goes into its own slot of the inbox and, by one bulk copy per peer that
+      // signals the peer's barrier, into the same slot of every other CTA of the cluster.  Nobody
+      // waits for anybody but the data: there is no cluster-wide barrier in a step.
+      const uint32_t par = static_cast<uint32_t>(gstep & 1);
+      const uint32_t bytes = static_cast<uint32_t>(DV) * 16u;
       if (p < Pa) {
-        // Every thread group adds the warps' sums (all groups get the same bits) and stores the
-        // result into the inboxes of the peers it serves: remote stores are posted, the barrier's
-        // release/acquire makes them visible, and phase B then reads local shared memory only.
-        const int groups = kFThreads / DV >= kFW ? kFW : (kFThreads / DV > 0 ? kFThreads / DV : 1);
-        const int grp = tid / DV, j = tid - grp * DV;
-        if (grp < groups) {
+        for (int j = tid; j < DV; j += kFThreads) {
           float4 s = wacc4[j];
 #pragma unroll
           for (int w = 1; w < kFW; ++w) {
             const float4 v = wacc4[w * DV + j];
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
           }
-          for (int q = grp; q < P; q += groups) cluster.map_shared_rank(part4, q)[p * DV + j] = s;
+          outbox4[par * DV + j] = s;
+          part4[p * DV + j] = s;
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the copies read what was just written
       }
-      cluster.sync();
+      __syncthreads();
+      // After a wait has run out this CTA takes no further part in the exchange: its barrier's
+      // phase never completed, and a second arrival in the same phase is not allowed.  Its peers
+      // then run into their own limits.
+      if (warp == 0 && *abort_flag == 0u) {
+        if (lane == 0) mbar_expect_tx(xbar_u32 + 8u * par, static_cast<uint32_t>(Pa - (p < Pa ? 1 : 0)) * bytes);
+        __syncwarp();
+        if (p < Pa && lane < P && lane != p && !prm.drop_copies)
+          bulk_copy_to_peer(map_to_rank(smem_u32(part4 + p * DV), static_cast<uint32_t>(lane)),
+                            smem_u32(outbox4 + par * DV), bytes,
+                            map_to_rank(xbar_u32 + 8u * par, static_cast<uint32_t>(lane)));
+      }
+      // barrier `par` is used every other step: its phase bit is bit 1 of the step count
+      mbar_wait(xbar_u32 + 8u * par, static_cast<uint32_t>((gstep >> 1) & 1), abort_flag, prm.timeout_cycles);
 
       // ---- phase B: batch gradient of the worker; the step unless statistics come first -----
       // The P partials are split over thread groups (group q takes partials q, q + groups, ...),
@@ -379,7 +412,9 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
         x4[j] = xv;
         if (p == 0) __stcg(Xpre4 + static_cast<long long>(m) * DV + j, xv);
       }
+      if (tid == 0 && abort_s != 0u) atomicOr(prm.flag, 1u);
       grid.sync();
+      const bool timed_out = __ldcg(prm.flag) != 0u;
 
       // ---- phase D: averaging, records, next batch size ---------------------------------------
       // The loads of this phase come from L2 and nothing else is left to overlap them with, so
@@ -400,7 +435,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
         a2 = warp_sum_dd(a2);
         nn = __shfl_sync(0xffffffffu, nn, 0);
         if (lane == 0) {
-          const abs_stats rec = record_from_sums(a0, nn, a1, a2, b, false);
+          const abs_stats rec = record_from_sums(a0, nn, a1, a2, b, timed_out);
           const long long T = test_size_from_record(rec, prm.cfg);
           T_s[w] = T;
           if (blockIdx.x == 0) {
@@ -497,7 +532,7 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
 
   const int DV = static_cast<int>(d / 4);
   KernelFn kernel = pick_kernel(DV);
-  const size_t smem_fixed = static_cast<size_t>(2 + kFW) * d * sizeof(float);   // + 2 P d floats of inboxes
+  const size_t smem_fixed = static_cast<size_t>(2 + kFW + 2) * d * sizeof(float);   // + 2 P d floats of inboxes
 
   // One cluster per worker: the largest cluster size that leaves all M clusters co-resident.
   cudaLaunchConfig_t lc = {};
@@ -546,6 +581,10 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
   prm.rounds = rounds; prm.M = M; prm.H = H; prm.P = P;
   prm.lr = lr; prm.cfg = *cfg;
   prm.X = X; prm.stats = stats; prm.T_out = T_out; prm.b_hist = b_hist; prm.b_dev = b_dev;
+  prm.flag = ctx->flags + 2;
+  prm.drop_copies = ctx->tuning.stats_fault_drop_loads != 0 ? 1 : 0;
+  prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
+  ABS_CUDA_TRY(ctx, cudaMemsetAsync(prm.flag, 0, sizeof(unsigned), static_cast<cudaStream_t>(stream)));
   prm.S = reinterpret_cast<double*>(ws);
   prm.Xpre = reinterpret_cast<float*>(ws + S_bytes);
   ABS_CUDA_TRY(ctx, cudaLaunchKernelEx(&lc, kernel, prm));

@@ -215,6 +215,39 @@ def test_fused_rounds_in_one_launch_equal_one_launch_per_round(ctx):
         params_close(X3, f64(X1), tol=1e-5)
 
 
+def test_fused_rounds_wait_that_runs_out_is_reported_and_the_context_stays_usable(ctx):
+    """Failure detection without a fault: with the partial gradients not sent (test hook) every CTA's
+    wait for its peers gives up after the shortened limit, the launch still reaches all its barriers
+    and ends, the records carry ABS_STATUS_TIMEOUT (so T = 0 and the batch size stays), and the next
+    ordinary call on the same context gives the same result as a context that never timed out."""
+    n, d, M, H, lr, b0, b_max, rounds = 4096, 256, 4, 3, 0.1, 64, 512, 2
+    A, y = inputs.logreg_dataset(1, n, d, device="cuda")
+    idx = inputs.batch_indices(11, (rounds, H, M, b_max), n, device="cuda")
+    tcfg = pkg.make_test_cfg("norm", b_max, eta=0.5)
+
+    def run():
+        X = torch.zeros((M, d), device="cuda")
+        stats = ctx.new_stats(rounds * M)
+        b_dev = torch.tensor([b0], dtype=torch.int64, device="cuda")
+        ctx.abs_logreg_rounds_fused(A, y, idx, X, H, lr, tcfg, stats, b_dev)
+        torch.cuda.synchronize()
+        return X, stats, int(b_dev.item())
+
+    X_ok, stats_ok, b_ok = run()
+    ctx.set_tuning("stats_timeout_cycles", 2_000_000)        # about a millisecond
+    ctx.set_tuning("stats_fault_drop_loads", 1)
+    try:
+        _, flagged, b_flagged = run()
+    finally:
+        ctx.set_tuning("stats_fault_drop_loads", 0)
+        ctx.set_tuning("stats_timeout_cycles", 0)
+    assert all(r["status"] & pkg.binding.STATUS_TIMEOUT for r in pkg.stats_to_dicts(flagged))
+    assert b_flagged == b0                                     # flagged records take no decision
+    X_again, stats_again, b_again = run()
+    assert b_again == b_ok and b_ok > b0
+    assert torch.equal(X_again, X_ok) and torch.equal(stats_again, stats_ok)
+
+
 def test_fused_rounds_refuse_shapes_they_do_not_cover(ctx):
     tcfg = pkg.make_test_cfg("norm", 64, eta=0.5)
     b_dev = torch.tensor([4], dtype=torch.int64, device="cuda")
