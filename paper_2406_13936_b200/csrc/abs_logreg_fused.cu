@@ -43,8 +43,6 @@ namespace cg = cooperative_groups;
 namespace absk {
 namespace {
 
-constexpr int kFW = 8;                     // warps per CTA
-constexpr int kFThreads = kFW * 32;
 constexpr int kMaxWorkersFused = 64;
 constexpr int kMaxDimFused = 1024;
 constexpr int kMaxCtasPerWorker = 16;        // = the largest cluster (16 needs the non-portable opt-in)
@@ -92,23 +90,25 @@ __device__ __forceinline__ float residual(float z, float label) {
 __device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 
 // KV: 16-byte column vectors per lane (slot k of a lane is vector k*32 + lane of the row).
-template <int KV>
-__global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const FusedParams prm) {
-  constexpr int U = 16 / KV;               // samples a warp keeps in flight (16 row vectors in registers)
+// NW: warps per CTA (16 for narrow rows, where a warp's registers allow it: fewer samples per warp).
+template <int KV, int NW>
+__global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedParams prm) {
+  constexpr int NT = NW * 32;
+  constexpr int U = (NW > 8 ? 8 : 16) / KV;   // samples a warp keeps in flight (8 or 16 row vectors in registers)
   cg::grid_group grid = cg::this_grid();
   extern __shared__ __align__(16) float smem_f[];
   const int d = prm.d, DV = d >> 2;
   float4* x4 = reinterpret_cast<float4*>(smem_f);              // [DV] parameters of this worker
   float4* g4 = x4 + DV;                                         // [DV] batch gradient of the step
-  float4* wacc4 = g4 + DV;                                      // [kFW][DV] per-warp partial sums
-  float4* inbox4 = wacc4 + kFW * DV;                            // [2][P][DV] the partial batch gradients of all
+  float4* wacc4 = g4 + DV;                                      // [NW][DV] per-warp partial sums
+  float4* inbox4 = wacc4 + NW * DV;                            // [2][P][DV] the partial batch gradients of all
                                                                 // CTAs of the cluster, written by their owners
   float4* outbox4 = inbox4 + 2 * prm.P * DV;                    // [2][DV] this CTA's partial, source of the copies
   __shared__ __align__(8) unsigned long long xbar[2];           // "all partials of the step have arrived"
   __shared__ unsigned abort_s;
   volatile unsigned* abort_flag = &abort_s;
   const uint32_t xbar_u32 = smem_u32(xbar);
-  __shared__ double red[kFW][3];
+  __shared__ double red[NW][3];
   __shared__ double N_s;
   __shared__ long long T_s[kMaxWorkersFused];
   __shared__ long long b_s;
@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
   float4* Xpre4 = reinterpret_cast<float4*>(prm.Xpre);
   const float lr = prm.lr;
 
-  for (int j = tid; j < DV; j += kFThreads) x4[j] = X4[static_cast<long long>(m) * DV + j];
+  for (int j = tid; j < DV; j += NT) x4[j] = X4[static_cast<long long>(m) * DV + j];
   long long b = prm.b_dev[0];
   if (b > prm.cfg.b_max) b = prm.cfg.b_max;
   if (b < 2) b = 2;                        // the variance needs two rows
@@ -135,13 +135,13 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
   }
   cg::this_cluster().sync();               // every CTA's barriers exist before a peer signals them
 
-  // Sample i of a step belongs to CTA i % P and there to warp (i / P) % 8.  The row index of the
+  // Sample i of a step belongs to CTA i % P and there to warp (i / P) % NW.  The row index of the
   // warp's t-th sample is fetched by lane t % 32 ahead of the loop over the samples; for the
   // first 32 samples of a warp (all of them unless b > 256 P) that load is issued a whole local
   // step earlier, and the rows themselves are prefetched before the grid barrier, so that after
   // the barrier nothing waits for memory that does not depend on the new parameters.
   const long long first = p + static_cast<long long>(P) * warp;     // this warp's first sample
-  const long long hop = static_cast<long long>(P) * kFW;
+  const long long hop = static_cast<long long>(P) * NW;
   auto clamp_row = [&](int raw) -> long long {                       // indices outside the data are clamped
     return raw < 0 ? 0 : (raw >= prm.n ? prm.n - 1 : static_cast<long long>(raw));
   };
@@ -243,10 +243,10 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
       const uint32_t par = static_cast<uint32_t>(gstep & 1);
       const uint32_t bytes = static_cast<uint32_t>(DV) * 16u;
       if (p < Pa) {
-        for (int j = tid; j < DV; j += kFThreads) {
+        for (int j = tid; j < DV; j += NT) {
           float4 s = wacc4[j];
 #pragma unroll
-          for (int w = 1; w < kFW; ++w) {
+          for (int w = 1; w < NW; ++w) {
             const float4 v = wacc4[w * DV + j];
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
           }
@@ -274,7 +274,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
       // The P partials are split over thread groups (group q takes partials q, q + groups, ...),
       // then the groups' sums are added in group order.
       {
-        const int groups = kFThreads / DV >= kFW ? kFW : (kFThreads / DV > 0 ? kFThreads / DV : 1);   // wacc4 has kFW rows
+        const int groups = NT / DV >= NW ? NW : (NT / DV > 0 ? NT / DV : 1);   // wacc4 has NW rows
         const int grp = tid / DV, j = tid - grp * DV;
         if (grp < groups) {
           float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
           wacc4[grp * DV + j] = s;
         }
         __syncthreads();
-        for (int jj = tid; jj < DV; jj += kFThreads) {
+        for (int jj = tid; jj < DV; jj += NT) {
           float4 s = wacc4[jj];
           for (int q = 1; q < groups; ++q) {
             const float4 v = wacc4[q * DV + jj];
@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
       __syncthreads();
       if (tid == 0 && p < Pa) {
         double a0 = 0.0, a1 = 0.0, a2 = 0.0;
-        for (int w = 0; w < kFW; ++w) {
+        for (int w = 0; w < NW; ++w) {
           a0 += red[w][0];
           a1 += red[w][1];
           a2 += red[w][2];
@@ -404,7 +404,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
         __stcg(dst + 3, N_s);
       }
       // the step that was held back, and this worker's parameters for the averaging
-      for (int j = tid; j < DV; j += kFThreads) {
+      for (int j = tid; j < DV; j += NT) {
         const float4 s = g4[j];
         float4 xv = x4[j];
         xv.x = fmaf(-lr, s.x, xv.x); xv.y = fmaf(-lr, s.y, xv.y);
@@ -421,7 +421,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
       // they are spread over the threads and issued together: the records by one warp per worker
       // (lane q reads the sums of CTA q; the shuffle tree adds them in a fixed order), the
       // parameters by thread groups that split the workers and are added in group order.
-      for (int w = warp; w < M; w += kFW) {
+      for (int w = warp; w < M; w += NW) {
         double a0 = 0.0, a1 = 0.0, a2 = 0.0, nn = 0.0;
         if (lane < Pa) {
           const double* src = prm.S + (static_cast<long long>(w) * P + lane) * 4;
@@ -446,7 +446,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
       }
       {
         const float inv_M = 1.0f / static_cast<float>(M);
-        const int groups = kFThreads / DV >= kFW ? kFW : (kFThreads / DV > 0 ? kFThreads / DV : 1);
+        const int groups = NT / DV >= NW ? NW : (NT / DV > 0 ? NT / DV : 1);
         const int grp = tid / DV, j = tid - grp * DV;
         if (grp < groups) {
           float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -458,7 +458,7 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
           wacc4[grp * DV + j] = s;
         }
         __syncthreads();
-        for (int jj = tid; jj < DV; jj += kFThreads) {
+        for (int jj = tid; jj < DV; jj += NT) {
           float4 s = wacc4[jj];
           for (int q = 1; q < groups; ++q) {
             const float4 v = wacc4[q * DV + jj];
@@ -485,11 +485,15 @@ __global__ void __launch_bounds__(kFThreads, 1) logreg_rounds_kernel(const Fused
 }
 
 using KernelFn = void (*)(const FusedParams);
-KernelFn pick_kernel(int DV) {
-  if (DV <= 32) return logreg_rounds_kernel<1>;
-  if (DV <= 64) return logreg_rounds_kernel<2>;
-  if (DV <= 128) return logreg_rounds_kernel<4>;
-  return logreg_rounds_kernel<8>;
+struct KernelChoice {
+  KernelFn fn;
+  int warps;
+};
+KernelChoice pick_kernel(int DV) {
+  if (DV <= 32) return {logreg_rounds_kernel<1, 16>, 16};
+  if (DV <= 64) return {logreg_rounds_kernel<2, 16>, 16};
+  if (DV <= 128) return {logreg_rounds_kernel<4, 8>, 8};
+  return {logreg_rounds_kernel<8, 8>, 8};
 }
 
 }  // namespace
@@ -531,8 +535,9 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
   } restore{prev, ctx->device};
 
   const int DV = static_cast<int>(d / 4);
-  KernelFn kernel = pick_kernel(DV);
-  const size_t smem_fixed = static_cast<size_t>(2 + kFW + 2) * d * sizeof(float);   // + 2 P d floats of inboxes
+  const KernelChoice choice = pick_kernel(DV);
+  KernelFn kernel = choice.fn;
+  const size_t smem_fixed = static_cast<size_t>(2 + choice.warps + 2) * d * sizeof(float);   // + 2 P d floats of inboxes
 
   // One cluster per worker: the largest cluster size that leaves all M clusters co-resident.
   cudaLaunchConfig_t lc = {};
@@ -540,7 +545,7 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
   attrs[0].id = cudaLaunchAttributeClusterDimension;
   attrs[1].id = cudaLaunchAttributeCooperative;
   attrs[1].val.cooperative = 1;
-  lc.blockDim = dim3(kFThreads);
+  lc.blockDim = dim3(static_cast<unsigned>(choice.warps * 32));
   lc.stream = static_cast<cudaStream_t>(stream);
   lc.attrs = attrs;
   lc.numAttrs = 2;
