@@ -353,6 +353,7 @@ PROFILE_CASES = {
     "stats_bf16_b128": dict(kind="stats", M=1, b=128, d=4_000_000, dtype="bf16"),
     "stats_bf16_b256": dict(kind="stats", M=1, b=256, d=2_000_000, dtype="bf16"),
     "adamw": dict(kind="adamw", M=8, d=8_000_000),
+    "logreg_fused": dict(kind="logreg_fused"),          # the 50 rounds of the logistic configuration, fused
     # full-size cases of the sweep, for timing only (not for multi-pass captures)
     "stats_f32_b64_d11m": dict(kind="stats", M=1, b=64, d=11_200_000, dtype="f32"),
     "stats_f32_b256_d11m": dict(kind="stats", M=1, b=256, d=11_200_000, dtype="f32"),
@@ -378,6 +379,10 @@ def run_profile_case(args):
         key, val = kv.split("=")
         ctx.set_tuning(key, int(val))
     peak, _ = measured_peak()
+    if case["kind"] == "logreg_fused":
+        print(json.dumps(dict(case=args.case, **logreg_rounds_fused(torch, pkg, inputs, ctx))))
+        ctx.close()
+        return
     if case["kind"] == "stats":
         M, b, d = case["M"], case["b"], case["d"]
         if case["dtype"] == "f32":
