@@ -261,7 +261,10 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
         del G
         torch.cuda.empty_cache()
     out["rounds_logreg"] = end_to_end_rounds(torch, pkg, inputs, ctx, "logreg")
-    out["rounds_logreg_fused"] = logreg_rounds_fused(torch, pkg, inputs, ctx)
+    try:
+        out["rounds_logreg_fused"] = logreg_rounds_fused(torch, pkg, inputs, ctx)
+    except pkg.AbsError as e:      # e.g. a tool that refuses cooperative cluster launches
+        out["rounds_logreg_fused"] = dict(unavailable=str(e))
     out["rounds_mlp"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp")
     out["rounds_mlp_fused_stats"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp_fused")
     return out
