@@ -82,8 +82,9 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_timeout_cycles" (SM clock cycles a wait for a tile copy may last before
  * the record is flagged ABS_STATUS_TIMEOUT; default about two seconds),
  * "stats_fault_drop_loads" (fault injection for tests: the loaders of the tiled
- * and of the tcgen05 kernel issue no copies, so every wait runs out and the
- * records come back flagged ABS_STATUS_TIMEOUT; nothing traps or hangs),
+ * and of the tcgen05 kernel issue no copies, and abs_logreg_rounds_fused sends no
+ * partial gradients, so every wait runs out and the records come back flagged
+ * ABS_STATUS_TIMEOUT; nothing traps or hangs),
  * "stats_cluster_rows" (target rows per CTA of the cluster kernel, 16..512),
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
  * cluster when b > 256),
@@ -336,7 +337,14 @@ int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, long long n, 
  *   size after the last round on exit.
  * Needs d <= 1024, d % 4 == 0, M <= 64 and 16-byte aligned A and X, else
  * ABS_ERR_UNSUPPORTED; scratch comes from the context's workspace
- * (ABS_ERR_WORKSPACE if it is too small).  Only enqueues.                          */
+ * (ABS_ERR_WORKSPACE if it is too small).  Each worker is one thread-block cluster
+ * and the launch is cooperative (all CTAs resident); ABS_ERR_UNSUPPORTED if the
+ * device cannot hold M clusters at once, ABS_ERR_CUDA if it refuses the launch.
+ * The CTAs of a cluster wait for one another's partial gradients with the limit of
+ * the "stats_timeout_cycles" tuning key; a wait that runs out never hangs the
+ * launch: the records of that round and of the following ones carry
+ * ABS_STATUS_TIMEOUT, which gives T = 0, and the parameters are then not to be
+ * used.  Only enqueues.                                                            */
 int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
                             const int* idx, long long idx_stride, int rounds, float* X, int M, int H,
                             float lr, const abs_test_cfg* cfg, abs_stats* stats, long long* T_out,
