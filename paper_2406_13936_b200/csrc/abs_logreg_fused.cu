@@ -137,9 +137,8 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
 
   // Sample i of a step belongs to CTA i % P and there to warp (i / P) % NW.  The row index of the
   // warp's t-th sample is fetched by lane t % 32 ahead of the loop over the samples; for the
-  // first 32 samples of a warp (all of them unless b > 256 P) that load is issued a whole local
-  // step earlier, and the rows themselves are prefetched before the grid barrier, so that after
-  // the barrier nothing waits for memory that does not depend on the new parameters.
+  // first 32 samples of a warp (all of them unless b > 32 NW P) that load is issued a whole local
+  // step earlier, and the rows themselves are prefetched before the partials are exchanged.
   const long long first = p + static_cast<long long>(P) * warp;     // this warp's first sample
   const long long hop = static_cast<long long>(P) * NW;
   auto clamp_row = [&](int raw) -> long long {                       // indices outside the data are clamped
