@@ -103,8 +103,10 @@ extern "C" int abs_create(abs_ctx** out, int device, size_t workspace_bytes) {
   ctx->workspace_bytes = workspace_bytes ? workspace_bytes : kDefaultWorkspace;
   DeviceScope scope(device);
   cudaError_t e = scope.ok ? cudaMalloc(&ctx->workspace, ctx->workspace_bytes) : cudaErrorInvalidDevice;
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->flags), 64 * sizeof(unsigned));
-  if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, 64 * sizeof(unsigned));
+  const size_t flag_bytes = static_cast<size_t>(kFlagWords + kTicketWords) * sizeof(unsigned);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->flags), flag_bytes);
+  if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, flag_bytes);
+  if (e == cudaSuccess) ctx->ticket_slots = kTicketWords;
   if (e != cudaSuccess) {
     set_error(nullptr, ABS_ERR_CUDA, "allocating the context failed: %s", cudaGetErrorString(e));
     if (ctx->workspace) cudaFree(ctx->workspace);

@@ -14,6 +14,8 @@ namespace absk {
 
 constexpr int kSmCountFallback = 148;
 constexpr size_t kDefaultWorkspace = 64ull << 20;
+constexpr int kFlagWords = 64;                              // flag words at the head of abs_ctx::flags
+constexpr int kTicketWords = 4096;                          // per-worker ticket counters that follow them
 constexpr int kMaxFastRows = 4096;                          // largest b the tiled and cluster kernels cover
 constexpr long long kDefaultTimeoutCycles = 4000000000ll;   // about two seconds of SM clock
 
@@ -41,7 +43,9 @@ struct abs_ctx {
   size_t smem_optin = 0;
   void* workspace = nullptr;       // device
   size_t workspace_bytes = 0;
-  unsigned* flags = nullptr;       // device, 64 words: [0] async-copy timeout flag
+  unsigned* flags = nullptr;       // device, 64 words: [0] async-copy timeout flag; then ticket_slots
+                                   // zeroed words, one per worker, for the split finalisation
+  int ticket_slots = 0;
   void* staging = nullptr;         // device buffer for *_host calls, grown on demand
   size_t staging_bytes = 0;
   void* staging_out = nullptr;     // device buffer for stats / gbar of *_host calls

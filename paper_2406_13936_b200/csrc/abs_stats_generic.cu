@@ -127,37 +127,60 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
   }
 }
 
-// One CTA per worker folds the P partial records in a fixed order and writes abs_stats.
+// Folds the P partial records of every worker in a fixed order and writes abs_stats.  Grid
+// (M, nb): the rows of a worker are split over nb CTAs (one when b < 128), because a single CTA
+// that reads P x b sums is slow for large batches (64 us at b = 1024, P = 132).  CTA y sums e_r
+// over the records for its rows and leaves sum e, sum e^2 (CTA 0 also V and N) in the first words
+// of its own rows of record 0 - rows no other CTA reads; the worker's last CTA to arrive (ticket
+// counter) adds the nb pairs in the order of y and writes the record, so the result does not
+// depend on which CTA that is.
 constexpr int kFinalThreads = 1024;
+constexpr int kFinalMaxSplit = 16;
+constexpr int kFinalRowsPerCta = 64;      // at least this many rows per CTA (>= 4: the words it borrows)
 
 __global__ void __launch_bounds__(kFinalThreads)
-abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, unsigned* __restrict__ flags,
-                          abs_stats* __restrict__ stats_out) {
+abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__ flags,
+                          unsigned* __restrict__ tickets, abs_stats* __restrict__ stats_out) {
   __shared__ double red[4][kFinalThreads / 32];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int m = blockIdx.x;
+  const int m = blockIdx.x, y = blockIdx.y, nb = gridDim.y;
   const size_t rec = static_cast<size_t>(b) + 2;
-  const double* base = ws + static_cast<size_t>(m) * P * rec;
+  double* base = ws + static_cast<size_t>(m) * P * rec;
+  const long long rows_per = (b + nb - 1) / nb;
+  const long long r_begin = y * rows_per;
+  const long long r_end = r_begin + rows_per < b ? r_begin + rows_per : b;
   pdl_wait();                    // the statistics kernel's partial records
   pdl_launch_dependents();
 
-  // Rows are spread over the threads; when b < 1024 several threads share a row and split the P
-  // records between them (record p goes to thread group p mod tpr), then the groups' sums are
-  // added in group order: the order of additions is fixed, the loads run in parallel.
+  // Rows are spread over the threads; when the CTA has fewer than 1024 rows several threads share
+  // a row and split the P records between them (record p goes to thread group p mod tpr), then
+  // the groups' sums are added in group order: the order of additions is fixed, the loads run in
+  // parallel.
   __shared__ double esum[kFinalThreads];
   int rb = 1;
-  while (rb < kFinalThreads && rb < b) rb <<= 1;          // rows handled per pass (power of two)
+  while (rb < kFinalThreads && rb < r_end - r_begin) rb <<= 1;   // rows handled per pass (power of two)
   const int tpr = kFinalThreads / rb;                     // threads per row
   const int col = tid & (rb - 1), grp = tid / rb;
   double se = 0.0, see = 0.0;
-  for (long long r0 = 0; r0 < b; r0 += rb) {
+  for (long long r0 = r_begin; r0 < r_end; r0 += rb) {
     const long long r = r0 + col;
     double e = 0.0;
-    if (r < b)
-      for (int p = grp; p < P; p += tpr) e += base[p * rec + r];
+    if (r < r_end) {
+      // eight loads are issued before the first sum needs one (a load per iteration would cost a
+      // round trip to L2 each); the sums are still taken in the order of p
+      int p = grp;
+      for (; p + 7 * tpr < P; p += 8 * tpr) {
+        double v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = base[static_cast<size_t>(p + u * tpr) * rec + r];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) e += v[u];
+      }
+      for (; p < P; p += tpr) e += base[static_cast<size_t>(p) * rec + r];
+    }
     esum[tid] = e;
     __syncthreads();
-    if (grp == 0 && r < b) {
+    if (grp == 0 && r < r_end) {
       double tot = 0.0;
       for (int g2 = 0; g2 < tpr; ++g2) tot += esum[g2 * rb + col];
       se += tot;
@@ -165,11 +188,13 @@ abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, uns
     }
     __syncthreads();
   }
-  // V and N: thread t takes the records p = t, t + 1024, ...
+  // V and N (CTA 0 of the worker): thread t takes the records p = t, t + 1024, ...
   double vn = 0.0, nn = 0.0;
-  for (int p = tid; p < P; p += kFinalThreads) {
-    vn += base[p * rec + b];
-    nn += base[p * rec + b + 1];
+  if (y == 0) {
+    for (int p = tid; p < P; p += kFinalThreads) {
+      vn += base[p * rec + b];
+      nn += base[p * rec + b + 1];
+    }
   }
   const double a0 = warp_sum_d(se), a1 = warp_sum_d(see), a2 = warp_sum_d(vn), a3 = warp_sum_d(nn);
   if (lane == 0) {
@@ -187,9 +212,31 @@ abs_stats_finalize_kernel(const double* __restrict__ ws, long long b, int P, uns
       V += red[2][w];
       N += red[3][w];
     }
+    if (nb > 1) {
+      // every read of this CTA's rows is done (the barriers above): borrow their first words
+      double* mine = base + r_begin;
+      __stcg(mine + 0, s_e);
+      __stcg(mine + 1, s_ee);
+      if (y == 0) {
+        __stcg(mine + 2, V);
+        __stcg(mine + 3, N);
+      }
+      __threadfence();
+      if (atomicAdd(tickets + m, 1u) != static_cast<unsigned>(nb - 1)) return;   // not the worker's last CTA
+      __threadfence();
+      tickets[m] = 0u;                                   // for the next call
+      s_e = 0.0;
+      s_ee = 0.0;
+      for (int y2 = 0; y2 < nb; ++y2) {
+        s_e += __ldcg(base + y2 * rows_per + 0);
+        s_ee += __ldcg(base + y2 * rows_per + 1);
+      }
+      V = __ldcg(base + 2);
+      N = __ldcg(base + 3);
+    }
     const bool timed_out = *reinterpret_cast<volatile unsigned*>(flags) != 0u;
-    // The last worker's block to get here clears the time-out flag (flags[0]) and the arrival
-    // counter (flags[1]) for the next call, which saves a memset per call.
+    // The last worker to get here clears the time-out flag (flags[0]) and the arrival counter
+    // (flags[1]) for the next call, which saves a memset per call.
     __threadfence();
     if (atomicAdd(flags + 1, 1u) == gridDim.x - 1) {
       flags[0] = 0u;
@@ -234,8 +281,13 @@ int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
 }
 
 int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P) {
-  ABS_CUDA_TRY(ctx, launch_dependent(abs_stats_finalize_kernel, dim3(a.M), dim3(kFinalThreads), 0, a.stream,
-                                     static_cast<const double*>(ctx->workspace), a.b, P, ctx->flags, a.stats_out));
+  // the rows of a worker are split over several CTAs when the context has a ticket word per worker
+  long long nb = a.M <= ctx->ticket_slots ? a.b / kFinalRowsPerCta : 1;
+  nb = nb < 1 ? 1 : (nb > kFinalMaxSplit ? kFinalMaxSplit : nb);
+  while (nb > 1 && (nb - 1) * ((a.b + nb - 1) / nb) + 4 > a.b) --nb;     // the last CTA keeps at least 4 rows
+  ABS_CUDA_TRY(ctx, launch_dependent(abs_stats_finalize_kernel, dim3(a.M, static_cast<unsigned>(nb)),
+                                     dim3(kFinalThreads), 0, a.stream, static_cast<double*>(ctx->workspace), a.b, P,
+                                     ctx->flags, ctx->flags + kFlagWords, a.stats_out));
   return ABS_OK;
 }
 
