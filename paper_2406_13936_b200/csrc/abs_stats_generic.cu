@@ -129,7 +129,7 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
 
 // Folds the P partial records of every worker in a fixed order and writes abs_stats.  Grid
 // (M, nb): the rows of a worker are split over nb CTAs (one when b < 128), because a single CTA
-// that reads P x b sums is slow for large batches (64 us at b = 1024, P = 132).  CTA y sums e_r
+// that reads P x b sums takes long for large batches.  CTA y sums e_r
 // over the records for its rows and leaves sum e, sum e^2 (CTA 0 also V and N) in the first words
 // of its own rows of record 0 - rows no other CTA reads; the worker's last CTA to arrive (ticket
 // counter) adds the nb pairs in the order of y and writes the record, so the result does not
@@ -151,6 +151,15 @@ abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__
   const long long r_end = r_begin + rows_per < b ? r_begin + rows_per : b;
   pdl_wait();                    // the statistics kernel's partial records
   pdl_launch_dependents();
+  // Loads whose values are only needed at the end are issued here, so that they are in flight
+  // while the rows are summed: the time-out flag, and the first V and N of every thread.
+  unsigned timeout_word = 0u;
+  if (tid == 0) timeout_word = *reinterpret_cast<volatile unsigned*>(flags);
+  double vn = 0.0, nn = 0.0;
+  if (y == 0 && tid < P) {
+    vn = base[tid * rec + b];
+    nn = base[tid * rec + b + 1];
+  }
 
   // Rows are spread over the threads; when the CTA has fewer than 1024 rows several threads share
   // a row and split the P records between them (record p goes to thread group p mod tpr), then
@@ -189,9 +198,8 @@ abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__
     __syncthreads();
   }
   // V and N (CTA 0 of the worker): thread t takes the records p = t, t + 1024, ...
-  double vn = 0.0, nn = 0.0;
   if (y == 0) {
-    for (int p = tid; p < P; p += kFinalThreads) {
+    for (int p = tid + kFinalThreads; p < P; p += kFinalThreads) {
       vn += base[p * rec + b];
       nn += base[p * rec + b + 1];
     }
@@ -204,14 +212,11 @@ abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__
     red[3][warp] = a3;
   }
   __syncthreads();
+  if (warp != 0) return;
+  // one value per warp and 32 warps: the first warp adds them with the same shuffle tree
+  double s_e = warp_sum_d(red[0][lane]), s_ee = warp_sum_d(red[1][lane]);
+  double V = warp_sum_d(red[2][lane]), N = warp_sum_d(red[3][lane]);
   if (tid == 0) {
-    double s_e = 0.0, s_ee = 0.0, V = 0.0, N = 0.0;
-    for (int w = 0; w < kFinalThreads / 32; ++w) {
-      s_e += red[0][w];
-      s_ee += red[1][w];
-      V += red[2][w];
-      N += red[3][w];
-    }
     if (nb > 1) {
       // every read of this CTA's rows is done (the barriers above): borrow their first words
       double* mine = base + r_begin;
@@ -225,16 +230,23 @@ abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__
       if (atomicAdd(tickets + m, 1u) != static_cast<unsigned>(nb - 1)) return;   // not the worker's last CTA
       __threadfence();
       tickets[m] = 0u;                                   // for the next call
-      s_e = 0.0;
-      s_ee = 0.0;
-      for (int y2 = 0; y2 < nb; ++y2) {
-        s_e += __ldcg(base + y2 * rows_per + 0);
-        s_ee += __ldcg(base + y2 * rows_per + 1);
+      double pe[kFinalMaxSplit], pee[kFinalMaxSplit];
+#pragma unroll
+      for (int y2 = 0; y2 < kFinalMaxSplit; ++y2) {       // all loads first, then the sums in CTA order
+        pe[y2] = y2 < nb ? __ldcg(base + y2 * rows_per + 0) : 0.0;
+        pee[y2] = y2 < nb ? __ldcg(base + y2 * rows_per + 1) : 0.0;
       }
       V = __ldcg(base + 2);
       N = __ldcg(base + 3);
+      s_e = 0.0;
+      s_ee = 0.0;
+#pragma unroll
+      for (int y2 = 0; y2 < kFinalMaxSplit; ++y2) {
+        s_e += pe[y2];
+        s_ee += pee[y2];
+      }
     }
-    const bool timed_out = *reinterpret_cast<volatile unsigned*>(flags) != 0u;
+    const bool timed_out = timeout_word != 0u;
     // The last worker to get here clears the time-out flag (flags[0]) and the arrival counter
     // (flags[1]) for the next call, which saves a memset per call.
     __threadfence();
