@@ -124,6 +124,7 @@ def _ratios(st, kind, cfg):
     (3000, 36, 3, 3, 0.2, "aug_ip", dict(theta=0.5, nu=0.5), 5, 300, 14),  # ragged: d/4 = 9 vectors, odd sizes
     (5000, 1024, 2, 2, 0.05, "norm", dict(eta=0.7), 2, 700, 8),            # widest rows, b from its minimum
     (4096, 128, 40, 1, 0.1, "norm", dict(eta=0.4), 3, 64, 6),              # many workers: few CTAs per worker
+    (2000, 384, 2, 2, 0.05, "norm", dict(eta=0.6), 4, 200, 6),             # four 16-byte vectors per lane
 ])
 def test_fused_logistic_rounds_teacher_forced(ctx, n, d, M, H, lr, kind, cfg, b, b_max, rounds):
     A, y = inputs.logreg_dataset(1, n, d, device="cuda")
