@@ -19,7 +19,10 @@ pairwise-difference U-statistic forms evaluated in exact rational arithmetic on
 tiny inputs, the b=2 special case, the split Var_norm = Var_ip/N + Var_orth,
 parallel / orthogonal special cases, the chi-square expectations for isotropic
 Gaussian rows, a hand-worked example, torch.optim.SGD / torch.optim.AdamW in
-fp64, and torch.autograd per-sample gradients for the two producer models.
+fp64, and torch.autograd per-sample gradients for the two producer models;
+the round functions (local_round, local_round_per_step, run_until_samples) on
+a one-dimensional quadratic whose batch sizes, test statistics, iterates and
+sample counts are worked by hand.
 
 Parity unpinned (no printed value or independent definition exists in the
 paper): the choice of AdamW variant itself (the paper only cites the optimiser;
@@ -290,7 +293,7 @@ def logreg_per_sample_grads(A, y, x):
     """Per-sample gradients of the logistic loss, rows (sigmoid(a_i^T x) - y_i) a_i.
 
     A [b, d] features, y [b] labels in {0, 1}, x [d] parameters; no bias, no
-    regulariser (Alg. 1, "compute per-sample gradients").
+    regulariser (Alg. 1, per-sample gradient step).
     """
     A = np.asarray(A, dtype=np.float64)
     y = np.asarray(y, dtype=np.float64)
@@ -394,3 +397,88 @@ def local_round(X, per_sample_grads, batches, lr, b_cur, b_max, kind, **cfg):
     X = replica_average(X)
     b_next, T = next_batch(stats, b_cur, b_max, kind, **cfg)
     return X, b_next, T, stats
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 1 as printed: the test after every local step, per worker
+# ----------------------------------------------------------------------------
+def local_round_per_step(X, per_sample_grads, H, lr, b_cur, b_max, kind, shared=False,
+                         eta_per_worker=None, **cfg):
+    """One round of Alg. 1: for every worker m and local step h = 0..H-1
+        sample a batch of the worker's current size b^m_{k,h},
+        per-sample gradients at x^m_{k,h}, their mean (Eq. batch_grad) and variance (Eq. def_var),
+        T^m_{k,h} (the ceiling of Alg. 1; Eq. test_stat),
+        b^m_{k,h+1} = max{T^m_{k,h}, b^m_{k,h}}  (capped at the maximum local batch size),
+        x^m_{k,h+1} = x^m_{k,h} - lr * batch gradient,
+    then the model averaging (Eq. local_sgd_alt, second line).
+
+    X [M, d]; per_sample_grads(m, h, x, b) returns G[b, d] of worker m's batch of size b at step h;
+    b_cur is the list [b^1_{k,0} .. b^M_{k,0}].  With shared=True every worker continues with the
+    maximum over the workers (the practical rule below Eq. test_stat), applied after every step.
+    eta_per_worker gives the constants eta_m of Eq. approx_norm_local.
+    Returns (X_next, b_next [M], b_used [H][M], T [H][M], stats [H][M], samples) where
+    samples = sum_m sum_h b^m_{k,h} is the round's term of the counter B of Alg. 1.
+    """
+    X = np.array(X, dtype=np.float64)
+    M = X.shape[0]
+    b = [int(v) for v in b_cur]
+    if len(b) != M:
+        raise ValueError("one current batch size per worker")
+    b_used, T_hist, stats_hist = [], [], []
+    samples = 0
+    for h in range(H):
+        Gb = np.empty_like(X)
+        stats = [None] * M
+        for m in range(M):
+            G = per_sample_grads(m, h, X[m], b[m])
+            if G.shape[0] != b[m]:
+                raise ValueError("the batch of worker %d at step %d must have %d rows" % (m, h, b[m]))
+            Gb[m] = batch_mean(G)
+            stats[m] = batch_test_stats(G)
+            samples += b[m]
+        b_used.append(list(b))
+        b, T = next_batch_local(stats, b, b_max, kind, eta_per_worker=eta_per_worker, **cfg)
+        if shared:
+            b = [max(b)] * M
+        T_hist.append(T)
+        stats_hist.append(stats)
+        X = sgd_step(X, Gb, lr)
+    X = replica_average(X)
+    return X, b, b_used, T_hist, stats_hist, samples
+
+
+def samples_of_round(H, M, b):
+    """The round's term of the sample counter in Alg. 2: B <- B + H M b_k."""
+    return H * M * b
+
+
+def run_until_samples(X0, per_sample_grads, H, lr, b0, b_max, kind, n_samples, per_step=False,
+                      shared=True, max_rounds=10 ** 6, **cfg):
+    """The outer loop of Alg. 1 / Alg. 2: rounds k = 0, 1, ... while B < N, the counter B growing
+    by the samples each round processed; the output is x_hat = x^1_{K,0}, K the first round count
+    with B >= N.
+
+    per_sample_grads(k, m, h, x, b) returns G[b, d].  per_step=False runs local_round (the test once
+    per round on the last step, B += H M b); per_step=True runs local_round_per_step (B += sum_m
+    sum_h b^m_{k,h}).  Returns (x_hat, K, B, history) with history[k] = the batch sizes round k
+    started with (an int, or a list per worker for per_step).
+    """
+    X = np.array(X0, dtype=np.float64)
+    M = X.shape[0]
+    B, k = 0, 0
+    b = [int(b0)] * M if per_step else int(b0)
+    history = []
+    while B < n_samples and k < max_rounds:
+        history.append(list(b) if per_step else b)
+        if per_step:
+            X, b, _, _, _, used = local_round_per_step(
+                X, lambda m, h, x, bb, k=k: per_sample_grads(k, m, h, x, bb), H, lr, b, b_max, kind,
+                shared=shared, **cfg)
+            B += used
+        else:
+            X, b_next, _, _ = local_round(
+                X, lambda m, h, x, k=k, b=b: per_sample_grads(k, m, h, x, b), H, lr, b, b_max, kind, **cfg)
+            B += samples_of_round(H, M, b)
+            b = b_next
+        k += 1
+    return X[0].copy(), k, B, history

@@ -436,3 +436,64 @@ def test_merged_sub_batches_equal_the_whole_batch(n_a, n_b):
     np.testing.assert_allclose(mean, whole["gbar"], rtol=1e-13, atol=1e-15)
     assert var == pytest.approx(whole["var_norm"], rel=1e-12)
     assert N == pytest.approx(whole["gbar_sq"], rel=1e-12)
+
+
+# ---------------------------------------------------------------- Algorithm 1: the test after every local step
+# f(x; xi) = 0.5 (x - xi)^2 in one dimension: per-sample gradient x - xi, so the batch variance is the
+# sample variance of the xi's and the batch gradient is x - mean(xi).  All numbers below are worked by hand.
+_XI = {(0, 0): [0, 4, 9], (0, 1): [1, 5, 3], (1, 0): [4, 4, 7], (1, 1): [2, 3, 8]}
+
+
+def _toy_grads(m, h, x, b):
+    return x[None, :] - np.array(_XI[(m, h)][:b], dtype=np.float64)[:, None]
+
+
+def test_per_step_round_by_hand_per_worker():
+    # worker 1: step 0, b=2, xi={0,4}: Var=8, gbar=3-2=1, T=ceil(8/(1/4))=32 -> b=min(3,32)=3, x=2.5
+    #           step 1, b=3, xi={1,5,3}: Var=4, gbar=-1/2, T=ceil(4/(1/16))=64, x=2.75
+    # worker 2: step 0, b=2, xi={4,4}: Var=0, gbar=-1, T=0 -> b=2, x=3.5
+    #           step 1, b=2, xi={2,3}: Var=1/2, gbar=1, T=ceil((1/2)/(1/4))=2, x=3
+    X, b, used, T, stats, samples = orc.local_round_per_step(
+        np.array([[3.0], [3.0]]), _toy_grads, 2, 0.5, [2, 2], 3, "norm", eta=0.5)
+    assert used == [[2, 2], [3, 2]] and T == [[32, 0], [64, 2]] and b == [3, 2]
+    assert samples == 2 + 3 + 2 + 2
+    np.testing.assert_allclose(X, [[2.875], [2.875]], rtol=1e-15)
+    assert stats[1][0]["var_norm"] == pytest.approx(4.0, rel=1e-15)
+    assert stats[1][0]["gbar_sq"] == pytest.approx(0.25, rel=1e-15)
+
+
+def test_per_step_round_by_hand_shared_size():
+    # as above, but after step 0 both workers continue with max(3, 2) = 3:
+    # worker 2, step 1, b=3, xi={2,3,8}: mean 13/3, Var=31/3, gbar=3.5-13/3=-5/6, N=25/36,
+    #           T=ceil((31/3)/((1/4)(25/36)))=ceil(59.52)=60, x=3.5+5/12
+    X, b, used, T, _, samples = orc.local_round_per_step(
+        np.array([[3.0], [3.0]]), _toy_grads, 2, 0.5, [2, 2], 3, "norm", shared=True, eta=0.5)
+    assert used == [[2, 2], [3, 3]] and T == [[32, 0], [64, 60]] and b == [3, 3]
+    assert samples == 10
+    np.testing.assert_allclose(X, [[(2.75 + 3.5 + 5.0 / 12.0) / 2.0]] * 2, rtol=1e-15)
+
+
+def test_per_step_round_with_per_worker_constants():
+    # eta_1 = 1 quarters worker 1's ratios (8/1 = 8 -> b=3; 4/(1/4) = 16), eta_2 = 1/4 quadruples worker 2's
+    # (step 1: (1/2)/((1/16) 1) = 8 -> b=min(3,8)=3)
+    _, b, used, T, _, _ = orc.local_round_per_step(
+        np.array([[3.0], [3.0]]), _toy_grads, 2, 0.5, [2, 2], 3, "norm", eta_per_worker=[1.0, 0.25])
+    assert T == [[8, 0], [16, 8]] and used == [[2, 2], [3, 2]] and b == [3, 3]
+
+
+def test_sample_counter_and_stop_rule():
+    # identical samples xi = c: zero variance, T = 0, the batch size never moves; each step contracts
+    # x - c by (1 - lr); Alg. 2 counts H M b samples per round and stops at the first K with B >= N
+    c, x0, lr, H, M, b = 2.0, 10.0, 0.25, 2, 2, 3
+    grads = lambda k, m, h, x, bb: np.tile(x - c, (bb, 1))
+    x_hat, K, B, hist = orc.run_until_samples(np.full((M, 1), x0), grads, H, lr, b, 64, "norm", 50, eta=0.5)
+    assert (K, B) == (5, 60) and hist == [3] * 5          # 12 samples per round: 48 < 50 <= 60
+    assert x_hat[0] == pytest.approx(c + (x0 - c) * (1 - lr) ** (H * K), rel=1e-14)
+    assert orc.samples_of_round(H, M, b) == 12
+    # Alg. 1 counts the sizes actually used: the hand-worked round above uses 9 samples
+    grads1 = lambda k, m, h, x, bb: _toy_grads(m, h, x, bb)
+    for N, K_exp in ((9, 1), (10, 2)):
+        _, K, B, hist = orc.run_until_samples(np.array([[3.0], [3.0]]), grads1, 2, 0.5, 2, 3, "norm", N,
+                                              per_step=True, shared=False, eta=0.5)
+        assert K == K_exp and hist[0] == [2, 2] and (B == 9 if K == 1 else B > 9)
+    assert hist[1] == [3, 2]                               # the second round starts from the sizes the first ended with
