@@ -115,14 +115,83 @@ def cpu_sample(divisor=4):
     return G, x, "first %d of %d columns (1/%d of the workload), all %d rows" % (d, WORKLOAD["d"], divisor, b)
 
 
-def time_cpu_baseline():
+def _limit_blas_threads():
+    """One thread per process: the vector products of the oracle would otherwise be spread over all
+    cores by the BLAS library and the stated core count would be wrong."""
+    try:
+        from threadpoolctl import threadpool_limits
+        return threadpool_limits(limits=1)
+    except Exception:
+        return None
+
+
+_POOL_SHM = None
+
+
+def _pool_attach(name, shape):
+    """Initialiser of an oracle worker process: attaches to the shared sample."""
+    global _POOL_SHM
     import numpy as np
+    from multiprocessing import shared_memory
+    import oracle.abs_oracle  # noqa: F401  (imported before the clock starts)
+    _limit_blas_threads()
+    shm = shared_memory.SharedMemory(name=name)
+    _POOL_SHM = (shm, np.ndarray(shape, dtype=np.float32, buffer=shm.buf))
+
+
+def _pool_block(job):
+    """The whole oracle step on one column block of the shared sample."""
+    import numpy as np
+    lo, hi, b = job
+    if hi <= lo:
+        return 0.0
+    G = _POOL_SHM[1][:, lo:hi]
+    x = np.zeros((1, hi - lo))
+    t0 = time.perf_counter()
+    oracle_step(G, x, np.zeros_like(x), np.zeros_like(x), b, 1)
+    return time.perf_counter() - t0
+
+
+def time_cpu_baseline():
+    """The oracle as it stands on a quarter of the columns: on one core, and with one process per host
+    core, each taking a block of the same columns (the processes are spawned, never forked)."""
+    import multiprocessing as mp
+    import numpy as np
+    from multiprocessing import shared_memory
     G, x, what = cpu_sample()
+    limit = _limit_blas_threads()
     t0 = time.perf_counter()
     oracle_step(G, x, np.zeros_like(x), np.zeros_like(x), WORKLOAD["b"], 1)
     dt = time.perf_counter() - t0
-    return dict(value=G.nbytes / dt / 1e9, unit="GB/s", cores=1, kind="oracle", sample=what,
-                seconds=round(dt, 3))
+    del limit
+    out = dict(value=G.nbytes / dt / 1e9, unit="GB/s", cores=1, kind="oracle", sample=what, seconds=round(dt, 3))
+    cores = os.cpu_count() or 1
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except Exception:
+        pass
+    procs = min(cores, 64)
+    shm = shared_memory.SharedMemory(create=True, size=G.nbytes)
+    try:
+        shared = np.ndarray(G.shape, dtype=np.float32, buffer=shm.buf)
+        shared[:] = G
+        d = G.shape[1]
+        edges = [d * k // procs for k in range(procs + 1)]
+        jobs = [(edges[k], edges[k + 1], WORKLOAD["b"]) for k in range(procs)]
+        with mp.get_context("spawn").Pool(procs, initializer=_pool_attach, initargs=(shm.name, G.shape)) as pool:
+            pool.map(_pool_block, [(0, 1, WORKLOAD["b"])] * procs)        # every process up and attached
+            t0 = time.perf_counter()
+            pool.map(_pool_block, jobs, chunksize=1)
+            dt_all = time.perf_counter() - t0
+        out["all_cores"] = dict(value=G.nbytes / dt_all / 1e9, unit="GB/s", cores=procs, host_cores=cores,
+                                kind="oracle", sample=what + ", one column block per process",
+                                seconds=round(dt_all, 3))
+    except Exception as e:      # a box that cannot spawn processes still reports the single-core figure
+        out["all_cores"] = dict(unavailable=str(e)[:200])
+    finally:
+        shm.close()
+        shm.unlink()
+    return out
 
 
 def run_reference(args):
@@ -179,8 +248,9 @@ def time_steps(torch, fn, steps, warmup):
     return e0.elapsed_time(e1) / 1e3 / steps
 
 
-def extra_legs(torch, pkg, inputs, ctx, peak):
-    """Fused optimiser steps and bf16 statistics on their own workloads (not the headline)."""
+def extra_legs(torch, pkg, inputs, ctx, peak, steps, warmup):
+    """The nine-cell statistics sweep, fused optimiser steps and bf16 statistics on their own workloads
+    (not the headline)."""
     out = {}
     # The short statistics legs come first: run after the long optimiser legs they measured 10-35 %
     # lower (fp32 [1, 4, 124 M]: 4.5 instead of 7.0 TB/s), the long legs themselves do not care.
@@ -207,6 +277,9 @@ def extra_legs(torch, pkg, inputs, ctx, peak):
                                               GBps=gbs, frac_of_peak=gbs / peak)
             del G
             torch.cuda.empty_cache()
+    # the nine cells of the statistics sweep (behind the short legs above, before the long ones below)
+    out["sweep"] = stats_sweep(torch, pkg, inputs, ctx, peak, steps, warmup)
+    out["worst_cell"] = worst_cell(out["sweep"])
     free = torch.cuda.mem_get_info()[0]
     # fused local AdamW + averaging: M=8 fp32 replicas of a GPT-2-small-sized model, H=16 steps per round
     M, d, H = 8, 124_439_808, 16
@@ -407,24 +480,18 @@ def run_profile_case(args):
     ctx.close()
 
 
-def run_sweep(args):
+def stats_sweep(torch, pkg, inputs, ctx, peak, steps, warmup):
     """The statistics sweep: b in {64, 256, 1024} x d in {1 M, 11.2 M, 25.6 M}, fp32, M = 1, each case
     abs_test_stats followed by abs_next_batch for the norm and the augmented inner-product test.
     The variance of the rows does not change what is read, so the sweep runs sigma = 1 only.
-    Inputs under 1 GB rotate over 4 buffers so that L2 does not serve them; one JSON line."""
-    import torch
-    import paper_2406_13936_b200 as pkg
-    from paper_2406_13936_b200 import inputs
-    pkg.build.build()
-    ctx = pkg.Context(0)
-    peak, peak_kind = measured_peak()
+    Inputs under 1 GB rotate over 4 buffers so that L2 does not serve them.  Returns the nine cells."""
     cfgs = [pkg.make_test_cfg("norm", 1 << 20, eta=0.5), pkg.make_test_cfg("aug_ip", 1 << 20, theta=0.5, nu=0.5)]
     table = []
     for b in (64, 256, 1024):
         for d in (1_000_000, 11_200_000, 25_600_000):
             nbytes = 4 * b * d
             if nbytes + (8 << 30) > torch.cuda.mem_get_info()[0]:
-                table.append(dict(b=b, d=d, note="does not fit on this device"))
+                table.append(dict(b=b, d=d, GB=nbytes / 1e9, note="does not fit on this device"))
                 continue
             copies = 4 if nbytes < (1 << 30) else 1
             Gs = [inputs.gaussian_rows(2 + k, 1, b, d, 1.0, device="cuda") for k in range(copies)]
@@ -437,14 +504,39 @@ def run_sweep(args):
                 for cfg in cfgs:
                     ctx.abs_next_batch(stats, cfg, b_cur, b_next)
 
-            sec = time_steps(torch, step, args.steps, args.warmup)
+            n = steps if nbytes < (20 << 30) else max(5, steps // 4)
+            sec = time_steps(torch, step, n, warmup)
             table.append(dict(b=b, d=d, GB=nbytes / 1e9, ms=sec * 1e3, GBps=nbytes / sec / 1e9,
                               frac_of_peak=nbytes / sec / 1e9 / peak, frac_of_nominal_8TBps=nbytes / sec / 8e12,
-                              buffers=copies, b_next=int(b_next.item())))
+                              buffers=copies, steps=n, b_next=int(b_next.item())))
             del Gs
             torch.cuda.empty_cache()
+    return table
+
+
+def worst_cell(table):
+    timed = [c for c in table if "GBps" in c]
+    if not timed:
+        return None
+    w = min(timed, key=lambda c: c["frac_of_peak"])
+    return dict(b=w["b"], d=w["d"], GBps=w["GBps"], frac=w["frac_of_peak"])
+
+
+def run_sweep(args):
+    """The statistics sweep alone; one JSON line."""
+    import torch
+    import paper_2406_13936_b200 as pkg
+    from paper_2406_13936_b200 import inputs
+    pkg.build.build()
+    ctx = pkg.Context(0)
+    for kv in args.tune:
+        key, val = kv.split("=")
+        ctx.set_tuning(key, int(val))
+    peak, peak_kind = measured_peak()
+    table = stats_sweep(torch, pkg, inputs, ctx, peak, args.steps, args.warmup)
     print(json.dumps(dict(sweep="stats fp32 M=1, abs_test_stats + 2 x abs_next_batch per step", steps=args.steps,
-                          warmup=args.warmup, peak_GBps=peak, peak_kind=peak_kind, cases=table)))
+                          warmup=args.warmup, peak_GBps=peak, peak_kind=peak_kind, cases=table,
+                          worst_cell=worst_cell(table))))
     ctx.close()
 
 
@@ -547,7 +639,7 @@ def run_ours(args):
 
     extra = None
     if rank == 0 and world == 1 and not args.no_extra:
-        extra = extra_legs(torch, pkg, inputs, ctx, peak)
+        extra = extra_legs(torch, pkg, inputs, ctx, peak, args.steps, max(args.warmup, 3))
     cpu = time_cpu_baseline() if (rank == 0 and world == 1) else None
 
     if rank == 0:

@@ -89,6 +89,8 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
  * cluster when b > 256),
  * "stats_no_gram" (1 = do not use the tensor-core Gram kernels for bf16, b <= 256),
+ * "stats_no_recheck" (1 = keep a Gram kernel's record even when its sums are
+ * ill-conditioned, i.e. never recompute it with the tiled kernel),
  * "stats_ctas_per_sm" (1: one CTA per SM, 64 KiB buffers, up to 16 rows per
  * thread; 2: two CTAs per SM, 32 KiB buffers, up to 8 rows per thread).
  * Unknown key or out-of-range value: ABS_ERR_INVALID_ARG. */
@@ -109,7 +111,9 @@ typedef struct {
   double sum_sq;      /* sum_i ||g_i||^2 = (b-1) var_norm + b N                  */
   long long rows;     /* b                                                       */
   unsigned status;    /* ABS_STATUS_* bits                                       */
-  unsigned reserved;  /* zero                                                    */
+  unsigned recomputed;/* 1: the tensor-core Gram kernel's sums were too ill-conditioned
+                         (rows dominated by a common vector) and the record comes
+                         from a second, centred pass over G; else 0              */
 } abs_stats;          /* 56 bytes */
 
 /* Batch-size test statistics of M workers (Eq. def_var applied per worker,
@@ -130,6 +134,14 @@ typedef struct {
  * Accumulation: fp32 within a tile (the Gram kernels: exact bf16 products added
  * in fp32 over at most 8192 columns), fp64 across tiles; the reduction order is
  * fixed, so repeated calls give bit-identical records.
+ * The Gram kernels only see uncentred products, so their variance is a difference
+ * of two sums of size sum_i ||g_i||^2: when b N exceeds a few tens (tcgen05) or a
+ * few thousand (mma.sync) times (b-1) var_norm -- rows dominated by a common
+ * vector -- or N exceeds about 2e5 sqrt(var_ip), the finalisation flags the
+ * result on the device and the tiled kernel, which accumulates centred values,
+ * recomputes it in a second pass (abs_stats.recomputed = 1).  The two guarded
+ * launches are always enqueued and return at once when not needed, so the call
+ * stays free of host synchronisation.
  * Errors: ABS_ERR_INVALID_ARG, ABS_ERR_WORKSPACE, ABS_ERR_CUDA.               */
 int abs_test_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long long b, long long d,
                    long long row_stride, long long worker_stride,
@@ -298,10 +310,45 @@ int local_shb_step(abs_ctx* ctx, float* X, float* Buf, const float* Gb, int M, l
 int replica_average(abs_ctx* ctx, float* X, int M, long long d, long long replica_stride,
                     void* stream);
 
+/* ---- the outer loop: sample counter, stop rule, cadence of the test ---------------------- */
+
+/* The counters of Algorithm 1 / Algorithm 2, kept on the DEVICE so that rounds can follow one
+ * another without a host read-back: B (samples processed), k (rounds completed) and the N of
+ * "while B < N".  The caller allocates it in device memory, initialises it and may copy it back
+ * at any time.  The drivers add, per round, sum_m sum_h b^m_{k,h} (Algorithm 1) -- which is
+ * H M b_k when the size is shared and constant over a round (Algorithm 2) -- and 1 to k.
+ * abs_logreg_rounds_fused_opts also obeys the stop rule on the device: it runs no round once
+ * samples >= n_stop (n_stop <= 0: no stop).  The enqueue-only per-round drivers cannot skip
+ * launches that are already enqueued; their caller reads the block back with the batch size. */
+typedef struct {
+  long long samples;    /* B                                                          */
+  long long rounds;     /* k                                                          */
+  long long n_stop;     /* N; <= 0: never stop                                        */
+  long long reserved;   /* zero                                                       */
+} abs_round_ctl;
+
+/* Cadence and ownership of the batch size (HOST struct, copied at the call).         */
+typedef struct {
+  int test_every_step;  /* 0: the test once per round, on the last local step's gradients
+                           (Section 4.3, last paragraph); 1: after every local step, the
+                           next step already using the new size (Algorithm 1)          */
+  int per_worker;       /* 1: b^m <- max{T^m, b^m} per worker (Eq. test_stat, Algorithm 1);
+                           0: every worker continues with the maximum over the workers
+                           (display below Eq. test_stat)                               */
+  const double* eta_m;  /* DEVICE [M] norm-test constants eta_m (Eq. approx_norm_local), or
+                           NULL: cfg->eta for every worker                             */
+  abs_round_ctl* ctl;   /* DEVICE counter block, or NULL                               */
+} abs_round_opts;
+
+/* samples += times * (sizes[0] + ... + sizes[n-1]);  rounds += add_rounds  -- one tiny launch.
+ * ctl, sizes: device.                                                                */
+int abs_round_count(abs_ctx* ctx, abs_round_ctl* ctl, const long long* sizes, int n, long long times,
+                    long long add_rounds, void* stream);
+
 /* ---- producers and round drivers for the synthetic end-to-end problems ------------------ */
 
-/* Per-sample gradients of the logistic loss (Algorithm 1, "compute per-sample
- * gradients"): row i of worker m is (sigmoid(a^T x^m) - y) a with a = A[idx[m][i]].
+/* Per-sample gradients of the logistic loss (Algorithm 1, per-sample gradient
+ * step): row i of worker m is (sigmoid(a^T x^m) - y) a with a = A[idx[m][i]].
  *   A [n][d] fp32 features, y [n] fp32 labels in {0,1}, idx [M][idx_stride] int32
  *   sample indices (the first b of each row are used), X [M][d] parameters,
  *   G [M][b][d] output (contiguous).                                              */
@@ -317,18 +364,37 @@ int abs_logreg_grads(abs_ctx* ctx, const float* A, const float* y, long long n, 
  *   idx [H][M][idx_stride] int32;  b the current batch size (host value, equal to
  *   *b_dev);  G_scratch [M][b][d], Gb_scratch [M][d], stats [M], T_out [M] or NULL;
  *   b_dev device int64: holds b on entry and the next batch size afterwards.
- * Only enqueues; read b_dev back before sizing the next round.                    */
+ *   ctl device counter block or NULL: B += H M b (Algorithm 2's counter), k += 1.
+ * Only enqueues; read b_dev (and ctl) back before sizing the next round.          */
 int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
                      const int* idx, long long idx_stride, float* X, int M, int H, long long b,
                      float lr, const abs_test_cfg* cfg, float* G_scratch, float* Gb_scratch,
-                     abs_stats* stats, long long* T_out, long long* b_dev, void* stream);
+                     abs_stats* stats, long long* T_out, long long* b_dev, abs_round_ctl* ctl,
+                     void* stream);
+
+/* The same round with the test after every local step (Algorithm 1 as printed): at step h
+ * worker m draws b^m_{k,h} samples, its statistics give T^m_{k,h}, and step h + 1 runs with
+ * b^m_{k,h+1} = min(b_max, max{T^m, b^m}) -- per worker, or the maximum over the workers
+ * for all of them (opts->per_worker).  opts may be NULL (shared size, cfg->eta, no counter).
+ *   b_host  HOST array [M]: the sizes the round starts with; on return the sizes after it
+ *   b_dev   device [M] scratch that holds the same values
+ *   idx [H][M][idx_stride] with idx_stride >= cfg->b_max;  G_scratch room for M * b_max rows
+ *   of d floats;  stats [H][M] and T_out [H][M] (or NULL): the records and T of every step.
+ * The grids of step h + 1 depend on sizes decided on the device in step h, so this call
+ * WAITS for the stream once per local step to read M integers back (the one driver of the
+ * library that synchronises; abs_logreg_rounds_fused_opts does the same work without).   */
+int abs_logreg_round_per_step(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
+                              const int* idx, long long idx_stride, float* X, int M, int H,
+                              long long* b_host, float lr, const abs_test_cfg* cfg,
+                              const abs_round_opts* opts, float* G_scratch, float* Gb_scratch,
+                              abs_stats* stats, long long* T_out, long long* b_dev, void* stream);
 
 /* `rounds` communication rounds of the same method in ONE cooperative launch
  * (Algorithm 2's structure, Algorithm 1's per-sample statistic once per round,
  * Section 4.3; b <- min(b_max, max{b, max_m T_m})): the parameters stay in shared
  * memory, the batch size stays on the device from round to round, the per-sample
- * gradient matrix is never written, and there is one grid-wide barrier per local
- * step.  For small problems, where abs_logreg_round is bound by launch latency.
+ * gradient matrix is never written, and there is one grid-wide barrier per round
+ * (none inside a local step).  For small problems, where abs_logreg_round is bound by launch latency.
  *   idx [rounds][H][M][idx_stride] int32 with idx_stride >= cfg->b_max (indices
  *   outside [0, n) are clamped);  X [M][d] in place (replica stride d);
  *   stats [rounds][M] records of each round's test;  T_out [rounds][M] or NULL;
@@ -350,6 +416,24 @@ int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float* y, long l
                             float lr, const abs_test_cfg* cfg, abs_stats* stats, long long* T_out,
                             long long* b_hist, long long* b_dev, void* stream);
 
+/* The same launch with the cadence, the ownership of the batch size, per-worker constants
+ * and the counters of Algorithm 1 / Algorithm 2 chosen by `opts` (HOST pointer; NULL gives
+ * abs_logreg_rounds_fused).  With opts:
+ *   b_dev   device [M]: every worker's size on entry and after the last round that ran
+ *   test once per round:   stats, T_out [rounds][M];  b_hist [rounds][M] (or NULL): the size
+ *                          each round ran with
+ *   test_every_step:       stats, T_out, b_hist [rounds][H][M]: record, T and the size of
+ *                          every local step (Algorithm 1); one cluster-wide barrier per step
+ *                          more, and a grid-wide one per step when the size is shared
+ *   opts->ctl              B and k are read at the start and written back at the end; no
+ *                          round starts once B >= n_stop (entries of rounds that did not
+ *                          run are left untouched); X holds x_{K,0} of the last round run.  */
+int abs_logreg_rounds_fused_opts(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
+                                 const int* idx, long long idx_stride, int rounds, float* X, int M,
+                                 int H, float lr, const abs_test_cfg* cfg, const abs_round_opts* opts,
+                                 abs_stats* stats, long long* T_out, long long* b_hist,
+                                 long long* b_dev, void* stream);
+
 /* Three-layer ReLU MLP with softmax cross-entropy (the second synthetic problem).
  * dims = {n0, n1, n2, n3} layer widths.  One replica's parameters are a flat fp32
  * vector W1 [n1][n0], b1 [n1], W2 [n2][n1], b2 [n2], W3 [n3][n2], b3 [n3] (each W
@@ -359,7 +443,7 @@ int abs_mlp_param_count(const int* dims, long long* out);
 int abs_mlp_scratch_bytes(int M, long long b, const int* dims, size_t* out);
 
 /* Forward and backward pass of all M workers on their batches (Algorithm 2,
- * "compute the local batch gradient"): writes the batch gradients Gb [M][d] and
+ * local batch gradient step): writes the batch gradients Gb [M][d] and
  * leaves activations and deltas in `scratch` (device, caller-owned) for
  * abs_mlp_per_sample.  inputs [n][n0] fp32, labels [n] int32, idx [M][idx_stride]
  * int32 sample indices (first b used), X [M][d] parameters (replica stride d).     */
@@ -370,7 +454,7 @@ int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* labels, long lon
 /* Per-sample gradients of one worker as rows G [b][row_stride] (row_stride >= d; a
  * multiple of 4 keeps the rows 16-byte aligned for the fast statistics kernels),
  * from the scratch a preceding abs_mlp_grads call with the same b filled
- * (Algorithm 1, "compute per-sample gradients").  b <= 65535.                       */
+ * (Algorithm 1, per-sample gradient step).  b <= 65535.                       */
 int abs_mlp_per_sample(abs_ctx* ctx, const int* dims, long long b, int worker, const void* scratch,
                        float* G, long long row_stride, void* stream);
 
@@ -393,7 +477,17 @@ int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* labels, long lon
                   const int* idx, long long idx_stride, float* X, int M, int H, long long b, float lr,
                   const abs_test_cfg* cfg, void* scratch, size_t scratch_bytes, float* G_scratch,
                   long long g_row_stride, float* Gb_scratch, abs_stats* stats, long long* T_out,
-                  long long* b_dev, void* stream);
+                  long long* b_dev, abs_round_ctl* ctl, void* stream);
+
+/* The MLP round with the test after every local step, as abs_logreg_round_per_step; the
+ * statistics of every step come from abs_mlp_fused_stats.  scratch must hold M workers at
+ * b_max (abs_mlp_scratch_bytes).  Waits for the stream once per local step.              */
+int abs_mlp_round_per_step(abs_ctx* ctx, const float* inputs, const int* labels, long long n,
+                           const int* dims, const int* idx, long long idx_stride, float* X, int M,
+                           int H, long long* b_host, float lr, const abs_test_cfg* cfg,
+                           const abs_round_opts* opts, void* scratch, size_t scratch_bytes,
+                           float* Gb_scratch, abs_stats* stats, long long* T_out, long long* b_dev,
+                           void* stream);
 
 #ifdef __cplusplus
 }

@@ -37,7 +37,17 @@ class AdamWCfg(ctypes.Structure):
 class Stats(ctypes.Structure):
     _fields_ = [("gbar_sq", ctypes.c_double), ("var_norm", ctypes.c_double), ("var_ip", ctypes.c_double),
                 ("var_orth", ctypes.c_double), ("sum_sq", ctypes.c_double), ("rows", ctypes.c_longlong),
-                ("status", ctypes.c_uint), ("reserved", ctypes.c_uint)]
+                ("status", ctypes.c_uint), ("recomputed", ctypes.c_uint)]
+
+
+class RoundCtl(ctypes.Structure):
+    _fields_ = [("samples", ctypes.c_longlong), ("rounds", ctypes.c_longlong), ("n_stop", ctypes.c_longlong),
+                ("reserved", ctypes.c_longlong)]
+
+
+class RoundOpts(ctypes.Structure):
+    _fields_ = [("test_every_step", ctypes.c_int), ("per_worker", ctypes.c_int), ("eta_m", ctypes.c_void_p),
+                ("ctl", ctypes.c_void_p)]
 
 
 class StatsPlan(ctypes.Structure):
@@ -70,11 +80,28 @@ EXPORTS = {
     "abs_logreg_round": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_longlong,
                          ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                          ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p, ctypes.c_void_p,
-                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "abs_logreg_rounds_fused": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
                                 ctypes.c_longlong, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_void_p,
                                 ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p,
                                 ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_logreg_rounds_fused_opts": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
+                                     ctypes.c_longlong, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_int,
+                                     ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+                                     ctypes.POINTER(TestCfg), ctypes.POINTER(RoundOpts), ctypes.c_void_p,
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_logreg_round_per_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
+                                  ctypes.c_longlong, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int,
+                                  ctypes.c_int, ctypes.POINTER(ctypes.c_longlong), ctypes.c_float,
+                                  ctypes.POINTER(TestCfg), ctypes.POINTER(RoundOpts), ctypes.c_void_p, ctypes.c_void_p,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_mlp_round_per_step": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_longlong,
+                               ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p,
+                               ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_longlong), ctypes.c_float,
+                               ctypes.POINTER(TestCfg), ctypes.POINTER(RoundOpts), ctypes.c_void_p, ctypes.c_size_t,
+                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+    "abs_round_count": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
+                        ctypes.c_longlong, ctypes.c_void_p],
     "abs_mlp_param_count": [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_longlong)],
     "abs_mlp_scratch_bytes": [ctypes.c_int, ctypes.c_longlong, ctypes.POINTER(ctypes.c_int),
                               ctypes.POINTER(ctypes.c_size_t)],
@@ -89,7 +116,7 @@ EXPORTS = {
                       ctypes.POINTER(ctypes.c_int), ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_int,
                       ctypes.c_int, ctypes.c_longlong, ctypes.c_float, ctypes.POINTER(TestCfg), ctypes.c_void_p,
                       ctypes.c_size_t, ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p,
-                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
+                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "abs_next_batch_local": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(TestCfg), ctypes.c_void_p,
                              ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p],
     "abs_stats_merge": [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong,
@@ -281,14 +308,51 @@ class Context:
                                                int(b), _ptr(G), _stream(stream)), "abs_logreg_grads")
 
     def abs_logreg_round(self, A, y, idx, X, H, b, lr, cfg, G_scratch, Gb_scratch, stats, b_dev, T_out=None,
-                         stream=None):
-        """idx [H, M, >=b] int32 (contiguous in H and M); b_dev int64 device tensor holding b."""
+                         ctl=None, stream=None):
+        """idx [H, M, >=b] int32 (contiguous in H and M); b_dev int64 device tensor holding b; ctl: the
+        device counter block from new_round_ctl, or None."""
         n, d = A.shape
         M = X.shape[0]
         self._check(self._lib.abs_logreg_round(self._h, _ptr(A), _ptr(y), n, d, _ptr(idx), idx.stride(1), _ptr(X), M,
                                                int(H), int(b), float(lr), ctypes.byref(cfg), _ptr(G_scratch),
-                                               _ptr(Gb_scratch), _ptr(stats), _ptr(T_out), _ptr(b_dev),
+                                               _ptr(Gb_scratch), _ptr(stats), _ptr(T_out), _ptr(b_dev), _ptr(ctl),
                                                _stream(stream)), "abs_logreg_round")
+
+    def new_round_ctl(self, n_stop=0, samples=0, rounds=0):
+        """Device counter block (abs_round_ctl) as an int64 tensor [samples, rounds, n_stop, 0]."""
+        return torch.tensor([int(samples), int(rounds), int(n_stop), 0], dtype=torch.int64,
+                            device="cuda:%d" % self.device)
+
+    def abs_round_count(self, ctl, sizes, times, add_rounds=0, stream=None):
+        self._check(self._lib.abs_round_count(self._h, _ptr(ctl), _ptr(sizes), sizes.numel(), int(times),
+                                              int(add_rounds), _stream(stream)), "abs_round_count")
+
+    def abs_logreg_round_per_step(self, A, y, idx, X, H, b_sizes, lr, cfg, opts, G_scratch, Gb_scratch, stats,
+                                  b_dev, T_out=None, stream=None):
+        """The round with the test after every local step.  b_sizes: list of M current sizes; returns the
+        list of sizes after the round.  idx [H, M, >= cfg.b_max]; stats from new_stats(H * M);
+        T_out [H, M] or None; b_dev int64 device tensor [M]; opts from make_round_opts or None."""
+        n, d = A.shape
+        M = X.shape[0]
+        sizes = (ctypes.c_longlong * M)(*[int(v) for v in b_sizes])
+        self._check(self._lib.abs_logreg_round_per_step(
+            self._h, _ptr(A), _ptr(y), n, d, _ptr(idx), idx.stride(1), _ptr(X), M, int(H), sizes, float(lr),
+            ctypes.byref(cfg), ctypes.byref(opts) if opts is not None else None, _ptr(G_scratch), _ptr(Gb_scratch),
+            _ptr(stats), _ptr(T_out), _ptr(b_dev), _stream(stream)), "abs_logreg_round_per_step")
+        return list(sizes)
+
+    def abs_mlp_round_per_step(self, inputs_, labels, dims, idx, X, H, b_sizes, lr, cfg, opts, scratch, Gb_scratch,
+                               stats, b_dev, T_out=None, stream=None):
+        """As abs_logreg_round_per_step for the MLP problem (statistics from activations and deltas)."""
+        n = inputs_.shape[0]
+        M = X.shape[0]
+        sizes = (ctypes.c_longlong * M)(*[int(v) for v in b_sizes])
+        self._check(self._lib.abs_mlp_round_per_step(
+            self._h, _ptr(inputs_), _ptr(labels), n, (ctypes.c_int * 4)(*dims), _ptr(idx), idx.stride(1), _ptr(X), M,
+            int(H), sizes, float(lr), ctypes.byref(cfg), ctypes.byref(opts) if opts is not None else None,
+            _ptr(scratch), scratch.numel(), _ptr(Gb_scratch), _ptr(stats), _ptr(T_out), _ptr(b_dev),
+            _stream(stream)), "abs_mlp_round_per_step")
+        return list(sizes)
 
     def abs_logreg_rounds_fused(self, A, y, idx, X, H, lr, cfg, stats, b_dev, T_out=None, b_hist=None, stream=None):
         """idx [rounds, H, M, >= cfg.b_max] int32 (contiguous but for the last stride); stats [rounds*M, 7] from
@@ -307,6 +371,27 @@ class Context:
                                                       int(rounds), _ptr(X), M, int(H), float(lr), ctypes.byref(cfg),
                                                       _ptr(stats), _ptr(T_out), _ptr(b_hist), _ptr(b_dev),
                                                       _stream(stream)), "abs_logreg_rounds_fused")
+
+    def abs_logreg_rounds_fused_opts(self, A, y, idx, X, H, lr, cfg, opts, stats, b_dev, T_out=None, b_hist=None,
+                                     stream=None):
+        """The fused rounds with the cadence / size ownership / counters of `opts` (make_round_opts).
+        b_dev int64 [M]; with opts.test_every_step: stats from new_stats(rounds * H * M), T_out and b_hist
+        [rounds, H, M]; else stats new_stats(rounds * M), T_out and b_hist [rounds, M]."""
+        n, d = A.shape
+        M = X.shape[0]
+        rounds = idx.shape[0]
+        if idx.dim() != 4 or idx.shape[1] != H or idx.shape[2] != M or idx.stride(3) != 1 or \
+                idx.stride(1) != M * idx.stride(2) or idx.stride(0) != H * idx.stride(1):
+            raise ValueError("idx must be [rounds, H, M, stride] with the first three dimensions packed")
+        per = H if opts.test_every_step else 1
+        if stats.shape[0] < rounds * per * M or b_dev.numel() < M:
+            raise ValueError("stats needs rounds * %d * M records and b_dev M entries" % per)
+        if not (A.is_contiguous() and X.is_contiguous()):
+            raise ValueError("A and X must be contiguous")
+        self._check(self._lib.abs_logreg_rounds_fused_opts(
+            self._h, _ptr(A), _ptr(y), n, d, _ptr(idx), idx.stride(2), int(rounds), _ptr(X), M, int(H), float(lr),
+            ctypes.byref(cfg), ctypes.byref(opts), _ptr(stats), _ptr(T_out), _ptr(b_hist), _ptr(b_dev),
+            _stream(stream)), "abs_logreg_rounds_fused_opts")
 
     def mlp_param_count(self, dims):
         out = ctypes.c_longlong()
@@ -341,14 +426,14 @@ class Context:
                     "abs_mlp_fused_stats")
 
     def abs_mlp_round(self, inputs_, labels, dims, idx, X, H, b, lr, cfg, scratch, G_scratch, g_row_stride,
-                      Gb_scratch, stats, b_dev, T_out=None, stream=None):
+                      Gb_scratch, stats, b_dev, T_out=None, ctl=None, stream=None):
         n = inputs_.shape[0]
         M = X.shape[0]
         self._check(self._lib.abs_mlp_round(self._h, _ptr(inputs_), _ptr(labels), n, (ctypes.c_int * 4)(*dims),
                                             _ptr(idx), idx.stride(1), _ptr(X), M, int(H), int(b), float(lr),
                                             ctypes.byref(cfg), _ptr(scratch), scratch.numel(), _ptr(G_scratch),
                                             int(g_row_stride), _ptr(Gb_scratch), _ptr(stats), _ptr(T_out),
-                                            _ptr(b_dev), _stream(stream)), "abs_mlp_round")
+                                            _ptr(b_dev), _ptr(ctl), _stream(stream)), "abs_mlp_round")
 
     def replica_average(self, X, stream=None):
         X2, M, d, stride = self._replicas(X)
@@ -388,7 +473,7 @@ def plan_stats(dtype, b, aligned=True, sm_count=148, smem_optin=232448):
 
 def _record_to_dict(r):
     return dict(gbar_sq=r.gbar_sq, var_norm=r.var_norm, var_ip=r.var_ip, var_orth=r.var_orth, sum_sq=r.sum_sq,
-                rows=r.rows, status=r.status)
+                rows=r.rows, status=r.status, recomputed=r.recomputed)
 
 
 def stats_to_dicts(stats):
@@ -404,6 +489,12 @@ def stats_to_dicts(stats):
 def make_test_cfg(kind, b_max, eta=0.0, theta=0.0, nu=0.0, row_weight=1.0, divisor=1.0):
     code = {"norm": ABS_TEST_NORM, "aug_ip": ABS_TEST_AUG_INNER_PRODUCT}[kind]
     return TestCfg(code, 0, float(eta), float(theta), float(nu), int(b_max), float(row_weight), float(divisor))
+
+
+def make_round_opts(test_every_step=False, per_worker=False, eta_m=None, ctl=None):
+    """abs_round_opts; eta_m: float64 device tensor [M] or None; ctl: tensor from Context.new_round_ctl or None.
+    The tensors must stay alive while the options are in use."""
+    return RoundOpts(int(bool(test_every_step)), int(bool(per_worker)), _ptr(eta_m), _ptr(ctl))
 
 
 def make_adamw_cfg(lr, beta1, beta2, eps, weight_decay, step):

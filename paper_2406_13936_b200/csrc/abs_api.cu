@@ -44,21 +44,47 @@ int validate_stats(abs_ctx* ctx, const void* G, abs_dtype dtype, int M, long lon
   return ABS_OK;
 }
 
+// Limits beyond which a Gram kernel's record is recomputed by the tiled kernel (see Recheck).
+// Measured on bf16 rows = common vector + unit noise, d = 4 M: the relative error of var_norm is
+// about 1e-5 (tcgen05, fp32 sums over 4096..8192 columns) resp. 1e-7 (mma.sync, 256 columns) times
+// b N / ((b-1) var_norm); var_ip stays below 4e-4 up to N / sqrt(var_ip) = 5e5.  The limits keep
+// both a factor of four inside the 1e-3 tolerance of bf16 inputs.
+constexpr double kRedoKvUmma = 25.0, kRedoKvMma = 2500.0, kRedoKip = 2.0e5;
+
 int run_stats(abs_ctx* ctx, const StatsLaunch& a) {
   // ctx->flags[0] (time-out flag) is zero here: abs_create clears it and the finalisation kernel
   // of the previous call cleared it again after reading it.
   int P = 0;
   int rc = ABS_ERR_UNSUPPORTED;
+  bool gram = false, umma = false;
   if (!ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_gram) {
     rc = launch_stats_gram(ctx, a, &P);
-    if (rc == ABS_ERR_UNSUPPORTED) rc = launch_stats_umma(ctx, a, &P);
+    if (rc == ABS_ERR_UNSUPPORTED) {
+      rc = launch_stats_umma(ctx, a, &P);
+      umma = rc == ABS_OK;
+    }
+    gram = rc == ABS_OK;
   }
   if (rc == ABS_ERR_UNSUPPORTED && !ctx->tuning.stats_force_generic && !ctx->tuning.stats_no_cluster)
     rc = launch_stats_cluster(ctx, a, &P);
   if (rc == ABS_ERR_UNSUPPORTED && !ctx->tuning.stats_force_generic) rc = launch_stats_tiled(ctx, a, &P);
   if (rc == ABS_ERR_UNSUPPORTED) rc = launch_stats_generic(ctx, a, &P);
   if (rc != ABS_OK) return rc;
-  return launch_stats_finalize(ctx, a, P);
+  if (!gram || ctx->tuning.stats_no_recheck || !stats_tiled_feasible(ctx, a)) return launch_stats_finalize(ctx, a, P);
+  // Tensor-core route: finalise with the conditioning check, then the centred kernel and its
+  // finalisation, both guarded by the word the check may have raised (flags[3]).
+  Recheck rk;
+  rk.max_kv = umma ? kRedoKvUmma : kRedoKvMma;
+  rk.max_kip = kRedoKip;
+  rk.redo = ctx->flags + 3;
+  rc = launch_stats_finalize(ctx, a, P, rk);
+  if (rc != ABS_OK) return rc;
+  StatsLaunch again = a;
+  again.guard = rk.redo;
+  rc = launch_stats_tiled(ctx, again, &P);
+  if (rc != ABS_OK) return rc;
+  rk.second = 1;
+  return launch_stats_finalize(ctx, again, P, rk);
 }
 
 int grow(abs_ctx* ctx, void** buf, size_t* have, size_t need) {
@@ -152,6 +178,8 @@ extern "C" int abs_set_tuning(abs_ctx* ctx, const char* key, long long value) {
     if (value != 0 && (value < 100000 || value > 4000000000ll))
       return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_timeout_cycles must be 0 or 1e5..4e9");
     ctx->tuning.stats_timeout_cycles = value;
+  } else if (strcmp(key, "stats_no_recheck") == 0) {
+    ctx->tuning.stats_no_recheck = value ? 1 : 0;
   } else if (strcmp(key, "stats_fault_drop_loads") == 0) {
     ctx->tuning.stats_fault_drop_loads = value ? 1 : 0;
   } else if (strcmp(key, "stats_cluster_rows") == 0) {

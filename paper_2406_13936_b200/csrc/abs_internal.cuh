@@ -28,6 +28,7 @@ struct Tuning {
   long long stats_ctas_per_sm = 0;
   long long stats_no_gram = 0;
   long long stats_no_cluster = 0;
+  long long stats_no_recheck = 0;          // 1: keep a Gram kernel's record whatever its conditioning
   long long stats_cluster_rows = 0;
   long long stats_timeout_cycles = 0;      // 0: about two seconds of SM clock
   long long stats_fault_drop_loads = 0;    // test hook: the tiled kernel's loader issues no copies
@@ -147,7 +148,7 @@ __device__ __forceinline__ abs_stats record_from_sums(double V, double N, double
   s.sum_sq = V + bd * N;
   s.rows = b;
   s.status = status;
-  s.reserved = 0u;
+  s.recomputed = 0u;
   return s;
 }
 #endif
@@ -165,6 +166,20 @@ struct StatsLaunch {
   float* gbar_out;
   abs_stats* stats_out;
   cudaStream_t stream;
+  const unsigned* guard = nullptr;   // device word or NULL: the tiled kernel returns at once while it is zero
+};
+
+// How the finalisation treats the records of a tensor-core Gram kernel.  Those kernels only ever
+// see uncentred products added in fp32, so sum_i ||g_i - gbar||^2 = tr K - 1'K1/b loses
+// b N / ((b-1) var_norm) in relative accuracy (rows dominated by a common vector), and
+// e_i = (K1)_i/b - N loses N / sqrt(var_ip).  A record beyond the limits raises *redo; the tiled
+// kernel (centred accumulation) and a second finalisation then run guarded by that word, and
+// return at once when it is zero.
+struct Recheck {
+  double max_kv = 0.0;       // 0: no check; else recompute when b N > max_kv (b-1) var_norm
+  double max_kip = 0.0;      //                          or when N^2 > max_kip^2 var_ip
+  unsigned* redo = nullptr;  // device word
+  int second = 0;            // 1: the finalisation of the recomputation: a no-op unless *redo, which it clears
 };
 
 // Returns ABS_OK, or ABS_ERR_UNSUPPORTED when the tiled kernel cannot take the call
@@ -174,7 +189,9 @@ int launch_stats_gram(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // b
 int launch_stats_umma(abs_ctx* ctx, const StatsLaunch& a, int* P_out);      // bf16, 32 < b <= 256 (tcgen05)
 int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out);   // 256 < b <= 4096
 int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
-int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P);
+int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P, const Recheck& rk = Recheck());
+// True when launch_stats_tiled would take the call (shape, alignment, workspace).
+bool stats_tiled_feasible(abs_ctx* ctx, const StatsLaunch& a);
 
 // Host-side planning shared by the launchers and abs_plan_stats; ABS_OK or ABS_ERR_UNSUPPORTED.
 int plan_stats_gram(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out);

@@ -31,8 +31,12 @@
 // flag, all later waits of the CTA return at once, the barriers that follow are still reached,
 // and the round's records carry ABS_STATUS_TIMEOUT.  No CTA leaves while a peer may still copy
 // into it: a grid barrier follows the last exchange.
-// Data that crosses clusters inside the launch goes through L2 only (st.cg / ld.cg) and is
-// reused no sooner than a grid barrier later.  Every CTA executes the same sequence of barriers:
+// Data that crosses clusters inside the launch goes through L2 only (st.cg / ld.cg).  A round has
+// one grid barrier, between the writers of S / Xpre and their readers (phase D); nothing holds a
+// fast worker back from running the next round's local steps and writing its sums again while a
+// slow CTA of another worker is still in phase D.  So S and Xpre exist twice and alternate by round:
+// the copy read in round r is written again in round r + 2, whose writers have passed the barrier
+// of round r + 1, which every CTA reaches only after its phase D of round r.  Every CTA executes the same sequence of barriers:
 // the trip counts depend only on (rounds, H) and on b, which all CTAs derive from the same values.
 #include <cooperative_groups.h>
 
@@ -65,9 +69,25 @@ struct FusedParams {
   unsigned* flag;   // device word, zero at launch: set when a wait for the peers' partials ran out
   long long timeout_cycles;
   int drop_copies;  // test hook: the partials are not sent, so the waits run out
-  double* S;        // [M][P][4]      V, sum e, sum e^2, N
-  float* Xpre;      // [M][d]         parameters before the averaging
+  double* S;        // [2][M][P][4]   V, sum e, sum e^2, N           (two copies that alternate by round:
+  float* Xpre;      // [2][M][d]      parameters before the averaging  see the note on the grid barrier)
+  long long* Sx;    // [2][M]         samples each worker used in the round (counter B of Alg. 1 / Alg. 2)
+  long long* Bx;    // [2][M]         sizes the workers ask for after a step (per-step cadence, shared size)
+  // cadence and bookkeeping (all zero / NULL: the test once per round, one size shared by all workers)
+  int every_step;   // the test after every local step (Algorithm 1)
+  int per_worker;   // every worker keeps its own size (Eq. test_stat); else the maximum over workers
+  int sizes_per_worker;   // b_dev / b_hist hold one value per worker
+  const double* eta_m;    // [M] norm-test constants per worker, or NULL
+  abs_round_ctl* ctl;     // sample counter and stop rule, or NULL
 };
+
+__device__ __forceinline__ void st_cluster_f64(uint32_t addr, double v) {
+  asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 __device__ __forceinline__ double warp_sum_dd(double v) {
 #pragma unroll
@@ -91,7 +111,10 @@ __device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefe
 
 // KV: 16-byte column vectors per lane (slot k of a lane is vector k*32 + lane of the row).
 // NW: warps per CTA (16 for narrow rows, where a warp's registers allow it: fewer samples per warp).
-template <int KV, int NW>
+// EVERY: the per-step cadence of Algorithm 1 (statistics, T and the size update after every local
+// step; one cluster barrier per step for the statistics' partial sums, and a grid barrier per step
+// when all workers share one size).
+template <int KV, int NW, bool EVERY>
 __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedParams prm) {
   constexpr int NT = NW * 32;
   constexpr int U = (NW > 8 ? 8 : 16) / KV;   // samples a warp keeps in flight (8 or 16 row vectors in registers)
@@ -112,6 +135,8 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
   __shared__ double N_s;
   __shared__ long long T_s[kMaxWorkersFused];
   __shared__ long long b_s;
+  __shared__ __align__(16) double sbox[2][kMaxCtasPerWorker][4];   // per-step cadence: V, sum e, sum e^2, abort
+                                                                    // of every CTA of the cluster, by step parity
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int M = prm.M, P = prm.P;
@@ -122,10 +147,18 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
   const float lr = prm.lr;
 
   for (int j = tid; j < DV; j += NT) x4[j] = X4[static_cast<long long>(m) * DV + j];
-  long long b = prm.b_dev[0];
+  long long b = prm.b_dev[prm.sizes_per_worker ? m : 0];
   if (b > prm.cfg.b_max) b = prm.cfg.b_max;
   if (b < 2) b = 2;                        // the variance needs two rows
-  if (blockIdx.x == 0 && tid == 0 && prm.b_hist != nullptr) prm.b_hist[0] = b;
+  if (blockIdx.x == 0 && tid == 0 && prm.b_hist != nullptr && !prm.sizes_per_worker) prm.b_hist[0] = b;
+  abs_test_cfg cfg_m = prm.cfg;            // this worker's constants (eta_m of Eq. approx_norm_local)
+  if (prm.eta_m != nullptr) cfg_m.eta = prm.eta_m[m];
+  long long B = 0, n_stop = 0;             // the counter B and the N of "while B < N"; the same in every CTA
+  if (prm.ctl != nullptr) {
+    B = prm.ctl->samples;
+    n_stop = prm.ctl->n_stop;
+  }
+  int rounds_done = 0;
   if (tid == 0) {
     mbar_init(xbar_u32, 1);
     mbar_init(xbar_u32 + 8u, 1);
@@ -149,15 +182,27 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
   long long chunk0_row = 0;                                          // row of sample `lane` of the current step
 
   for (int r = 0; r < prm.rounds; ++r) {
-    const int Pa = static_cast<int>(b < P ? b : P);                 // CTAs of a worker that have samples
-    const long long n_mine = b > first ? (b - first + hop - 1) / hop : 0;
-    const float inv_b = 1.0f / static_cast<float>(b);
+    if (n_stop > 0 && B >= n_stop) break;                           // Alg. 1 / Alg. 2: while B < N
+    long long used = 0;                                             // samples of this worker in this round
+    int Pa = static_cast<int>(b < P ? b : P);                       // CTAs of a worker that have samples
+    long long n_mine = b > first ? (b - first + hop - 1) / hop : 0;
+    float inv_b = 1.0f / static_cast<float>(b);
     chunk0_row = lane < n_mine ? fetch_row(prm.idx + (static_cast<long long>(r) * prm.H * M + m) * prm.idx_stride, lane) : 0;
     for (int h = 0; h < prm.H; ++h) {
       const long long gstep = static_cast<long long>(r) * prm.H + h;
       const bool last = h == prm.H - 1;
+      const bool test_now = EVERY || last;                          // statistics on this step's gradients
       const int* idx_m = prm.idx + (gstep * M + m) * prm.idx_stride;
       float4* part4 = inbox4 + (gstep & 1) * static_cast<long long>(P) * DV;
+      if (EVERY && h > 0) {
+        // the size may have grown since the last step: the step's quantities again, and the first
+        // chunk of row indices now (nothing was fetched ahead for lanes that had no sample before)
+        Pa = static_cast<int>(b < P ? b : P);
+        n_mine = b > first ? (b - first + hop - 1) / hop : 0;
+        inv_b = 1.0f / static_cast<float>(b);
+        chunk0_row = lane < n_mine ? fetch_row(idx_m, lane) : 0;
+      }
+      used += b;
 
       // ---- phase A: partial batch gradient of this CTA ------------------------------------
       float4 acc[KV];
@@ -168,7 +213,7 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
       // (the value is not touched before the samples of this step are done: an instruction that
       // used it here would make the warp wait for the load)
       int ahead_raw = 0;
-      if (!last && lane < n_mine) ahead_raw = (idx_m + static_cast<long long>(M) * prm.idx_stride)[first + lane * hop];
+      if (!EVERY && !last && lane < n_mine) ahead_raw = (idx_m + static_cast<long long>(M) * prm.idx_stride)[first + lane * hop];
       for (long long t0 = 0; t0 < n_mine; t0 += 32) {
         const int cnt = static_cast<int>(n_mine - t0 < 32 ? n_mine - t0 : 32);
         long long my_row = chunk0_row;
@@ -223,7 +268,7 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
         const int j = k * 32 + lane;
         if (j < DV) wacc4[warp * DV + j] = acc[k];
       }
-      if (!last) {
+      if (!EVERY && !last) {
         // the next step's rows on their way into L1 while the barrier is crossed
         const long long ahead_row = clamp_row(ahead_raw);
         const int cnt0 = static_cast<int>(n_mine < 32 ? n_mine : 32);
@@ -293,7 +338,7 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
           }
           s.x *= inv_b; s.y *= inv_b; s.z *= inv_b; s.w *= inv_b;
           g4[jj] = s;
-          if (!last) {
+          if (!test_now) {
             float4 xv = x4[jj];
             xv.x = fmaf(-lr, s.x, xv.x); xv.y = fmaf(-lr, s.y, xv.y);
             xv.z = fmaf(-lr, s.z, xv.z); xv.w = fmaf(-lr, s.w, xv.w);
@@ -302,7 +347,7 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
         }
         __syncthreads();
       }
-      if (!last) continue;
+      if (!test_now) continue;
 
       // ---- phase C: statistics of the last local step's per-sample gradients -----------------
       if (warp == 0) {
@@ -389,27 +434,106 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
         red[warp][2] = see;
       }
       __syncthreads();
-      if (tid == 0 && p < Pa) {
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0;
-        for (int w = 0; w < NW; ++w) {
-          a0 += red[w][0];
-          a1 += red[w][1];
-          a2 += red[w][2];
+      if (EVERY) {
+        // ---- per-step cadence: the cluster's sums, this worker's record, T and the size update ----
+        // Every CTA puts its three partial sums (and whether one of its waits ran out) into its slot
+        // of every CTA of the cluster; the cluster barrier makes them visible; every CTA then adds
+        // the P slots in slot order, so all of them take the same decision.  The slots alternate by
+        // step: a peer writes step h + 2 only after the barrier of step h + 1, which this CTA reaches
+        // after it has read the slots of step h.
+        const int par2 = static_cast<int>(gstep & 1);
+        if (tid < P) {
+          double a0 = 0.0, a1 = 0.0, a2 = 0.0;
+          for (int w = 0; w < NW; ++w) {
+            a0 += red[w][0];
+            a1 += red[w][1];
+            a2 += red[w][2];
+          }
+          const uint32_t slot = map_to_rank(smem_u32(&sbox[par2][p][0]), static_cast<uint32_t>(tid));
+          st_cluster_f64(slot, a0);
+          st_cluster_f64(slot + 8u, a1);
+          st_cluster_f64(slot + 16u, a2);
+          st_cluster_f64(slot + 24u, abort_s != 0u ? 1.0 : 0.0);
         }
-        double* dst = prm.S + (static_cast<long long>(m) * P + p) * 4;
-        __stcg(dst + 0, a0);
-        __stcg(dst + 1, a1);
-        __stcg(dst + 2, a2);
-        __stcg(dst + 3, N_s);
-      }
-      // the step that was held back, and this worker's parameters for the averaging
-      for (int j = tid; j < DV; j += NT) {
-        const float4 s = g4[j];
-        float4 xv = x4[j];
-        xv.x = fmaf(-lr, s.x, xv.x); xv.y = fmaf(-lr, s.y, xv.y);
-        xv.z = fmaf(-lr, s.z, xv.z); xv.w = fmaf(-lr, s.w, xv.w);
-        x4[j] = xv;
-        if (p == 0) __stcg(Xpre4 + static_cast<long long>(m) * DV + j, xv);
+        cluster_barrier();
+        if (tid == 0) {
+          double V = 0.0, se = 0.0, see = 0.0, ab = 0.0;
+          for (int q = 0; q < P; ++q) {
+            V += sbox[par2][q][0];
+            se += sbox[par2][q][1];
+            see += sbox[par2][q][2];
+            ab += sbox[par2][q][3];
+          }
+          const bool timed_out = ab != 0.0;
+          if (timed_out && p == 0) atomicOr(prm.flag, 1u);
+          const abs_stats rec = record_from_sums(V, N_s, se, see, b, timed_out);
+          const long long T = test_size_from_record(rec, cfg_m);
+          long long want = T > b ? T : b;                             // Alg. 1: b <- max{T, b}
+          want = want < prm.cfg.b_max ? want : prm.cfg.b_max;
+          if (p == 0) {
+            const long long slot = gstep * M + m;
+            prm.stats[slot] = rec;
+            if (prm.T_out != nullptr) prm.T_out[slot] = T;
+            if (prm.b_hist != nullptr) prm.b_hist[slot] = b;          // the size this step ran with
+            if (!prm.per_worker) __stcg(prm.Bx + static_cast<long long>(par2) * M + m, want);
+          }
+          b_s = want;
+        }
+        // the step that was held back
+        for (int j = tid; j < DV; j += NT) {
+          const float4 s = g4[j];
+          float4 xv = x4[j];
+          xv.x = fmaf(-lr, s.x, xv.x); xv.y = fmaf(-lr, s.y, xv.y);
+          xv.z = fmaf(-lr, s.z, xv.z); xv.w = fmaf(-lr, s.w, xv.w);
+          x4[j] = xv;
+          if (last && p == 0) __stcg(Xpre4 + (static_cast<long long>(r & 1) * M + m) * DV + j, xv);
+        }
+        if (!prm.per_worker) {
+          // one size for all workers: the maximum of what they ask for (display below Eq. test_stat),
+          // taken after every step, which costs a grid barrier per step
+          grid.sync();
+          if (tid == 0) {
+            long long best = 0;
+            for (int w = 0; w < M; ++w) {
+              const long long v = __ldcg(prm.Bx + static_cast<long long>(par2) * M + w);
+              best = v > best ? v : best;
+            }
+            b_s = best;
+          }
+        }
+        __syncthreads();
+        b = b_s;
+        if (!last) continue;
+        if (tid == 0 && p == 0 && prm.ctl != nullptr) __stcg(prm.Sx + static_cast<long long>(r & 1) * M + m, used);
+      } else {
+        if (tid == 0) {
+          // CTAs without samples contribute zeros, so that a reader need not know how many CTAs of
+          // another worker (whose size may differ) were active
+          double a0 = 0.0, a1 = 0.0, a2 = 0.0;
+          for (int w = 0; w < NW; ++w) {
+            a0 += red[w][0];
+            a1 += red[w][1];
+            a2 += red[w][2];
+          }
+          double* dst = prm.S + ((static_cast<long long>(r & 1) * M + m) * P + p) * 4;
+          __stcg(dst + 0, a0);
+          __stcg(dst + 1, a1);
+          __stcg(dst + 2, a2);
+          __stcg(dst + 3, N_s);
+          if (p == 0) {
+            if (prm.ctl != nullptr) __stcg(prm.Sx + static_cast<long long>(r & 1) * M + m, used);
+            if (prm.per_worker) __stcg(prm.Bx + static_cast<long long>(r & 1) * M + m, b);
+          }
+        }
+        // the step that was held back, and this worker's parameters for the averaging
+        for (int j = tid; j < DV; j += NT) {
+          const float4 s = g4[j];
+          float4 xv = x4[j];
+          xv.x = fmaf(-lr, s.x, xv.x); xv.y = fmaf(-lr, s.y, xv.y);
+          xv.z = fmaf(-lr, s.z, xv.z); xv.w = fmaf(-lr, s.w, xv.w);
+          x4[j] = xv;
+          if (p == 0) __stcg(Xpre4 + (static_cast<long long>(r & 1) * M + m) * DV + j, xv);
+        }
       }
       if (tid == 0 && abort_s != 0u) atomicOr(prm.flag, 1u);
       grid.sync();
@@ -420,26 +544,32 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
       // they are spread over the threads and issued together: the records by one warp per worker
       // (lane q reads the sums of CTA q; the shuffle tree adds them in a fixed order), the
       // parameters by thread groups that split the workers and are added in group order.
-      for (int w = warp; w < M; w += NW) {
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0, nn = 0.0;
-        if (lane < Pa) {
-          const double* src = prm.S + (static_cast<long long>(w) * P + lane) * 4;
-          a0 = __ldcg(src + 0);
-          a1 = __ldcg(src + 1);
-          a2 = __ldcg(src + 2);
-          nn = __ldcg(src + 3);
-        }
-        a0 = warp_sum_dd(a0);
-        a1 = warp_sum_dd(a1);
-        a2 = warp_sum_dd(a2);
-        nn = __shfl_sync(0xffffffffu, nn, 0);
-        if (lane == 0) {
-          const abs_stats rec = record_from_sums(a0, nn, a1, a2, b, timed_out);
-          const long long T = test_size_from_record(rec, prm.cfg);
-          T_s[w] = T;
-          if (blockIdx.x == 0) {
-            prm.stats[static_cast<long long>(r) * M + w] = rec;
-            if (prm.T_out != nullptr) prm.T_out[static_cast<long long>(r) * M + w] = T;
+      if (!EVERY) {
+        for (int w = warp; w < M; w += NW) {
+          double a0 = 0.0, a1 = 0.0, a2 = 0.0, nn = 0.0;
+          if (lane < P) {
+            const double* src = prm.S + ((static_cast<long long>(r & 1) * M + w) * P + lane) * 4;
+            a0 = __ldcg(src + 0);
+            a1 = __ldcg(src + 1);
+            a2 = __ldcg(src + 2);
+            nn = __ldcg(src + 3);
+          }
+          a0 = warp_sum_dd(a0);
+          a1 = warp_sum_dd(a1);
+          a2 = warp_sum_dd(a2);
+          nn = __shfl_sync(0xffffffffu, nn, 0);
+          if (lane == 0) {
+            const long long b_w = prm.per_worker ? __ldcg(prm.Bx + static_cast<long long>(r & 1) * M + w) : b;
+            abs_test_cfg cfg_w = prm.cfg;
+            if (prm.eta_m != nullptr) cfg_w.eta = prm.eta_m[w];
+            const abs_stats rec = record_from_sums(a0, nn, a1, a2, b_w, timed_out);
+            const long long T = test_size_from_record(rec, cfg_w);
+            T_s[w] = T;
+            if (blockIdx.x == 0) {
+              prm.stats[static_cast<long long>(r) * M + w] = rec;
+              if (prm.T_out != nullptr) prm.T_out[static_cast<long long>(r) * M + w] = T;
+              if (prm.b_hist != nullptr && prm.sizes_per_worker) prm.b_hist[static_cast<long long>(r) * M + w] = b_w;
+            }
           }
         }
       }
@@ -451,7 +581,7 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
           float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
           for (int w = grp; w < M; w += groups) {
-            const float4 v = __ldcg(Xpre4 + static_cast<long long>(w) * DV + j);
+            const float4 v = __ldcg(Xpre4 + (static_cast<long long>(r & 1) * M + w) * DV + j);
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
           }
           wacc4[grp * DV + j] = s;
@@ -465,22 +595,43 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
           }
           s.x *= inv_M; s.y *= inv_M; s.z *= inv_M; s.w *= inv_M;
           x4[jj] = s;
-          if (p == 0 && r == prm.rounds - 1) X4[static_cast<long long>(m) * DV + jj] = s;
         }
       }
       __syncthreads();
       if (tid == 0) {
         long long best = b;
-        for (int w = 0; w < M; ++w) best = T_s[w] > best ? T_s[w] : best;
-        best = best < prm.cfg.b_max ? best : prm.cfg.b_max;
+        if (!EVERY) {
+          if (prm.per_worker) {
+            best = T_s[m] > best ? T_s[m] : best;                    // Eq. test_stat: the worker's own T
+          } else {
+            for (int w = 0; w < M; ++w) best = T_s[w] > best ? T_s[w] : best;
+          }
+          best = best < prm.cfg.b_max ? best : prm.cfg.b_max;
+        }
         b_s = best;
-        if (blockIdx.x == 0 && prm.b_hist != nullptr) prm.b_hist[r + 1] = best;
+        if (blockIdx.x == 0 && prm.b_hist != nullptr && !prm.sizes_per_worker) prm.b_hist[r + 1] = best;
+        // the round's term of the sample counter: sum_m sum_h b^m_{k,h} (Alg. 1), which is H M b_k when
+        // the size is shared and constant over the round (Alg. 2)
+        long long tot = 0;
+        if (prm.ctl != nullptr)
+          for (int w = 0; w < M; ++w) tot += __ldcg(prm.Sx + static_cast<long long>(r & 1) * M + w);
+        T_s[0] = tot;       // T_s is free again: every thread is past the loop above (barrier before this block)
       }
       __syncthreads();
       b = b_s;
+      B += T_s[0];
+      ++rounds_done;
+      __syncthreads();      // T_s[0] is overwritten by the next round's records
     }
   }
-  if (blockIdx.x == 0 && tid == 0) prm.b_dev[0] = b;
+  // the parameters after the last round that ran (x^m_{K,0}: the output of Alg. 1 / Alg. 2 is replica 1)
+  if (p == 0 && rounds_done > 0)
+    for (int jj = tid; jj < DV; jj += NT) X4[static_cast<long long>(m) * DV + jj] = x4[jj];
+  if (tid == 0 && p == 0 && (prm.sizes_per_worker || m == 0)) prm.b_dev[prm.sizes_per_worker ? m : 0] = b;
+  if (blockIdx.x == 0 && tid == 0 && prm.ctl != nullptr) {
+    prm.ctl->samples = B;
+    prm.ctl->rounds += rounds_done;
+  }
 }
 
 using KernelFn = void (*)(const FusedParams);
@@ -488,11 +639,17 @@ struct KernelChoice {
   KernelFn fn;
   int warps;
 };
-KernelChoice pick_kernel(int DV) {
-  if (DV <= 32) return {logreg_rounds_kernel<1, 16>, 16};
-  if (DV <= 64) return {logreg_rounds_kernel<2, 16>, 16};
-  if (DV <= 128) return {logreg_rounds_kernel<4, 8>, 8};
-  return {logreg_rounds_kernel<8, 8>, 8};
+KernelChoice pick_kernel(int DV, bool every) {
+  if (every) {
+    if (DV <= 32) return {logreg_rounds_kernel<1, 16, true>, 16};
+    if (DV <= 64) return {logreg_rounds_kernel<2, 16, true>, 16};
+    if (DV <= 128) return {logreg_rounds_kernel<4, 8, true>, 8};
+    return {logreg_rounds_kernel<8, 8, true>, 8};
+  }
+  if (DV <= 32) return {logreg_rounds_kernel<1, 16, false>, 16};
+  if (DV <= 64) return {logreg_rounds_kernel<2, 16, false>, 16};
+  if (DV <= 128) return {logreg_rounds_kernel<4, 8, false>, 8};
+  return {logreg_rounds_kernel<8, 8, false>, 8};
 }
 
 }  // namespace
@@ -500,10 +657,11 @@ KernelChoice pick_kernel(int DV) {
 
 using namespace absk;
 
-extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
-                                       const int* idx, long long idx_stride, int rounds, float* X, int M, int H,
-                                       float lr, const abs_test_cfg* cfg, abs_stats* stats, long long* T_out,
-                                       long long* b_hist, long long* b_dev, void* stream) {
+extern "C" int abs_logreg_rounds_fused_opts(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
+                                            const int* idx, long long idx_stride, int rounds, float* X, int M, int H,
+                                            float lr, const abs_test_cfg* cfg, const abs_round_opts* opts,
+                                            abs_stats* stats, long long* T_out, long long* b_hist, long long* b_dev,
+                                            void* stream) {
   if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
   if (A == nullptr || y == nullptr || idx == nullptr || X == nullptr || cfg == nullptr || stats == nullptr ||
       b_dev == nullptr)
@@ -514,7 +672,8 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
     return set_error(ctx, ABS_ERR_INVALID_ARG, "unknown test kind %d", cfg->kind);
   if (cfg->b_max < 2 || !(cfg->row_weight > 0.0) || !(cfg->divisor > 0.0))
     return set_error(ctx, ABS_ERR_INVALID_ARG, "need b_max >= 2, row_weight > 0, divisor > 0");
-  if (cfg->kind == ABS_TEST_NORM ? !(cfg->eta > 0.0) : !(cfg->theta > 0.0 && cfg->nu > 0.0))
+  if (cfg->kind == ABS_TEST_NORM ? !(cfg->eta > 0.0 || (opts != nullptr && opts->eta_m != nullptr))
+                                 : !(cfg->theta > 0.0 && cfg->nu > 0.0))
     return set_error(ctx, ABS_ERR_INVALID_ARG, "test constants must be positive");
   if (idx_stride < cfg->b_max)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "idx_stride (%lld) must cover b_max (%lld): the batch may grow to it",
@@ -533,8 +692,9 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
     ~Restore() { if (prev != dev) cudaSetDevice(prev); }
   } restore{prev, ctx->device};
 
+  const bool every = opts != nullptr && opts->test_every_step != 0;
   const int DV = static_cast<int>(d / 4);
-  const KernelChoice choice = pick_kernel(DV);
+  const KernelChoice choice = pick_kernel(DV, every);
   KernelFn kernel = choice.fn;
   const size_t smem_fixed = static_cast<size_t>(2 + choice.warps + 2) * d * sizeof(float);   // + 2 P d floats of inboxes
 
@@ -553,7 +713,7 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
   int P = 0;
   for (int cand = kMaxCtasPerWorker; cand >= 1 && P == 0; cand >>= 1) {
     const size_t smem = smem_fixed + 2ull * cand * d * sizeof(float);
-    if (smem + 1024 > ctx->smem_optin) continue;      // 1 KiB for the static shared variables
+    if (smem + 2048 > ctx->smem_optin) continue;      // 2 KiB for the static shared variables
     ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel),
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     lc.dynamicSmemBytes = smem;
@@ -571,12 +731,13 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
   }
   if (P == 0) return set_error(ctx, ABS_ERR_UNSUPPORTED, "%d workers do not fit a co-resident grid", M);
 
-  // scratch in the context's workspace: statistics partials, pre-average parameters
-  const size_t S_bytes = static_cast<size_t>(M) * P * 4 * sizeof(double);
-  const size_t xpre_bytes = static_cast<size_t>(M) * d * sizeof(float);
-  if (S_bytes + xpre_bytes > ctx->workspace_bytes)
+  // scratch in the context's workspace: statistics partials, pre-average parameters, sample counts, sizes
+  const size_t S_bytes = 2 * static_cast<size_t>(M) * P * 4 * sizeof(double);       // two copies each,
+  const size_t xpre_bytes = 2 * static_cast<size_t>(M) * d * sizeof(float);          // alternating by round
+  const size_t cnt_bytes = 2 * static_cast<size_t>(M) * sizeof(long long);
+  if (S_bytes + xpre_bytes + 2 * cnt_bytes > ctx->workspace_bytes)
     return set_error(ctx, ABS_ERR_WORKSPACE, "workspace of %zu bytes is too small (%zu needed)", ctx->workspace_bytes,
-                     S_bytes + xpre_bytes);
+                     S_bytes + xpre_bytes + 2 * cnt_bytes);
   unsigned char* ws = static_cast<unsigned char*>(ctx->workspace);
 
   FusedParams prm;
@@ -590,7 +751,22 @@ extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
   ABS_CUDA_TRY(ctx, cudaMemsetAsync(prm.flag, 0, sizeof(unsigned), static_cast<cudaStream_t>(stream)));
   prm.S = reinterpret_cast<double*>(ws);
-  prm.Xpre = reinterpret_cast<float*>(ws + S_bytes);
+  prm.Sx = reinterpret_cast<long long*>(ws + S_bytes);
+  prm.Bx = reinterpret_cast<long long*>(ws + S_bytes + cnt_bytes);
+  prm.Xpre = reinterpret_cast<float*>(ws + S_bytes + 2 * cnt_bytes);
+  prm.every_step = every ? 1 : 0;
+  prm.per_worker = opts != nullptr && opts->per_worker != 0 ? 1 : 0;
+  prm.sizes_per_worker = opts != nullptr ? 1 : 0;
+  prm.eta_m = opts != nullptr ? opts->eta_m : nullptr;
+  prm.ctl = opts != nullptr ? opts->ctl : nullptr;
   ABS_CUDA_TRY(ctx, cudaLaunchKernelEx(&lc, kernel, prm));
   return ABS_OK;
+}
+
+extern "C" int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
+                                       const int* idx, long long idx_stride, int rounds, float* X, int M, int H,
+                                       float lr, const abs_test_cfg* cfg, abs_stats* stats, long long* T_out,
+                                       long long* b_hist, long long* b_dev, void* stream) {
+  return abs_logreg_rounds_fused_opts(ctx, A, y, n, d, idx, idx_stride, rounds, X, M, H, lr, cfg, nullptr, stats,
+                                      T_out, b_hist, b_dev, stream);
 }

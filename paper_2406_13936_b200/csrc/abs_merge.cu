@@ -85,7 +85,7 @@ __global__ void merge_records_kernel(abs_stats* __restrict__ ra, const abs_stats
   o.status = ((a.status | b.status) & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) | ABS_STATUS_NORM_ONLY;
   if (!(isfinite(S) && isfinite(msq))) o.status |= ABS_STATUS_NONFINITE;
   if (msq == 0.0) o.status |= ABS_STATUS_ZERO_MEAN;
-  o.reserved = 0u;
+  o.recomputed = 0u;
   ra[m] = o;
 }
 

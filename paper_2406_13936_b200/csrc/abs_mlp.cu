@@ -300,20 +300,26 @@ void launch_gemm(const GemmArgs& g, int batch, cudaStream_t st) {
   sgemm_kernel<<<grid, 256, 0, st>>>(g);
 }
 
+// Sample indices outside [0, n) are clamped: a bad index never becomes an out-of-range read.
+__device__ __forceinline__ long long clamp_sample(int raw, long long n) {
+  return raw < 0 ? 0 : (raw >= n ? n - 1 : static_cast<long long>(raw));
+}
+
 // Xin[m][i][:] = inputs[idx[m][i]][:]
-__global__ void gather_rows_kernel(const float* __restrict__ inputs, const int* __restrict__ idx, long long idx_stride,
-                                   long long b, int n0, float* __restrict__ scratch, long long per_worker) {
+__global__ void gather_rows_kernel(const float* __restrict__ inputs, long long n, const int* __restrict__ idx,
+                                   long long idx_stride, long long b, int n0, float* __restrict__ scratch,
+                                   long long per_worker) {
   const int m = blockIdx.y;
   const long long i = blockIdx.x;
-  const float* src = inputs + static_cast<long long>(idx[m * idx_stride + i]) * n0;
+  const float* src = inputs + clamp_sample(idx[m * idx_stride + i], n) * n0;
   float* dst = scratch + m * per_worker + i * n0;
   for (int j = threadIdx.x; j < n0; j += blockDim.x) dst[j] = src[j];
 }
 
 // In place on the logits: D3[i][:] = softmax(logits_i) - onehot(label_i); one thread per sample.
 __global__ void softmax_delta_kernel(float* __restrict__ scratch, long long per_worker, long long off, long long b,
-                                     int n3, const int* __restrict__ labels, const int* __restrict__ idx,
-                                     long long idx_stride) {
+                                     int n3, const int* __restrict__ labels, long long n,
+                                     const int* __restrict__ idx, long long idx_stride) {
   const int m = blockIdx.y;
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= b) return;
@@ -326,7 +332,7 @@ __global__ void softmax_delta_kernel(float* __restrict__ scratch, long long per_
     z[c] = e;
     sum += e;
   }
-  const int label = labels[idx[m * idx_stride + i]];
+  const int label = labels[clamp_sample(idx[m * idx_stride + i], n)];
   for (int c = 0; c < n3; ++c) z[c] = z[c] / sum - (c == label ? 1.f : 0.f);
 }
 
@@ -539,7 +545,7 @@ fused_finalize_kernel(const float* __restrict__ scratch, long long per_worker, l
     o.status = 0u;
     if (!(isfinite(qsum) && isfinite(N) && isfinite(ss))) o.status |= ABS_STATUS_NONFINITE;
     if (N == 0.0) o.status |= ABS_STATUS_ZERO_MEAN;
-    o.reserved = 0u;
+    o.recomputed = 0u;
     stats[m] = o;
   }
 }
@@ -590,7 +596,7 @@ extern "C" int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* label
   const long long pw = s.per_worker, d = s.d;
   const float inv_b = 1.0f / static_cast<float>(b);
 
-  gather_rows_kernel<<<dim3(static_cast<unsigned>(b), M), 128, 0, st>>>(inputs, idx, idx_stride, b, s.n0, ws, pw);
+  gather_rows_kernel<<<dim3(static_cast<unsigned>(b), M), 128, 0, st>>>(inputs, n, idx, idx_stride, b, s.n0, ws, pw);
 
   GemmArgs g;
   // forward: H1 = relu(Xin W1^T + b1), H2 = relu(H1 W2^T + b2), logits = H2 W3^T + b3
@@ -604,7 +610,7 @@ extern "C" int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* label
                static_cast<int>(b), s.n3, s.n2, 1.f, 2};
   launch_gemm(g, M, st);
   softmax_delta_kernel<<<dim3(static_cast<unsigned>((b + 127) / 128), M), 128, 0, st>>>(ws, pw, s.sD3, b, s.n3, labels,
-                                                                                       idx, idx_stride);
+                                                                                       n, idx, idx_stride);
   // backward: D2 = (D3 W3) .* (H2 > 0), D1 = (D2 W2) .* (H1 > 0)
   g = GemmArgs{ws + s.sD3, s.n3, 1, pw, X + s.oW3, s.n2, 1, d, ws + s.sD2, s.n2, pw, nullptr, 0, ws + s.sH2, s.n2, pw,
                static_cast<int>(b), s.n2, s.n3, 1.f, 3};
@@ -717,7 +723,7 @@ extern "C" int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* label
                              const int* idx, long long idx_stride, float* X, int M, int H, long long b, float lr,
                              const abs_test_cfg* cfg, void* scratch, size_t scratch_bytes, float* G_scratch,
                              long long g_row_stride, float* Gb_scratch, abs_stats* stats, long long* T_out,
-                             long long* b_dev, void* stream) {
+                             long long* b_dev, abs_round_ctl* ctl, void* stream) {
   if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
   if (cfg == nullptr || Gb_scratch == nullptr || stats == nullptr || b_dev == nullptr)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
@@ -743,6 +749,10 @@ extern "C" int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* label
       }
     }
     rc = local_sgd_step(ctx, X, Gb_scratch, M, d, d, lr, h == H - 1 ? 1 : 0, stream);
+    if (rc != ABS_OK) return rc;
+  }
+  if (ctl != nullptr) {      // Alg. 2: B <- B + H M b_k, k <- k + 1 (with the size the round ran with)
+    rc = abs_round_count(ctx, ctl, b_dev, 1, static_cast<long long>(H) * M, 1, stream);
     if (rc != ABS_OK) return rc;
   }
   return abs_next_batch(ctx, stats, M, cfg, b_dev, T_out, b_dev, stream);

@@ -1,5 +1,5 @@
 // Producers of per-sample gradients for the two synthetic end-to-end problems (Algorithm 1,
-// "compute per-sample gradients"; Algorithm 2 for the round structure), and the round drivers
+// per-sample gradient step; Algorithm 2 for the round structure), and the round drivers
 // that chain producer -> statistics -> local SGD step -> averaging -> batch-size update.
 //
 //   logistic regression   g_i = (sigmoid(a_i^T x) - y_i) a_i
@@ -27,7 +27,7 @@ struct DeviceScopeP {
 // ---- logistic regression --------------------------------------------------------------------
 // One warp per (worker, sample): dot product, sigmoid, scaled copy of the feature row.
 __global__ void __launch_bounds__(256)
-logreg_grads_kernel(const float* __restrict__ A, const float* __restrict__ y, long long d,
+logreg_grads_kernel(const float* __restrict__ A, const float* __restrict__ y, long long n, long long d,
                     const int* __restrict__ idx, long long idx_stride, const float* __restrict__ X, int M,
                     long long b, float* __restrict__ G) {
   const long long w = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
@@ -35,7 +35,9 @@ logreg_grads_kernel(const float* __restrict__ A, const float* __restrict__ y, lo
   if (w >= static_cast<long long>(M) * b) return;
   const int m = static_cast<int>(w / b);
   const long long i = w % b;
-  const long long row = idx[static_cast<long long>(m) * idx_stride + i];
+  // indices outside the data are clamped, as in the fused rounds: never an out-of-range read
+  const long long raw = idx[static_cast<long long>(m) * idx_stride + i];
+  const long long row = raw < 0 ? 0 : (raw >= n ? n - 1 : raw);
   const float* a = A + row * d;
   const float* x = X + static_cast<long long>(m) * d;
   float z = 0.f;
@@ -68,7 +70,7 @@ extern "C" int abs_logreg_grads(abs_ctx* ctx, const float* A, const float* y, lo
   const long long warps = static_cast<long long>(M) * b;
   const long long blocks = (warps * 32 + 255) / 256;
   logreg_grads_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      A, y, d, idx, idx_stride, X, M, b, G);
+      A, y, n, d, idx, idx_stride, X, M, b, G);
   ABS_CUDA_TRY(ctx, cudaGetLastError());
   return ABS_OK;
 }
@@ -78,7 +80,7 @@ extern "C" int abs_logreg_grads(abs_ctx* ctx, const float* A, const float* y, lo
 extern "C" int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
                                 const int* idx, long long idx_stride, float* X, int M, int H, long long b, float lr,
                                 const abs_test_cfg* cfg, float* G_scratch, float* Gb_scratch, abs_stats* stats,
-                                long long* T_out, long long* b_dev, void* stream) {
+                                long long* T_out, long long* b_dev, abs_round_ctl* ctl, void* stream) {
   if (ctx == nullptr) return ABS_ERR_INVALID_ARG;
   if (cfg == nullptr || G_scratch == nullptr || Gb_scratch == nullptr || stats == nullptr || b_dev == nullptr)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
@@ -91,6 +93,10 @@ extern "C" int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, lo
     rc = abs_test_stats(ctx, G_scratch, ABS_F32, M, b, d, d, b * d, Gb_scratch, stats, stream);
     if (rc != ABS_OK) return rc;
     rc = local_sgd_step(ctx, X, Gb_scratch, M, d, d, lr, h == H - 1 ? 1 : 0, stream);
+    if (rc != ABS_OK) return rc;
+  }
+  if (ctl != nullptr) {      // Alg. 2: B <- B + H M b_k, k <- k + 1 (with the size the round ran with)
+    const int rc = abs_round_count(ctx, ctl, b_dev, 1, static_cast<long long>(H) * M, 1, stream);
     if (rc != ABS_OK) return rc;
   }
   return abs_next_batch(ctx, stats, M, cfg, b_dev, T_out, b_dev, stream);

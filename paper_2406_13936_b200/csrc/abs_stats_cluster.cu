@@ -39,6 +39,7 @@ struct ClusterParams {
   float* gbar_out;
   unsigned* flags;
   long long timeout_cycles;
+  int drop_loads;        // fault injection for the bounded waits: no tile load is issued
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -56,8 +57,10 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// RMAX: rows per thread and register set, exactly ceil(rows per CTA / row groups) (two sets
-// alternate); FULL: every thread of every CTA owns exactly RMAX rows, so nothing is predicated.
+// RMAX: rows per thread and register set, ceil(rows per CTA / row groups) (two sets alternate);
+// FULL: every thread of every CTA owns exactly RMAX rows, so nothing is predicated.  Otherwise
+// a thread owns n_rows_mine <= RMAX rows -- the cluster's last CTA holds b - (C-1)*RC rows, which
+// can be several row groups short of RC -- and every row index is checked against that count.
 template <typename T, int RMAX, bool FULL>
 __global__ void __launch_bounds__(kThreadsC, 1)
 abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const ClusterParams prm) {
@@ -93,8 +96,12 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
 
   const long long n_mine = (prm.n_iters > cl) ? (prm.n_iters - cl + prm.n_clusters - 1) / prm.n_clusters : 0;
 
-  // Loads tile i of this cluster (rows of this CTA) into its ring buffer; thread 0 only.
+  // Loads tile i of this cluster (rows of this CTA) into its ring buffer; thread 0 only.  After a
+  // wait has run out nothing more is issued, so the loads that were issued are a prefix 0..issued-1.
+  long long issued = 0;
   auto issue_load = [&](long long i) {
+    if (prm.drop_loads || *abort_flag) return;     // drop_loads: test hook, the waits must run out, not hang
+    ++issued;
     const int s = static_cast<int>(i % S);
     const uint32_t full = full_u32 + 8u * s;
     mbar_expect_tx(full, prm.stage_bytes);
@@ -124,7 +131,6 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
   const int RG = kCW * subs;                     // row groups
   const int rg = warp * subs + sub;
   const int n_rows_mine = (b_loc > rg) ? (b_loc - rg + RG - 1) / RG : 0;
-  const bool last_ok = n_rows_mine >= RMAX;       // RMAX is exactly ceil(RC / RG): only the last row can be missing
   const unsigned row_step = static_cast<unsigned>(RG) * row_bytes;
   const uint32_t my_off = static_cast<uint32_t>(rg) * row_bytes + static_cast<uint32_t>(cv) * 16u;
   const float inv_b = 1.0f / static_cast<float>(b);
@@ -150,7 +156,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
         // rows past the batch: safe address, zeroed by a select (no branch around the loads)
-        const bool ok = FULL || k < RMAX - 1 || last_ok;
+        const bool ok = FULL || k < n_rows_mine;
         uint4 u = lds128(ok ? base + static_cast<uint32_t>(k) * row_step : base0);
         if (!ok) u = make_uint4(0u, 0u, 0u, 0u);
         cur[k] = u;
@@ -235,7 +241,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
       for (int j = 0; j < VE; ++j) vl[j] = 0.f;
 #pragma unroll
       for (int k = 0; k < RMAX; ++k) {
-        const bool ok = FULL || k < RMAX - 1 || last_ok;
+        const bool ok = FULL || k < n_rows_mine;
         float x[VE];
         Vec<T>::unpack(prev[k], x);
         float ea = 0.f, eb = 0.f;
@@ -262,7 +268,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
         for (int k = 0; k < RMAX; ++k) {
           float ek = e[k];
           for (int off = 1; off < lpr; off <<= 1) ek += __shfl_xor_sync(0xffffffffu, ek, off);
-          if (cv == 0 && (FULL || k < RMAX - 1 || last_ok)) e_acc[rg + k * RG] += static_cast<double>(ek);
+          if (cv == 0 && (FULL || k < n_rows_mine)) e_acc[rg + k * RG] += static_cast<double>(ek);
           e[k] = 0.f;
         }
       }
@@ -295,6 +301,14 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
     out[b] = vs;
     out[b + 1] = ns;
     if (*abort_flag) atomicOr(prm.flags, 1u);
+    // Leave no copy in flight into this CTA's shared memory: every armed phase of the tile ring and
+    // of the exchange barriers must have completed before the CTA may exit.  Normally all of them
+    // have been waited for already; after a wait that ran out these are bounded waits of their own.
+    volatile unsigned ignore = 0u;
+    for (int s = 0; s < S && s < issued; ++s)
+      mbar_wait(full_u32 + 8u * s, static_cast<uint32_t>(((issued - 1 - s) / S) & 1), &ignore, prm.timeout_cycles);
+    for (int q = 0; q < kDepth && q < n_mine; ++q)
+      mbar_wait(xbar_u32 + 8u * q, static_cast<uint32_t>(((n_mine - 1 - q) / kDepth) & 1), &ignore, prm.timeout_cycles);
   }
   cluster_sync_all();      // nobody leaves while a peer could still address its shared memory
 }
@@ -419,6 +433,7 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
+  prm.drop_loads = ctx->tuning.stats_fault_drop_loads ? 1 : 0;
   const bool full = geo.full;
 #define ABS_CLUSTER_CASE(T, R) \
   case R: return launch_cluster_variant<T, R, false>(ctx, tmap, prm, a, C, smem, P_out);

@@ -140,7 +140,7 @@ constexpr int kFinalRowsPerCta = 64;      // at least this many rows per CTA (>=
 
 __global__ void __launch_bounds__(kFinalThreads)
 abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__ flags,
-                          unsigned* __restrict__ tickets, abs_stats* __restrict__ stats_out) {
+                          unsigned* __restrict__ tickets, abs_stats* __restrict__ stats_out, const Recheck rk) {
   __shared__ double red[4][kFinalThreads / 32];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m = blockIdx.x, y = blockIdx.y, nb = gridDim.y;
@@ -151,6 +151,8 @@ abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__
   const long long r_end = r_begin + rows_per < b ? r_begin + rows_per : b;
   pdl_wait();                    // the statistics kernel's partial records
   pdl_launch_dependents();
+  // the finalisation of a recomputation that was not needed: the records stand as they are
+  if (rk.second && *reinterpret_cast<volatile unsigned*>(rk.redo) == 0u) return;
   // Loads whose values are only needed at the end are issued here, so that they are in flight
   // while the rows are summed: the time-out flag, and the first V and N of every thread.
   unsigned timeout_word = 0u;
@@ -249,12 +251,20 @@ abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__
     const bool timed_out = timeout_word != 0u;
     // The last worker to get here clears the time-out flag (flags[0]) and the arrival counter
     // (flags[1]) for the next call, which saves a memset per call.
+    abs_stats rec = record_from_sums(V, N, s_e, s_ee, b, timed_out);
+    if (rk.second) rec.recomputed = 1u;
+    if (!rk.second && rk.redo != nullptr && (rec.status & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) == 0u) {
+      const double bd = static_cast<double>(b);
+      if (bd * N > rk.max_kv * (bd - 1.0) * rec.var_norm || N * N > rk.max_kip * rk.max_kip * rec.var_ip)
+        atomicOr(rk.redo, 1u);
+    }
     __threadfence();
     if (atomicAdd(flags + 1, 1u) == gridDim.x - 1) {
       flags[0] = 0u;
       flags[1] = 0u;
+      if (rk.second) *rk.redo = 0u;
     }
-    stats_out[m] = record_from_sums(V, N, s_e, s_ee, b, timed_out);
+    stats_out[m] = rec;
   }
 }
 
@@ -292,14 +302,14 @@ int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   return ABS_OK;
 }
 
-int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P) {
+int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P, const Recheck& rk) {
   // the rows of a worker are split over several CTAs when the context has a ticket word per worker
   long long nb = a.M <= ctx->ticket_slots ? a.b / kFinalRowsPerCta : 1;
   nb = nb < 1 ? 1 : (nb > kFinalMaxSplit ? kFinalMaxSplit : nb);
   while (nb > 1 && (nb - 1) * ((a.b + nb - 1) / nb) + 4 > a.b) --nb;     // the last CTA keeps at least 4 rows
   ABS_CUDA_TRY(ctx, launch_dependent(abs_stats_finalize_kernel, dim3(a.M, static_cast<unsigned>(nb)),
                                      dim3(kFinalThreads), 0, a.stream, static_cast<double*>(ctx->workspace), a.b, P,
-                                     ctx->flags, ctx->flags + kFlagWords, a.stats_out));
+                                     ctx->flags, ctx->flags + kFlagWords, a.stats_out, rk));
   return ABS_OK;
 }
 

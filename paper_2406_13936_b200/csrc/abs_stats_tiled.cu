@@ -49,6 +49,7 @@ struct TiledParams {
   int drop_loads;        // fault injection for the bounded waits: the loader issues nothing
   int boxes_per_copy;    // neighbouring boxes that one copy brings in as one tile row: 1; 2, 4 or 8 for very small batches
   int segment_map;       // the tensor map is the 4-D segment map (x counted in segments of 256 elements)
+  const unsigned* guard; // NULL, or a device word: while it is zero the kernel has nothing to do
 };
 
 // ---- the kernel ----------------------------------------------------------------------------
@@ -61,6 +62,8 @@ __global__ void __launch_bounds__(kThreads, (RMAX <= 8 ? 2 : 1))
 abs_stats_tiled_kernel(const __grid_constant__ CUtensorMap tmap, const TiledParams prm) {
   constexpr int VE = Vec<T>::VE;
   extern __shared__ __align__(128) unsigned char smem_raw[];
+  // a recomputation that the finalisation before this launch did not ask for
+  if (prm.guard != nullptr && *reinterpret_cast<const volatile unsigned*>(prm.guard) == 0u) return;
 
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -461,6 +464,15 @@ int plan_stats_tiled(const Tuning& t, size_t smem_optin, abs_dtype dtype, long l
   return ABS_OK;
 }
 
+bool stats_tiled_feasible(abs_ctx* ctx, const StatsLaunch& a) {
+  if (a.b > kMaxFastRows || !tma_addressable(a)) return false;
+  TileChoice c;
+  if (!tiled_choice(ctx->tuning, ctx->smem_optin, a.dtype == ABS_F32 ? 4 : 8, a.b, &c)) return false;
+  // the launcher never uses more than two CTAs per SM
+  const size_t worst = static_cast<size_t>(ctx->sm_count) * 2 + static_cast<size_t>(a.M);
+  return worst * (a.b + 2) * sizeof(double) <= ctx->workspace_bytes;
+}
+
 int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   const int es = a.dtype == ABS_F32 ? 4 : 2;
   const int ve = 16 / es;
@@ -525,6 +537,7 @@ int launch_stats_tiled(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   prm.drop_loads = ctx->tuning.stats_fault_drop_loads ? 1 : 0;
   prm.boxes_per_copy = boxes_per_copy;
   prm.segment_map = segment_map;
+  prm.guard = a.guard;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
 
   const dim3 grid(static_cast<unsigned>(P), static_cast<unsigned>(a.M));

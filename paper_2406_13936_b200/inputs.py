@@ -71,10 +71,14 @@ def student_t_rows(seed, M, b, d, scale=1e-3, dof=3, mean_frac=0.1, device="cpu"
 
 
 def tile_columns(small, d):
-    """Repeat the columns of small[..., d0] periodically up to width d."""
+    """Repeat the columns of small[..., d0] periodically up to width d.  The result is allocated
+    once and filled period by period, so a 100 GB tensor needs no second copy of itself."""
     d0 = small.shape[-1]
-    reps = (d + d0 - 1) // d0
-    return small.repeat(*([1] * (small.dim() - 1)), reps)[..., :d].contiguous()
+    out = torch.empty(tuple(small.shape[:-1]) + (d,), device=small.device, dtype=small.dtype)
+    for lo in range(0, d, d0):
+        w = min(d0, d - lo)
+        out[..., lo:lo + w].copy_(small[..., :w])
+    return out
 
 
 def adamw_problem(seed, M, d, pool=4, x_std=0.02, grad_std=0.01, device="cpu"):

@@ -42,6 +42,8 @@ def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(binding.Stats) == 56
     assert ctypes.sizeof(binding.TestCfg) == 56
     assert ctypes.sizeof(binding.AdamWCfg) == 32
+    assert ctypes.sizeof(binding.RoundCtl) == 32
+    assert ctypes.sizeof(binding.RoundOpts) == 24
 
 
 def test_create_fails_loudly_without_a_device():

@@ -216,6 +216,30 @@ def test_fused_rounds_in_one_launch_equal_one_launch_per_round(ctx):
         params_close(X3, f64(X1), tol=1e-5)
 
 
+@pytest.mark.parametrize("M,d,b0,b_max", [(16, 64, 4, 64), (8, 256, 8, 128), (40, 128, 3, 48)])
+def test_fused_rounds_with_one_step_per_round_and_many_workers(ctx, M, d, b0, b_max):
+    """H = 1 leaves the least work between two rounds' exchanges through global memory (a fast
+    worker could be a round ahead of a slow reader, which is why the exchange buffers alternate by
+    round): many rounds in one launch must equal one launch per round bit for bit, repeatedly."""
+    n, H, lr, rounds = 4096, 1, 0.1, 40
+    A, y = inputs.logreg_dataset(5, n, d, device="cuda")
+    idx = inputs.batch_indices(12, (rounds, H, M, b_max), n, device="cuda")
+    tcfg = pkg.make_test_cfg("norm", b_max, eta=0.6)
+    X2 = torch.zeros((M, d), device="cuda")
+    stats2 = ctx.new_stats(rounds * M)
+    b2 = torch.tensor([b0], dtype=torch.int64, device="cuda")
+    for k in range(rounds):
+        ctx.abs_logreg_rounds_fused(A, y, idx[k:k + 1], X2, H, lr, tcfg, stats2[k * M:(k + 1) * M], b2)
+    torch.cuda.synchronize()
+    for _ in range(5):
+        X1 = torch.zeros((M, d), device="cuda")
+        stats1 = ctx.new_stats(rounds * M)
+        b1 = torch.tensor([b0], dtype=torch.int64, device="cuda")
+        ctx.abs_logreg_rounds_fused(A, y, idx, X1, H, lr, tcfg, stats1, b1)
+        torch.cuda.synchronize()
+        assert torch.equal(X1, X2) and torch.equal(stats1, stats2) and int(b1.item()) == int(b2.item())
+
+
 def test_fused_rounds_wait_that_runs_out_is_reported_and_the_context_stays_usable(ctx):
     """Failure detection without a fault: with the partial gradients not sent (test hook) every CTA's
     wait for its peers gives up after the shortened limit, the launch still reaches all its barriers

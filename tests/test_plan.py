@@ -46,7 +46,9 @@ def check_plan(dtype, b, p):
     assert R * groups >= p["rows_per_cta"]
     if p["keep_in_registers"]:
         assert R <= 16
-        assert (R - 1) * groups < p["rows_per_cta"]          # only the last row of a thread may be missing
+        if p["route"] == 2:
+            # the single-CTA kernel predicates only a thread's last row: all others must exist
+            assert (R - 1) * groups < b
     else:
         assert R <= 32
     if p["full"]:
