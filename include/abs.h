@@ -190,7 +190,10 @@ int abs_test_stats_host(abs_ctx* ctx, const void* G_host, abs_dtype dtype, int M
  * device.  Some callers cannot accept that: programs whose device memory is handed
  * out entirely by their own pool, plug-ins that run under a fixed memory budget,
  * latency-critical sections that must not hit an implicit device synchronisation.
- * For them this call computes exactly what abs_test_stats computes, takes no
+ * For them this call computes the same statistics as abs_test_stats (the same
+ * records up to floating-point rounding: it only uses the tiled kernel and the
+ * alignment-free kernel, so bf16 input with b <= 256 and any input with b > 256
+ * take another, slower kernel than in the context call), takes no
  * context, and keeps its scratch (per-CTA partial sums and a status word) in a
  * fixed array of ABS_NOALLOC_SCRATCH_BYTES + 256 bytes that is part of the library
  * image: every GPU on which the library is loaded holds that array until the

@@ -5,8 +5,10 @@ own, or they are inside a section that must not meet the device-wide synchronisa
 cudaMalloc.  abs_test_stats_noalloc serves them with a fixed scratch array inside the library.
 This test calls it through the C ABI twice in a row (the second call finds the first call's
 partial sums still in the array) and compares each result with abs_test_stats on the same input.
-Both entry points launch the same kernels in the same configuration, so the records agree to the
-last bit; the check allows the suite's fp32 tolerance of 1e-5 all the same.  It also checks that
+The allocation-free call only has the tiled and the alignment-free kernel, so for bf16 rows with
+b <= 256 and for any b > 256 (the second case below) the two entry points run different kernels
+and agree to rounding, not to the bit: the check uses the suite's tolerances, 1e-5 for fp32 and
+1e-3 for bf16 input.  It also checks that
 device memory in use does not change across a call (once the first call has made the runtime
 place the fixed array on the GPU) and that oversize problems are refused.
 The file sorts last so that a failure here cannot hide the results of the other tests.
