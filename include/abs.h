@@ -88,6 +88,10 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_cluster_rows" (target rows per CTA of the cluster kernel, 16..512),
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
  * cluster when b > 256),
+ * "stats_no_secondary" (1 = the cluster kernel leaves the SMs idle that its
+ * clusters cannot occupy instead of giving them a second launch of two-CTA
+ * clusters), "stats_secondary_pct" (the speed of an SM of that second launch in
+ * per cent of an SM of the first, which sets its share of the columns; 0 = 95),
  * "stats_no_gram" (1 = do not use the tensor-core Gram kernels for bf16, b <= 256),
  * "stats_no_recheck" (1 = keep a Gram kernel's record even when its sums are
  * ill-conditioned, i.e. never recompute it with the tiled kernel),

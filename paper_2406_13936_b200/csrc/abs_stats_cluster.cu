@@ -32,8 +32,12 @@ struct ClusterParams {
   int stages;
   int box_rows, n_row_boxes;
   unsigned stage_bytes;  // rows_pad * lpr * 16
-  long long n_iters;     // column strips per worker
-  int n_clusters;        // clusters per worker
+  long long col_begin;   // first column of this launch's share of the row (a multiple of the strip width)
+  long long n_iters;     // column strips of that share, per worker
+  int n_clusters;        // clusters per worker in this launch
+  int rec_base;          // first partial record of this launch (a second launch appends its records)
+  int rec_total;         // partial records per worker over all launches
+  int wait_primary;      // this launch runs beside the one before it in the stream: wait for that one before exit
   int flush_every;
   double* ws;
   float* gbar_out;
@@ -105,7 +109,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
     const int s = static_cast<int>(i % S);
     const uint32_t full = full_u32 + 8u * s;
     mbar_expect_tx(full, prm.stage_bytes);
-    const long long x = (cl + i * prm.n_clusters) * cols;
+    const long long x = prm.col_begin + (cl + i * prm.n_clusters) * cols;
     const uint32_t dst0 = stage_u32 + static_cast<uint32_t>(s) * prm.stage_bytes;
     for (int rb = 0; rb < prm.n_row_boxes; ++rb)
       tma_load_3d(dst0 + static_cast<uint32_t>(rb * prm.box_rows) * row_bytes, &tmap, static_cast<int>(x),
@@ -222,7 +226,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
         for (int j = 0; j < VE; ++j) nl = fmaf(g[j], g[j], nl);
         nacc += static_cast<double>(nl);
         if (prm.gbar_out != nullptr) {
-          const long long col = ((cl + t * prm.n_clusters) * static_cast<long long>(lpr) + cv) * VE;
+          const long long col = prm.col_begin + ((cl + t * prm.n_clusters) * static_cast<long long>(lpr) + cv) * VE;
           float* dst = prm.gbar_out + static_cast<long long>(m) * prm.d + col;
           if (col + VE <= prm.d && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
 #pragma unroll
@@ -287,7 +291,7 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
     red[kCW + warp] = nacc;
   }
   __syncthreads();
-  double* out = prm.ws + (static_cast<size_t>(m) * gridDim.x + blockIdx.x) * (static_cast<size_t>(b) + 2);
+  double* out = prm.ws + (static_cast<size_t>(m) * prm.rec_total + prm.rec_base + blockIdx.x) * (static_cast<size_t>(b) + 2);
   for (int r = tid; r < b; r += kThreadsC) {
     const int loc = r - row0;
     out[r] = (loc >= 0 && loc < b_loc) ? e_acc[loc] : 0.0;     // rows of other CTAs: their records carry them
@@ -311,11 +315,22 @@ abs_stats_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Cluster
       mbar_wait(xbar_u32 + 8u * q, static_cast<uint32_t>(((n_mine - 1 - q) / kDepth) & 1), &ignore, prm.timeout_cycles);
   }
   cluster_sync_all();      // nobody leaves while a peer could still address its shared memory
+  // A launch that ran beside its predecessor (on the SMs that one cannot use) must not complete before
+  // it: the finalisation waits for this grid only.
+  if (prm.wait_primary) pdl_wait();
 }
+
+// What one launch of the kernel covers.  n_clusters == 0 asks only how many clusters of this size
+// can be resident at once (*max_clusters_out), without launching.
+struct ClusterShare {
+  int n_clusters = 0;
+  bool beside_previous = false;   // programmatic dependent launch that starts while the launch before it runs
+  int* max_clusters_out = nullptr;
+};
 
 template <typename T, int RMAX, bool FULL>
 int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams prm, const StatsLaunch& a, int C,
-                           size_t smem, int* records_out) {
+                           size_t smem, const ClusterShare& share) {
   auto kern = abs_stats_cluster_kernel<T, RMAX, FULL>;
   ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   if (C > 8 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
@@ -323,38 +338,34 @@ int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams 
     return ABS_ERR_UNSUPPORTED;
   }
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = static_cast<unsigned>(C);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.blockDim = dim3(kThreadsC);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = a.stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cfg.gridDim = dim3(static_cast<unsigned>(C), 1, 1);
-  int max_clusters = 0;
-  const cudaError_t occ = cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg);
-  if (occ != cudaSuccess || max_clusters < 1) {
-    cudaGetLastError();
-    set_error(ctx, ABS_ERR_UNSUPPORTED, "a cluster of %d CTAs cannot be scheduled (%s, %d clusters)", C,
-              cudaGetErrorString(occ), max_clusters);
-    return ABS_ERR_UNSUPPORTED;
+  cfg.numAttrs = share.beside_previous ? 2 : 1;
+  if (share.n_clusters == 0) {
+    cfg.gridDim = dim3(static_cast<unsigned>(C), 1, 1);
+    cfg.numAttrs = 1;
+    int max_clusters = 0;
+    const cudaError_t occ = cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg);
+    if (occ != cudaSuccess || max_clusters < 1) {
+      cudaGetLastError();
+      set_error(ctx, ABS_ERR_UNSUPPORTED, "a cluster of %d CTAs cannot be scheduled (%s, %d clusters)", C,
+                cudaGetErrorString(occ), max_clusters);
+      return ABS_ERR_UNSUPPORTED;
+    }
+    *share.max_clusters_out = max_clusters;
+    return ABS_OK;
   }
-  long long n_clusters = ctx->tuning.stats_ctas_per_worker > 0 ? ctx->tuning.stats_ctas_per_worker
-                                                               : static_cast<long long>(max_clusters) / a.M;
-  if (n_clusters < 1) n_clusters = 1;
-  if (n_clusters > prm.n_iters) n_clusters = prm.n_iters;
-  if (n_clusters * C > 65535) n_clusters = 65535 / C;
-  const size_t need = static_cast<size_t>(a.M) * n_clusters * C * (a.b + 2) * sizeof(double);
-  if (need > ctx->workspace_bytes)
-    return set_error(ctx, ABS_ERR_WORKSPACE, "abs_test_stats needs %zu workspace bytes, context has %zu", need,
-                     ctx->workspace_bytes);
-  prm.n_clusters = static_cast<int>(n_clusters);
-  cfg.gridDim = dim3(static_cast<unsigned>(n_clusters * C), static_cast<unsigned>(a.M), 1);
+  cfg.gridDim = dim3(static_cast<unsigned>(share.n_clusters * C), static_cast<unsigned>(a.M), 1);
   ABS_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, kern, tmap, prm));
-  *records_out = static_cast<int>(n_clusters * C);
   return ABS_OK;
 }
 
@@ -403,56 +414,129 @@ int preferred_cluster_size(const Tuning& t, long long b) {
   return C;
 }
 
-// One attempt with a given cluster size; ABS_ERR_UNSUPPORTED if that size cannot be used.
-int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
-  ClusterGeom geo;
-  if (!cluster_geometry(ctx->tuning, ctx->smem_optin, a.dtype == ABS_F32 ? 4 : 2, a.b, C, &geo))
-    return ABS_ERR_UNSUPPORTED;
-  const int RC = geo.RC, lpr_log2 = geo.lpr_log2, rmax = geo.rmax, n_row_boxes = geo.n_row_boxes;
-  const int box_rows = geo.box_rows, stages = geo.stages, cols = geo.cols;
-  const unsigned stage_bytes = geo.stage_bytes;
-  const size_t smem = geo.smem;
-
+// One launch (or one occupancy query) of the variant that fits the geometry.
+int cluster_dispatch(abs_ctx* ctx, const StatsLaunch& a, int C, const ClusterGeom& geo, ClusterParams prm,
+                     const ClusterShare& share) {
   CUtensorMap tmap;
-  int rc = encode_g_tensor_map(ctx, a, cols, box_rows, &tmap);
+  int rc = encode_g_tensor_map(ctx, a, geo.cols, geo.box_rows, &tmap);
   if (rc != ABS_OK) return rc;
-
-  ClusterParams prm;
   prm.b = a.b;
   prm.d = a.d;
-  prm.rows_per_cta = RC;
-  prm.lpr_log2 = lpr_log2;
-  prm.stages = stages;
-  prm.box_rows = box_rows;
-  prm.n_row_boxes = n_row_boxes;
-  prm.stage_bytes = stage_bytes;
-  prm.n_iters = (a.d + cols - 1) / cols;
-  prm.n_clusters = 1;
+  prm.rows_per_cta = geo.RC;
+  prm.lpr_log2 = geo.lpr_log2;
+  prm.stages = geo.stages;
+  prm.box_rows = geo.box_rows;
+  prm.n_row_boxes = geo.n_row_boxes;
+  prm.stage_bytes = geo.stage_bytes;
   prm.flush_every = static_cast<int>(ctx->tuning.stats_flush_every > 0 ? ctx->tuning.stats_flush_every : 64);
   prm.ws = static_cast<double*>(ctx->workspace);
   prm.gbar_out = a.gbar_out;
   prm.flags = ctx->flags;
   prm.timeout_cycles = ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles;
   prm.drop_loads = ctx->tuning.stats_fault_drop_loads ? 1 : 0;
+  prm.n_clusters = share.n_clusters;
+  prm.wait_primary = share.beside_previous ? 1 : 0;
+  const int rmax = geo.rmax;
+  const size_t smem = geo.smem;
   const bool full = geo.full;
 #define ABS_CLUSTER_CASE(T, R) \
-  case R: return launch_cluster_variant<T, R, false>(ctx, tmap, prm, a, C, smem, P_out);
+  case R: return launch_cluster_variant<T, R, false>(ctx, tmap, prm, a, C, smem, share);
 #define ABS_CLUSTER_DISPATCH(T)                                                                        \
   if (full) {                                                                                          \
-    return rmax == 8 ? launch_cluster_variant<T, 8, true>(ctx, tmap, prm, a, C, smem, P_out)           \
-                     : launch_cluster_variant<T, 16, true>(ctx, tmap, prm, a, C, smem, P_out);         \
+    return rmax == 8 ? launch_cluster_variant<T, 8, true>(ctx, tmap, prm, a, C, smem, share)           \
+                     : launch_cluster_variant<T, 16, true>(ctx, tmap, prm, a, C, smem, share);         \
   }                                                                                                    \
   switch (rmax) {                                                                                      \
     ABS_CLUSTER_CASE(T, 1) ABS_CLUSTER_CASE(T, 2) ABS_CLUSTER_CASE(T, 3) ABS_CLUSTER_CASE(T, 4)        \
     ABS_CLUSTER_CASE(T, 5) ABS_CLUSTER_CASE(T, 6) ABS_CLUSTER_CASE(T, 7) ABS_CLUSTER_CASE(T, 8)        \
     ABS_CLUSTER_CASE(T, 9) ABS_CLUSTER_CASE(T, 10) ABS_CLUSTER_CASE(T, 11) ABS_CLUSTER_CASE(T, 12)     \
     ABS_CLUSTER_CASE(T, 13) ABS_CLUSTER_CASE(T, 14) ABS_CLUSTER_CASE(T, 15)                            \
-    default: return launch_cluster_variant<T, 16, false>(ctx, tmap, prm, a, C, smem, P_out);           \
+    default: return launch_cluster_variant<T, 16, false>(ctx, tmap, prm, a, C, smem, share);           \
   }
   if (a.dtype == ABS_F32) { ABS_CLUSTER_DISPATCH(float) }
   ABS_CLUSTER_DISPATCH(__nv_bfloat16)
 #undef ABS_CLUSTER_DISPATCH
 #undef ABS_CLUSTER_CASE
+}
+
+// One attempt with a given cluster size; ABS_ERR_UNSUPPORTED if that size cannot be used.
+//
+// Clusters of C CTAs cannot be placed on every SM (a cluster lives inside one GPC, and a GPC's SM
+// count need not be a multiple of C: 33 clusters of 4 occupy 132 of 148 SMs).  The SMs that are left
+// over come in pairs, so a second launch of the same kernel with clusters of two CTAs (twice the
+// rows per CTA, half the row width) takes a share of the columns of its own: it is enqueued as a
+// programmatic dependent of the first launch, starts as soon as that one is resident, finds only
+// the left-over SMs free, and waits for the first launch before it completes.  Its partial records
+// follow the first launch's in the workspace, and the finalisation folds them all.
+int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
+  const int es = a.dtype == ABS_F32 ? 4 : 2;
+  ClusterGeom geo;
+  if (!cluster_geometry(ctx->tuning, ctx->smem_optin, es, a.b, C, &geo)) return ABS_ERR_UNSUPPORTED;
+  int max_clusters = 0;
+  ClusterShare query;
+  query.max_clusters_out = &max_clusters;
+  int rc = cluster_dispatch(ctx, a, C, geo, ClusterParams(), query);
+  if (rc != ABS_OK) return rc;
+
+  const long long strips = (a.d + geo.cols - 1) / geo.cols;
+  long long n1 = ctx->tuning.stats_ctas_per_worker > 0 ? ctx->tuning.stats_ctas_per_worker
+                                                       : static_cast<long long>(max_clusters) / a.M;
+  if (n1 < 1) n1 = 1;
+  if (n1 > strips) n1 = strips;
+  if (n1 * C > 65535) n1 = 65535 / C;
+
+  // the second launch: clusters of two on the SMs the first cannot use
+  ClusterGeom geo2;
+  long long n2 = 0, cols_second = 0;
+  const long long idle = ctx->sm_count - n1 * a.M * C;
+  if (C > 2 && !ctx->tuning.stats_no_secondary && ctx->tuning.stats_ctas_per_worker == 0 && idle >= 2 &&
+      n1 * a.M == (static_cast<long long>(max_clusters) / a.M) * a.M &&
+      cluster_geometry(ctx->tuning, ctx->smem_optin, es, a.b, 2, &geo2)) {
+    n2 = (idle / 2) / a.M;
+    // its share of the columns: in proportion to its SMs, each counted at `pct` per cent of an SM of
+    // the first launch (measured: the two finish together at about 100, and every per cent beyond
+    // that costs a per cent of the whole call, so the default stays a little below); at least 64
+    // strips per cluster
+    const long long pct = ctx->tuning.stats_secondary_pct > 0 ? ctx->tuning.stats_secondary_pct : 95;
+    const double w2 = static_cast<double>(n2 * 2) * pct / 100.0;
+    cols_second = static_cast<long long>(static_cast<double>(a.d) * w2 / (static_cast<double>(n1 * C) + w2));
+    if (n2 < 1 || cols_second < 64 * n2 * geo2.cols) n2 = 0;
+  }
+  long long cols_first = a.d;
+  if (n2 > 0) {
+    cols_first = (a.d - cols_second) / geo.cols * geo.cols;      // whole strips of the first launch
+    if (cols_first <= 0 || cols_first >= a.d) n2 = 0, cols_first = a.d;
+  }
+  const long long strips1 = (cols_first + geo.cols - 1) / geo.cols;
+  if (n1 > strips1) n1 = strips1;
+  const long long strips2 = n2 > 0 ? (a.d - cols_first + geo2.cols - 1) / geo2.cols : 0;
+  const long long records = n1 * C + n2 * 2;
+  const size_t need = static_cast<size_t>(a.M) * records * (a.b + 2) * sizeof(double);
+  if (need > ctx->workspace_bytes)
+    return set_error(ctx, ABS_ERR_WORKSPACE, "abs_test_stats needs %zu workspace bytes, context has %zu", need,
+                     ctx->workspace_bytes);
+
+  ClusterParams prm;
+  prm.col_begin = 0;
+  prm.n_iters = strips1;
+  prm.rec_base = 0;
+  prm.rec_total = static_cast<int>(records);
+  ClusterShare first;
+  first.n_clusters = static_cast<int>(n1);
+  rc = cluster_dispatch(ctx, a, C, geo, prm, first);
+  if (rc != ABS_OK) return rc;
+  if (n2 > 0) {
+    prm.col_begin = cols_first;
+    prm.n_iters = strips2;
+    prm.rec_base = static_cast<int>(n1 * C);
+    ClusterShare second;
+    second.n_clusters = static_cast<int>(n2);
+    second.beside_previous = true;
+    rc = cluster_dispatch(ctx, a, 2, geo2, prm, second);
+    if (rc != ABS_OK) return rc;
+  }
+  *P_out = static_cast<int>(records);
+  return ABS_OK;
 }
 
 }  // namespace

@@ -348,6 +348,40 @@ def test_mlp_fused_statistics_match_materialised_gradients(ctx, dims, M, b):
         assert abs(f["var_orth"] - r["var_orth"]) <= 2e-5 * r["var_norm"]
 
 
+@pytest.mark.parametrize("b", [32, 600])
+def test_mlp_fused_statistics_against_the_oracle_at_full_network_size(ctx, b):
+    """784-1024-1024-10: the statistics formed from activations and deltas (no gradient matrix)
+    against the oracle, two ways.  (i) Same inputs: the oracle's definitions applied to the very
+    per-sample gradient rows the GPU can write out, at 2e-5 (the expansion sum_i ||g_i||^2 - b N and
+    the fp32 layer products are what separates the two).  (ii) The whole pipeline: the oracle's own
+    fp64 forward/backward per sample, at 2e-4 (fp32 against fp64 producers)."""
+    dims, n = (784, 1024, 1024, 10), 8192
+    inp, lab, X = mlp_problem(5, n, dims, 1)
+    X += 0.02 * torch.randn(X.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(9))
+    d = ctx.mlp_param_count(dims)
+    idx = inputs.batch_indices(6, (1, b), n, device="cuda")
+    scratch = ctx.mlp_scratch(1, b, dims)
+    Gb = torch.empty((1, d), device="cuda")
+    ctx.abs_mlp_grads(inp, lab, dims, idx, X, b, Gb, scratch)
+    fused = ctx.new_stats(1)
+    ctx.abs_mlp_fused_stats(dims, b, scratch, Gb, fused)
+    stride = (d + 3) // 4 * 4
+    G = torch.zeros((b, stride), device="cuda")
+    ctx.abs_mlp_per_sample(dims, b, 0, scratch, G)
+    torch.cuda.synchronize()
+    rec = pkg.stats_to_dicts(fused)[0]
+    assert rec["rows"] == b and rec["status"] == 0
+    same_inputs = orc.batch_test_stats(f64(G[:, :d]))
+    rows = idx[0].cpu().numpy()
+    pipeline = orc.batch_test_stats(orc.mlp_per_sample_grads(f64(inp)[rows], lab.cpu().numpy()[rows], f64(X[0]), dims))
+    for ref, tol in ((same_inputs, 2e-5), (pipeline, 2e-4)):
+        for key in ("gbar_sq", "var_norm", "var_ip", "sum_sq"):
+            assert rec[key] == pytest.approx(ref[key], rel=tol)
+        orth_decides = ref["var_orth"] * ref["gbar_sq"] >= ref["var_ip"]
+        assert abs(rec["var_orth"] - ref["var_orth"]) <= tol * (ref["var_orth"] if orth_decides else ref["var_norm"])
+    np.testing.assert_allclose(f64(Gb[0]), pipeline["gbar"], rtol=0, atol=1e-5 * np.abs(pipeline["gbar"]).max())
+
+
 def run_mlp_rounds(ctx, dims, n, M, H, lr, b, b_max, rounds, check_rounds, theta=0.5, nu=0.5, seed=5, fused=False):
     """Runs `rounds` rounds on the GPU; the first `check_rounds` are compared with the oracle."""
     inp, lab, X = mlp_problem(seed, n, dims, M)
@@ -403,9 +437,12 @@ def test_mlp_rounds_small_network_teacher_forced(ctx, fused):
     assert torch.equal(X[0], X[7])
 
 
-def test_mlp_rounds_full_network_first_rounds(ctx):
-    # the 784-1024-1024-10 classifier with two workers: the oracle is too slow for more
-    run_mlp_rounds(ctx, (784, 1024, 1024, 10), n=8192, M=2, H=4, lr=0.01, b=32, b_max=4096, rounds=2, check_rounds=2)
+@pytest.mark.parametrize("fused", [False, True])
+def test_mlp_rounds_full_network_first_rounds(ctx, fused):
+    # the 784-1024-1024-10 classifier with all eight workers, three teacher-forced rounds (the oracle
+    # runs M H b backward passes of a 1.9 M-parameter network per round)
+    run_mlp_rounds(ctx, (784, 1024, 1024, 10), n=8192, M=8, H=4, lr=0.01, b=32, b_max=4096, rounds=3, check_rounds=3,
+                   fused=fused)
 
 
 def mlp_loss(ctx, inp, lab, x, dims):

@@ -491,7 +491,9 @@ def test_largest_sweep_cell_through_periodic_columns(ctx):
     check_record(recs[0], ref, 1e-5, b)
     np.testing.assert_allclose(gbar[0, :d0].cpu().numpy(), ref["gbar"], rtol=1e-5, atol=1e-6 * np.abs(ref["gbar"]).max())
     K = d // d0
-    assert torch.equal(gbar[0, (K - 1) * d0:K * d0], gbar[0, :d0])           # the last whole period
+    # the last whole period (it may come from the second launch, which adds the rows in another order)
+    np.testing.assert_allclose(gbar[0, (K - 1) * d0:K * d0].cpu().numpy(), gbar[0, :d0].cpu().numpy(), rtol=1e-5,
+                               atol=1e-6 * np.abs(ref["gbar"]).max())
 
 
 @pytest.mark.parametrize("ratio", [10.0, 30.0, 100.0])
