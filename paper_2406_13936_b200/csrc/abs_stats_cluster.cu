@@ -463,7 +463,7 @@ int cluster_dispatch(abs_ctx* ctx, const StatsLaunch& a, int C, const ClusterGeo
 //
 // Clusters of C CTAs cannot be placed on every SM (a cluster lives inside one GPC, and a GPC's SM
 // count need not be a multiple of C: 33 clusters of 4 occupy 132 of 148 SMs).  The SMs that are left
-// over come in pairs, so a second launch of the same kernel with clusters of two CTAs (twice the
+// over come in pairs, so a second launch of the same kernel with clusters of half the size (twice the
 // rows per CTA, half the row width) takes a share of the columns of its own: it is enqueued as a
 // programmatic dependent of the first launch, starts as soon as that one is resident, finds only
 // the left-over SMs free, and waits for the first launch before it completes.  Its partial records
@@ -489,16 +489,20 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   ClusterGeom geo2;
   long long n2 = 0, cols_second = 0;
   const long long idle = ctx->sm_count - n1 * a.M * C;
-  if (C > 2 && !ctx->tuning.stats_no_secondary && ctx->tuning.stats_ctas_per_worker == 0 && idle >= 2 &&
+  // Only pairs are known to fit what four-CTA clusters leave over; clusters of four beside clusters
+  // of eight were tried (b = 2048) and mostly ran after the first launch instead of beside it:
+  // 6.7 -> 8.8 ms.
+  const int C2 = 2;
+  if (C == 4 && !ctx->tuning.stats_no_secondary && ctx->tuning.stats_ctas_per_worker == 0 && idle >= C2 &&
       n1 * a.M == (static_cast<long long>(max_clusters) / a.M) * a.M &&
-      cluster_geometry(ctx->tuning, ctx->smem_optin, es, a.b, 2, &geo2)) {
-    n2 = (idle / 2) / a.M;
+      cluster_geometry(ctx->tuning, ctx->smem_optin, es, a.b, C2, &geo2)) {
+    n2 = (idle / C2) / a.M;
     // its share of the columns: in proportion to its SMs, each counted at `pct` per cent of an SM of
     // the first launch (measured: the two finish together at about 100, and every per cent beyond
     // that costs a per cent of the whole call, so the default stays a little below); at least 64
     // strips per cluster
     const long long pct = ctx->tuning.stats_secondary_pct > 0 ? ctx->tuning.stats_secondary_pct : 95;
-    const double w2 = static_cast<double>(n2 * 2) * pct / 100.0;
+    const double w2 = static_cast<double>(n2 * C2) * pct / 100.0;
     cols_second = static_cast<long long>(static_cast<double>(a.d) * w2 / (static_cast<double>(n1 * C) + w2));
     if (n2 < 1 || cols_second < 64 * n2 * geo2.cols) n2 = 0;
   }
@@ -510,7 +514,7 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   const long long strips1 = (cols_first + geo.cols - 1) / geo.cols;
   if (n1 > strips1) n1 = strips1;
   const long long strips2 = n2 > 0 ? (a.d - cols_first + geo2.cols - 1) / geo2.cols : 0;
-  const long long records = n1 * C + n2 * 2;
+  const long long records = n1 * C + n2 * C2;
   const size_t need = static_cast<size_t>(a.M) * records * (a.b + 2) * sizeof(double);
   if (need > ctx->workspace_bytes)
     return set_error(ctx, ABS_ERR_WORKSPACE, "abs_test_stats needs %zu workspace bytes, context has %zu", need,
@@ -532,7 +536,7 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
     ClusterShare second;
     second.n_clusters = static_cast<int>(n2);
     second.beside_previous = true;
-    rc = cluster_dispatch(ctx, a, 2, geo2, prm, second);
+    rc = cluster_dispatch(ctx, a, C2, geo2, prm, second);
     if (rc != ABS_OK) return rc;
   }
   *P_out = static_cast<int>(records);
