@@ -28,7 +28,7 @@ HP = dict(lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) of one abs_stats_tiled_kernel<float,16,keep,full> launch on the 1.024 GB case
 # of profiles/stats_tiled_f32_b256_d1m.txt; traffic grows in proportion to the columns processed.
-NCU_TRAFFIC_SMALL = dict(dram_bytes=1.024042e9 + 4.618e6, d=1_000_000)
+NCU_TRAFFIC_SMALL = dict(dram_bytes=1.024040e9 + 3.832e6, d=1_000_000)
 
 
 def measured_peak():
