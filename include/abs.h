@@ -88,6 +88,8 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_cluster_rows" (target rows per CTA of the cluster kernel, 16..512),
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block
  * cluster when b > 256),
+ * "mlp_no_tensor_cores" (1 = the matrix products of the MLP producer run on the
+ * CUDA cores in fp32 with fp64 folding instead of on the tensor cores),
  * "stats_no_secondary" (1 = the cluster kernel leaves the SMs idle that its
  * clusters cannot occupy instead of giving them a second launch of two-CTA
  * clusters), "stats_secondary_pct" (the speed of an SM of that second launch in

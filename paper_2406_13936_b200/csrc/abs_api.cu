@@ -178,6 +178,8 @@ extern "C" int abs_set_tuning(abs_ctx* ctx, const char* key, long long value) {
     if (value != 0 && (value < 100000 || value > 4000000000ll))
       return set_error(ctx, ABS_ERR_INVALID_ARG, "stats_timeout_cycles must be 0 or 1e5..4e9");
     ctx->tuning.stats_timeout_cycles = value;
+  } else if (strcmp(key, "mlp_no_tensor_cores") == 0) {
+    ctx->tuning.mlp_no_tensor_cores = value ? 1 : 0;
   } else if (strcmp(key, "stats_no_secondary") == 0) {
     ctx->tuning.stats_no_secondary = value ? 1 : 0;
   } else if (strcmp(key, "stats_secondary_pct") == 0) {

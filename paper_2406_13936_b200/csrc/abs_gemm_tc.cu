@@ -1,0 +1,391 @@
+// The MLP producer's batched GEMM on the tcgen05 tensor cores (sm_100a): C = epilogue(A B) for
+// fp32 operands with fp32-grade accuracy.
+//
+// A TF32 tensor-core product keeps 11 significant bits of each operand.  Every fp32 operand is
+// therefore split in the loaders into hi = the value rounded to 11 bits and lo = the exact
+// remainder, and one product a b becomes three tensor-core products a_hi b_hi + a_hi b_lo + a_lo b_hi
+// (what is dropped is below 2^-22 |a b|).  The tensor core accumulates in fp32 in tensor memory
+// without rounding to nearest, so a long sum would drift; an accumulator only ever takes 128
+// values of k (48 instructions) and is then added, rounded to nearest, to a running fp32 sum in
+// the registers of the epilogue warps.  Two accumulators alternate so that this overlaps the next
+// chunk's products.
+//
+// CTA = one 128 x 128 tile of C.  Warp roles: 0-3 loaders (global -> registers -> split -> shared
+// memory in the K-major, 128-byte-swizzled layout the tensor core reads, whatever the operand's
+// layout in global memory is: an operand whose contiguous index is not k is transposed on the way),
+// 4-7 epilogue (tcgen05.ld, running sum, bias / ReLU / mask, store), 8 MMA issue and TMEM
+// allocation.  Every wait is bounded: one that runs out raises the CTA's abort flag, every role
+// falls through its loop, tensor memory is freed and the device flag word is set.
+#include "abs_gemm.cuh"
+#include "abs_pipeline.cuh"
+
+namespace absk {
+namespace {
+
+constexpr int kTM = 128, kTN = 128;             // tile of C
+constexpr int kTK = 32;                         // k-block: 32 floats = one 128-byte swizzled row
+constexpr int kStagesT = 3;
+constexpr int kChunkKB = 4;                     // k-blocks per tensor-memory accumulator (128 values of k)
+constexpr int kOperandBytes = kTM * 128;        // one 128 x 32 fp32 operand tile
+constexpr int kStageBytesT = 4 * kOperandBytes; // A_hi, A_lo, B_hi, B_lo
+constexpr int kLoaders = 128;
+constexpr int kThreadsT = 288;
+constexpr int kTmemCols = 256;                  // two accumulators of 128 columns
+constexpr size_t kSmemT = static_cast<size_t>(kStagesT) * kStageBytesT + 1024 + 256;
+
+struct TcParams {
+  GemmArgs g;
+  unsigned* flag;
+  long long timeout_cycles;
+};
+
+__device__ __forceinline__ void fence_async_smem_t() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ bool elect_one_t() {
+  uint32_t is_leader;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(is_leader));
+  return is_leader != 0;
+}
+// D (fp32, TMEM) (+)= A (tf32, smem, K-major) * B^T (tf32, smem, K-major); issued by one thread.
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_t(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32_t(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%32];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr), "r"(taddr + 16u)
+      : "memory");
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+// Bounded wait that sleeps between polls, for the warps that wait long (they leave the issue slots
+// to the loaders and the MMA thread).
+__device__ __forceinline__ bool mbar_wait_sleep(uint32_t bar, uint32_t parity, volatile unsigned* abort_flag,
+                                                long long limit) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (*abort_flag) return false;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag || clock64() - t0 > limit) {
+      *abort_flag = 1u;
+      return false;
+    }
+    __nanosleep(64);
+  }
+  return true;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, float4 v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t addr, float v) {
+  asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+// hi: the value rounded to 11 significant bits (its low 13 mantissa bits are zero, so the tensor
+// core's own conversion changes nothing); lo: the exact remainder, of which the tensor core keeps
+// the leading 11 bits.
+__device__ __forceinline__ void split_tf32(float a, float& hi, float& lo) {
+  hi = __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xffffe000u);
+  lo = a - hi;
+}
+__device__ __forceinline__ void split4(const float4 a, float4& hi, float4& lo) {
+  split_tf32(a.x, hi.x, lo.x);
+  split_tf32(a.y, hi.y, lo.y);
+  split_tf32(a.z, hi.z, lo.z);
+  split_tf32(a.w, hi.w, lo.w);
+}
+
+// Four consecutive elements starting at p; elements at or past `left` read as zero.
+__device__ __forceinline__ float4 load4_guard(const float* p, long long left, bool vec) {
+  if (left >= 4 && vec) return __ldg(reinterpret_cast<const float4*>(p));
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (left > 0) v.x = __ldg(p);
+  if (left > 1) v.y = __ldg(p + 1);
+  if (left > 2) v.z = __ldg(p + 2);
+  if (left > 3) v.w = __ldg(p + 3);
+  return v;
+}
+
+// One operand tile [128 rows of the tile] x [32 values of k] of a k-block, into registers.
+//   KC (k contiguous):  element (row, k) at P[row * rs + k];   piece e -> row e / 8, k quad e % 8
+//   else (row contiguous): element (row, k) at P[k * ks + row]; piece e -> k = e % 32, row quad e / 32
+template <bool KC>
+__device__ __forceinline__ void fetch_operand(const float* P, long long rs_or_ks, long long row_base, long long n_rows,
+                                              int k0, int K, bool vec, int t, float4 (&r)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int e = t + kLoaders * i;
+    if (KC) {
+      const long long row = row_base + (e >> 3);
+      const int k = k0 + 4 * (e & 7);
+      r[i] = load4_guard(P + row * rs_or_ks + k, row < n_rows ? K - k : 0, vec);
+    } else {
+      const int k = k0 + (e & 31);
+      const long long row = row_base + 4 * (e >> 5);
+      r[i] = load4_guard(P + k * rs_or_ks + row, k < K ? n_rows - row : 0, vec);
+    }
+  }
+}
+// ... and from registers into the hi and lo tiles (K-major rows of 128 bytes; the 16-byte chunk c
+// of row r sits at chunk position c ^ (r % 8)).
+template <bool KC>
+__device__ __forceinline__ void stash_operand(uint32_t hi_tile, uint32_t lo_tile, int t, const float4 (&r)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int e = t + kLoaders * i;
+    float4 hi, lo;
+    split4(r[i], hi, lo);
+    if (KC) {
+      const uint32_t row = static_cast<uint32_t>(e >> 3), ch = static_cast<uint32_t>(e & 7);
+      const uint32_t off = row * 128u + ((ch ^ (row & 7u)) << 4);
+      sts128(hi_tile + off, hi);
+      sts128(lo_tile + off, lo);
+    } else {
+      const uint32_t k = static_cast<uint32_t>(e & 31), row0 = 4u * static_cast<uint32_t>(e >> 5);
+      const float h[4] = {hi.x, hi.y, hi.z, hi.w}, l[4] = {lo.x, lo.y, lo.z, lo.w};
+#pragma unroll
+      for (uint32_t j = 0; j < 4; ++j) {
+        const uint32_t row = row0 + j;
+        const uint32_t off = row * 128u + (((k >> 2) ^ (row & 7u)) << 4) + (k & 3u) * 4u;
+        sts32(hi_tile + off, h[j]);
+        sts32(lo_tile + off, l[j]);
+      }
+    }
+  }
+}
+
+template <bool A_KC, bool B_KC>
+__global__ void __launch_bounds__(kThreadsT, 1)
+gemm_tc_kernel(const TcParams prm) {
+  extern __shared__ unsigned char smem_dyn[];
+  const GemmArgs& g = prm.g;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int z = blockIdx.z;
+  const long long r0 = static_cast<long long>(blockIdx.y) * kTM, c0 = static_cast<long long>(blockIdx.x) * kTN;
+
+  const uint32_t raw_u32 = smem_u32(smem_dyn);
+  const uint32_t ring_u32 = (raw_u32 + 1023u) & ~1023u;            // the swizzle is a function of the address
+  unsigned char* tail = smem_dyn + (ring_u32 - raw_u32) + static_cast<size_t>(kStagesT) * kStageBytesT;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);   // full[3] empty[3] accfull[2] accempty[2] done
+  volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + 12);
+  unsigned* tmem_slot = const_cast<unsigned*>(abort_flag) + 1;
+  const uint32_t full_u32 = smem_u32(bars);
+  const uint32_t empty_u32 = full_u32 + 8u * kStagesT;
+  const uint32_t accfull_u32 = empty_u32 + 8u * kStagesT;
+  const uint32_t accempty_u32 = accfull_u32 + 16u;
+  const uint32_t done_u32 = accempty_u32 + 16u;
+
+  if (tid == 0) {
+    for (int s = 0; s < kStagesT; ++s) {
+      mbar_init(full_u32 + 8u * s, kLoaders);
+      mbar_init(empty_u32 + 8u * s, 1);
+    }
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(accfull_u32 + 8u * k, 1);
+      mbar_init(accempty_u32 + 8u * k, 128);
+    }
+    mbar_init(done_u32, 1);
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(static_cast<uint32_t>(kTmemCols))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_before();
+  __syncthreads();
+  tc_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_kb = (g.K + kTK - 1) / kTK;
+  const int n_chunks = (n_kb + kChunkKB - 1) / kChunkKB;
+
+  if (warp < 4) {
+    // ---- loaders ----------------------------------------------------------------------------
+    const float* A = g.A + z * g.a_bs;
+    const float* B = g.B + z * g.b_bs;
+    const long long a_str = A_KC ? g.a_rs : g.a_cs, b_str = B_KC ? g.b_cs : g.b_rs;
+    const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (a_str & 3) == 0 &&
+                       (A_KC || (r0 & 3) == 0);
+    const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (b_str & 3) == 0 &&
+                       (B_KC || (c0 & 3) == 0);
+    int s = 0;
+    uint32_t pass = 0;
+    for (int kb = 0; kb < n_kb; ++kb) {
+      const int k0 = kb * kTK;
+      float4 ra[8], rb[8];
+      fetch_operand<A_KC>(A, a_str, r0, g.rows, k0, g.K, a_vec, tid, ra);   // the loads are in flight while
+      fetch_operand<B_KC>(B, b_str, c0, g.cols, k0, g.K, b_vec, tid, rb);   // the stage is waited for
+      if (pass > 0) mbar_wait(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles);
+      const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * kStageBytesT;
+      stash_operand<A_KC>(stage, stage + kOperandBytes, tid, ra);
+      stash_operand<B_KC>(stage + 2 * kOperandBytes, stage + 3 * kOperandBytes, tid, rb);
+      fence_async_smem_t();                        // these stores, before the tensor core reads them
+      mbar_arrive(full_u32 + 8u * s);
+      if (++s == kStagesT) {
+        s = 0;
+        ++pass;
+      }
+    }
+  } else if (warp == 8) {
+    // ---- MMA issue ----------------------------------------------------------------------------
+    // instruction descriptor: fp32 accumulate (bit 4), tf32 x tf32 (2 at bits 7 and 10), both K-major,
+    // N / 8 at bit 17, M / 16 at bit 24
+    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(kTN >> 3) << 17) |
+                           (static_cast<uint32_t>(kTM >> 4) << 24);
+    // operand descriptor, K-major with 128-byte swizzle: start address / 16, 8-row groups 1024 bytes
+    // apart (64 << 32), descriptor version 1 (bit 46), swizzle mode 2 (bits 61-63)
+    const uint64_t desc_hi = (64ull << 32) | (1ull << 46) | (2ull << 61) | (1ull << 16);
+    int s = 0;
+    uint32_t pass = 0;
+    for (int kb = 0; kb < n_kb; ++kb) {
+      const int chunk = kb / kChunkKB, pos = kb - chunk * kChunkKB;
+      const uint32_t buf = static_cast<uint32_t>(chunk) & 1u, use = static_cast<uint32_t>(chunk) >> 1;
+      if (pos == 0 && use > 0) mbar_wait(accempty_u32 + 8u * buf, (use - 1) & 1u, abort_flag, prm.timeout_cycles);
+      mbar_wait(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles);
+      fence_async_smem_t();
+      tc_after();
+      const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(kTN);
+      const uint32_t base = ((ring_u32 + static_cast<uint32_t>(s) * kStageBytesT) & 0x3ffffu) >> 4;
+      const uint32_t op16 = kOperandBytes >> 4;
+      const bool last_of_chunk = pos == kChunkKB - 1 || kb == n_kb - 1;
+      if (elect_one_t()) {
+#pragma unroll
+        for (int k = 0; k < kTK / 8; ++k) {                          // an instruction takes 8 values of k (32 bytes)
+          const uint64_t a_hi = desc_hi | static_cast<uint64_t>(base + 2u * k);
+          const uint64_t a_lo = desc_hi | static_cast<uint64_t>(base + op16 + 2u * k);
+          const uint64_t b_hi = desc_hi | static_cast<uint64_t>(base + 2u * op16 + 2u * k);
+          const uint64_t b_lo = desc_hi | static_cast<uint64_t>(base + 3u * op16 + 2u * k);
+          umma_tf32(d_tmem, a_lo, b_hi, idesc, (pos == 0 && k == 0) ? 0u : 1u);   // the small terms first
+          umma_tf32(d_tmem, a_hi, b_lo, idesc, 1u);
+          umma_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
+        }
+        umma_commit_t(empty_u32 + 8u * s);                           // the stage may be refilled
+        if (last_of_chunk) umma_commit_t(accfull_u32 + 8u * buf);
+      }
+      __syncwarp();
+      if (++s == kStagesT) {
+        s = 0;
+        ++pass;
+      }
+    }
+    if (elect_one_t()) umma_commit_t(done_u32);
+    __syncwarp();
+    volatile unsigned ignore = 0u;
+    mbar_wait(done_u32, 0u, &ignore, prm.timeout_cycles);            // no MMA in flight when TMEM is freed
+  } else {
+    // ---- epilogue: this thread owns row 32 (warp % 4) + lane of the tile -------------------------
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    float acc[kTN];
+#pragma unroll
+    for (int j = 0; j < kTN; ++j) acc[j] = 0.f;
+    for (int chunk = 0; chunk < n_chunks; ++chunk) {
+      const uint32_t buf = static_cast<uint32_t>(chunk) & 1u, use = static_cast<uint32_t>(chunk) >> 1;
+      mbar_wait_sleep(accfull_u32 + 8u * buf, use & 1u, abort_flag, prm.timeout_cycles);
+      tc_after();
+      const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(kTN) + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll
+      for (int c32 = 0; c32 < kTN; c32 += 32) {
+        float v[32];
+        tmem_ld32_t(taddr + static_cast<uint32_t>(c32), v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[c32 + j] += v[j];           // rounded to nearest
+      }
+      tc_before();
+      mbar_arrive(accempty_u32 + 8u * buf);
+    }
+    const long long r = r0 + row;
+    if (r < g.rows) {
+      float* Crow = g.C + z * g.c_bs + r * g.c_rs + c0;
+      const float* bias = (g.mode == 1 || g.mode == 2) ? g.bias + z * g.bias_bs + c0 : nullptr;
+      const float* mrow = g.mode == 3 ? g.mask + z * g.mask_bs + r * g.mask_rs + c0 : nullptr;
+      const bool vec = (reinterpret_cast<uintptr_t>(Crow) & 15u) == 0;
+#pragma unroll
+      for (int j = 0; j < kTN; j += 4) {
+        float o[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const long long c = c0 + j + u;
+          float v = acc[j + u];
+          if (c < g.cols) {
+            if (g.mode == 0) v *= g.alpha;
+            else if (g.mode == 1) v = fmaxf(v + bias[j + u], 0.f);
+            else if (g.mode == 2) v = v + bias[j + u];
+            else v = mrow[j + u] > 0.f ? v : 0.f;
+          }
+          o[u] = v;
+        }
+        if (vec && c0 + j + 3 < g.cols) {
+          *reinterpret_cast<float4*>(Crow + j) = make_float4(o[0], o[1], o[2], o[3]);
+        } else {
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (c0 + j + u < g.cols) Crow[j + u] = o[u];
+        }
+      }
+    }
+  }
+  tc_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(kTmemCols))
+                 : "memory");
+  }
+  if (tid == 0 && *abort_flag) atomicOr(prm.flag, 1u);
+}
+
+template <bool A_KC, bool B_KC>
+bool launch_tc_variant(const TcParams& prm, dim3 grid, cudaStream_t st) {
+  auto kern = gemm_tc_kernel<A_KC, B_KC>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemT)) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  kern<<<grid, kThreadsT, kSmemT, st>>>(prm);
+  return true;
+}
+
+}  // namespace
+
+bool launch_gemm_tc(const GemmArgs& g, int batch, unsigned* flag, long long timeout_cycles, cudaStream_t st) {
+  const bool a_kc = g.a_cs == 1, a_rc = g.a_rs == 1, b_kc = g.b_rs == 1, b_cc = g.b_cs == 1;
+  if (!(a_kc || a_rc) || !(b_kc || b_cc)) return false;
+  if (g.rows < 96 || g.cols < 96 || g.K < 64) return false;     // a 128 x 128 tile must be mostly used
+  const unsigned gx = static_cast<unsigned>((g.cols + kTN - 1) / kTN), gy = static_cast<unsigned>((g.rows + kTM - 1) / kTM);
+  if (gy > 65535u || batch > 65535) return false;
+  TcParams prm{g, flag, timeout_cycles};
+  const dim3 grid(gx, gy, static_cast<unsigned>(batch));
+  if (a_kc && b_kc) return launch_tc_variant<true, true>(prm, grid, st);
+  if (a_kc) return launch_tc_variant<true, false>(prm, grid, st);
+  if (b_kc) return launch_tc_variant<false, true>(prm, grid, st);
+  return launch_tc_variant<false, false>(prm, grid, st);
+}
+
+}  // namespace absk

@@ -30,6 +30,7 @@ struct Tuning {
   long long stats_no_cluster = 0;
   long long stats_no_secondary = 0;        // 1: the cluster kernel does not use the SMs its clusters cannot occupy
   long long stats_secondary_pct = 0;       // speed of an SM of the second launch, per cent of the first's (0: 95)
+  long long mlp_no_tensor_cores = 0;       // 1: the MLP producer's products stay on the CUDA cores
   long long stats_no_recheck = 0;          // 1: keep a Gram kernel's record whatever its conditioning
   long long stats_cluster_rows = 0;
   long long stats_timeout_cycles = 0;      // 0: about two seconds of SM clock

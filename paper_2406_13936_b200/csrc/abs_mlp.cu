@@ -16,7 +16,7 @@
 // and with N = ||gbar||^2:  sum_i ||g_i - gbar||^2 = sum_i ||g_i||^2 - b N  (Eq. def_var expanded),
 // Var_i <g_i, gbar> directly.  The expansions cancel only when the variance is far below b N,
 // i.e. when the test is satisfied by a wide margin anyway.
-#include "abs_internal.cuh"
+#include "abs_gemm.cuh"
 
 namespace absk {
 namespace {
@@ -54,18 +54,7 @@ MlpShape make_shape(const int* dims, long long b) {
   return s;
 }
 
-// ---- batched fp32 GEMM with strided operands and a small epilogue ---------------------------
-struct GemmArgs {
-  const float* A; long long a_rs, a_cs, a_bs;    // element (r, k) at A[z*a_bs + r*a_rs + k*a_cs]
-  const float* B; long long b_rs, b_cs, b_bs;    // element (k, c)
-  float* C; long long c_rs, c_bs;                // element (r, c) at C[z*c_bs + r*c_rs + c]
-  const float* bias; long long bias_bs;          // per column (modes 1, 2)
-  const float* mask; long long mask_rs, mask_bs; // shape of C (mode 3)
-  int rows, cols, K;
-  float alpha;
-  int mode;   // 0: alpha*acc   1: relu(acc + bias)   2: acc + bias   3: acc where mask > 0, else 0
-};
-
+// ---- batched fp32 GEMM with strided operands and a small epilogue (GemmArgs: abs_gemm.cuh) ----
 constexpr int kTile = 64, kTileK = 16;
 
 __global__ void __launch_bounds__(256)
@@ -284,7 +273,13 @@ sgemm_big_kernel(const GemmArgs g) {
   }
 }
 
-void launch_gemm(const GemmArgs& g, int batch, cudaStream_t st) {
+void launch_gemm(abs_ctx* ctx, const GemmArgs& g, int batch, cudaStream_t st) {
+  // large products go to the tensor cores (3 x TF32 split, abs_gemm_tc.cu); a wait that runs out there
+  // raises the context's time-out word, which the statistics that follow report
+  if (!ctx->tuning.mlp_no_tensor_cores &&
+      launch_gemm_tc(g, batch, ctx->flags,
+                     ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles, st))
+    return;
   // the large-tile kernel where a 128 x 128 tile is mostly used and both operands have a contiguous index
   const bool a_ok = g.a_cs == 1 || g.a_rs == 1, b_ok = g.b_rs == 1 || g.b_cs == 1;
   if (a_ok && b_ok && g.rows >= 96 && g.cols >= 96) {
@@ -497,9 +492,11 @@ fused_norm_kernel(const float* __restrict__ Gb, long long d, float* __restrict__
 // One block per worker: abs_stats from c_i, q_i and N.
 __global__ void __launch_bounds__(1024)
 fused_finalize_kernel(const float* __restrict__ scratch, long long per_worker, long long sCQ, long long b,
-                      abs_stats* __restrict__ stats) {
+                      abs_stats* __restrict__ stats, unsigned* __restrict__ flags) {
   __shared__ double red[3][32];
   const int m = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  unsigned timeout_word = 0u;      // raised by a tensor-core product whose wait ran out
+  if (tid == 0) timeout_word = *reinterpret_cast<volatile unsigned*>(flags);
   const double* cq = reinterpret_cast<const double*>(scratch + m * per_worker + sCQ);
   const double bd = static_cast<double>(b);
   auto block_sum = [&](double v, int slot) {
@@ -545,7 +542,14 @@ fused_finalize_kernel(const float* __restrict__ scratch, long long per_worker, l
     o.status = 0u;
     if (!(isfinite(qsum) && isfinite(N) && isfinite(ss))) o.status |= ABS_STATUS_NONFINITE;
     if (N == 0.0) o.status |= ABS_STATUS_ZERO_MEAN;
+    if (timeout_word != 0u) o.status |= ABS_STATUS_TIMEOUT;
     o.recomputed = 0u;
+    // the last worker to get here clears the time-out word and the arrival counter for the next call
+    __threadfence();
+    if (atomicAdd(flags + 1, 1u) == gridDim.x - 1) {
+      flags[0] = 0u;
+      flags[1] = 0u;
+    }
     stats[m] = o;
   }
 }
@@ -602,32 +606,32 @@ extern "C" int abs_mlp_grads(abs_ctx* ctx, const float* inputs, const int* label
   // forward: H1 = relu(Xin W1^T + b1), H2 = relu(H1 W2^T + b2), logits = H2 W3^T + b3
   g = GemmArgs{ws + s.sX, s.n0, 1, pw, X + s.oW1, 1, s.n0, d, ws + s.sH1, s.n1, pw, X + s.ob1, d, nullptr, 0, 0,
                static_cast<int>(b), s.n1, s.n0, 1.f, 1};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   g = GemmArgs{ws + s.sH1, s.n1, 1, pw, X + s.oW2, 1, s.n1, d, ws + s.sH2, s.n2, pw, X + s.ob2, d, nullptr, 0, 0,
                static_cast<int>(b), s.n2, s.n1, 1.f, 1};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   g = GemmArgs{ws + s.sH2, s.n2, 1, pw, X + s.oW3, 1, s.n2, d, ws + s.sD3, s.n3, pw, X + s.ob3, d, nullptr, 0, 0,
                static_cast<int>(b), s.n3, s.n2, 1.f, 2};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   softmax_delta_kernel<<<dim3(static_cast<unsigned>((b + 127) / 128), M), 128, 0, st>>>(ws, pw, s.sD3, b, s.n3, labels,
                                                                                        n, idx, idx_stride);
   // backward: D2 = (D3 W3) .* (H2 > 0), D1 = (D2 W2) .* (H1 > 0)
   g = GemmArgs{ws + s.sD3, s.n3, 1, pw, X + s.oW3, s.n2, 1, d, ws + s.sD2, s.n2, pw, nullptr, 0, ws + s.sH2, s.n2, pw,
                static_cast<int>(b), s.n2, s.n3, 1.f, 3};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   g = GemmArgs{ws + s.sD2, s.n2, 1, pw, X + s.oW2, s.n1, 1, d, ws + s.sD1, s.n1, pw, nullptr, 0, ws + s.sH1, s.n1, pw,
                static_cast<int>(b), s.n1, s.n2, 1.f, 3};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   // batch gradients: dW_l = (1/b) D_l^T H_{l-1}, db_l = (1/b) sum_i D_l[i]
   g = GemmArgs{ws + s.sD3, 1, s.n3, pw, ws + s.sH2, s.n2, 1, pw, Gb + s.oW3, s.n2, d, nullptr, 0, nullptr, 0, 0,
                s.n3, s.n2, static_cast<int>(b), inv_b, 0};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   g = GemmArgs{ws + s.sD2, 1, s.n2, pw, ws + s.sH1, s.n1, 1, pw, Gb + s.oW2, s.n1, d, nullptr, 0, nullptr, 0, 0,
                s.n2, s.n1, static_cast<int>(b), inv_b, 0};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   g = GemmArgs{ws + s.sD1, 1, s.n1, pw, ws + s.sX, s.n0, 1, pw, Gb + s.oW1, s.n0, d, nullptr, 0, nullptr, 0, 0,
                s.n1, s.n0, static_cast<int>(b), inv_b, 0};
-  launch_gemm(g, M, st);
+  launch_gemm(ctx, g, M, st);
   bias_grad_kernel<<<dim3((s.n3 + 31) / 32, M), 1024, 0, st>>>(ws, pw, s.sD3, b, s.n3, Gb, d, s.ob3);
   bias_grad_kernel<<<dim3((s.n2 + 31) / 32, M), 1024, 0, st>>>(ws, pw, s.sD2, b, s.n2, Gb, d, s.ob2);
   bias_grad_kernel<<<dim3((s.n1 + 31) / 32, M), 1024, 0, st>>>(ws, pw, s.sD1, b, s.n1, Gb, d, s.ob1);
@@ -703,13 +707,13 @@ extern "C" int abs_mlp_fused_stats(abs_ctx* ctx, const int* dims, long long b, i
     // U[i][o] = sum_k h[i][k] dW[o][k]
     GemmArgs g{ws + sH, n_in, 1, pw, Gb + oW, 1, n_in, d, ws + s.sU, n_out, pw, nullptr, 0, nullptr, 0, 0,
                static_cast<int>(b), n_out, n_in, 1.f, 0};
-    launch_gemm(g, M, st);
+    launch_gemm(ctx, g, M, st);
     fused_rowdot_kernel<<<dim3(warp_blocks, M), 256, 0, st>>>(ws, pw, sD, s.sU, s.sCQ, b, n_out, Gb, d, ob);
   };
   layer(s.sD1, s.sX, s.n1, s.n0, s.oW1, s.ob1);
   layer(s.sD2, s.sH1, s.n2, s.n1, s.oW2, s.ob2);
   layer(s.sD3, s.sH2, s.n3, s.n2, s.oW3, s.ob3);
-  fused_finalize_kernel<<<M, 1024, 0, st>>>(ws, pw, s.sCQ, b, stats);
+  fused_finalize_kernel<<<M, 1024, 0, st>>>(ws, pw, s.sCQ, b, stats, ctx->flags);
   const cudaError_t e = cudaGetLastError();
   if (prev != ctx->device) cudaSetDevice(prev);
   if (e != cudaSuccess) return set_error(ctx, ABS_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));

@@ -294,7 +294,11 @@ def mlp_problem(seed, n, dims, M, device="cuda"):
 
 
 @pytest.mark.parametrize("dims,M,b", [((6, 5, 4, 3), 2, 4), ((20, 33, 17, 7), 3, 9), ((70, 130, 65, 10), 2, 67),
-                                      ((784, 1024, 1024, 10), 1, 3)])
+                                      ((784, 1024, 1024, 10), 1, 3),
+                                      # large enough for the tensor-core products (rows, columns >= 96, K >= 64),
+                                      # with ragged tiles, an odd parameter count (replica 1 is not 16-byte
+                                      # aligned) and every operand layout
+                                      ((200, 257, 191, 10), 3, 130), ((784, 1024, 1024, 10), 2, 150)])
 def test_mlp_batch_and_per_sample_gradients(ctx, dims, M, b):
     n = 300
     inp, lab, X = mlp_problem(5, n, dims, M)
@@ -317,6 +321,43 @@ def test_mlp_batch_and_per_sample_gradients(ctx, dims, M, b):
         ref_b = orc.batch_mean(ref)
         assert np.abs(f64(Gb[m]) - ref_b).max() <= 1e-5 * np.abs(ref_b).max()
         assert torch.all(G[:, d:] == 0)          # the padding columns are left alone
+
+
+@pytest.mark.parametrize("dims,M,b", [((200, 257, 191, 10), 3, 130), ((784, 1024, 1024, 10), 2, 300),
+                                      ((300, 400, 500, 12), 2, 1000)])
+def test_mlp_tensor_core_products_match_the_cuda_core_products(ctx, dims, M, b):
+    """The same forward/backward pass twice: matrix products on the tensor cores (fp32 operands split
+    into two TF32 parts, three products each, 128-value chunks added in fp32) and on the CUDA cores
+    (fp32 products folded into fp64).  Batch gradients, activations and deltas agree to a few fp32
+    ulps of the largest entry."""
+    n = 4000
+    inp, lab, X = mlp_problem(7, n, dims, M)
+    X += 0.03 * torch.randn(X.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(3))
+    d = ctx.mlp_param_count(dims)
+    idx = inputs.batch_indices(8, (M, b), n, device="cuda")
+    out = []
+    for no_tc in (0, 1):
+        scratch = ctx.mlp_scratch(M, b, dims)
+        scratch.zero_()
+        Gb = torch.zeros((M, d), device="cuda")
+        ctx.set_tuning("mlp_no_tensor_cores", no_tc)
+        try:
+            ctx.abs_mlp_grads(inp, lab, dims, idx, X, b, Gb, scratch)
+            st = ctx.new_stats(M)
+            ctx.abs_mlp_fused_stats(dims, b, scratch, Gb, st)
+        finally:
+            ctx.set_tuning("mlp_no_tensor_cores", 0)
+        torch.cuda.synchronize()
+        # a worker's scratch starts with Xin, H1, H2, D3, D2, D1 (inputs, activations, deltas)
+        acts = scratch.view(torch.float32).view(M, -1)[:, :b * (dims[0] + 2 * dims[1] + 2 * dims[2] + dims[3])].clone()
+        out.append((Gb, acts, pkg.stats_to_dicts(st)))
+    (g_tc, a_tc, s_tc), (g_cc, a_cc, s_cc) = out
+    assert (g_tc - g_cc).abs().max().item() <= 5e-6 * g_cc.abs().max().item()
+    assert (a_tc - a_cc).abs().max().item() <= 5e-6 * a_cc.abs().max().item()
+    for t, c in zip(s_tc, s_cc):
+        assert t["status"] == c["status"] == 0
+        for key in ("gbar_sq", "var_norm", "var_ip", "sum_sq"):
+            assert t[key] == pytest.approx(c[key], rel=2e-5)
 
 
 @pytest.mark.parametrize("dims,M,b", [((20, 33, 17, 7), 3, 9), ((70, 130, 65, 10), 2, 67),
