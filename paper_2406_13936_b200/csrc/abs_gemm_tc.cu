@@ -5,16 +5,21 @@
 // therefore split in the loaders into hi = the value rounded to 11 bits and lo = the exact
 // remainder, and one product a b becomes three tensor-core products a_hi b_hi + a_hi b_lo + a_lo b_hi
 // (what is dropped is below 2^-22 |a b|).  The tensor core accumulates in fp32 in tensor memory
-// without rounding to nearest, so a long sum would drift; an accumulator only ever takes 128
-// values of k (48 instructions) and is then added, rounded to nearest, to a running fp32 sum in
-// the registers of the epilogue warps.  Two accumulators alternate so that this overlaps the next
-// chunk's products.
+// without rounding to nearest, so a long sum would drift: an accumulator only ever takes 32 values
+// of k, the cross terms (2^-11 of the main term) have an accumulator of their own so that the main
+// one sees four additions, and both are then added, rounded to nearest, to a running fp32 sum in
+// the registers of the epilogue warps.  Two accumulator pairs alternate so that this overlaps the
+// next k-block's products.  Measured against fp64 on the first layer of the MLP (K = 784, values up
+// to 11): rms error 4.4e-7 with all three products in one accumulator of 32 values of k, 1e-5 (max)
+// with 128 values; the CUDA-core kernels (fp32 slices folded into fp64) have 1.3e-7.
 //
-// CTA = one 128 x 128 tile of C.  Warp roles: 0-3 loaders (global -> registers -> split -> shared
-// memory in the K-major, 128-byte-swizzled layout the tensor core reads, whatever the operand's
-// layout in global memory is: an operand whose contiguous index is not k is transposed on the way),
-// 4-7 epilogue (tcgen05.ld, running sum, bias / ReLU / mask, store), 8 MMA issue and TMEM
-// allocation.  Every wait is bounded: one that runs out raises the CTA's abort flag, every role
+// CTA = one 128 x 128 tile of C.  Warp roles: 0-7 loaders in two sets that take alternate k-blocks
+// (global -> registers -> split -> shared memory with the 128-byte swizzle: K-major when k is the
+// operand's contiguous index in global memory, MN-major when the tile's rows are, so every global
+// load and every shared-memory store moves whole 16-byte pieces and nothing is transposed; a
+// set's loads of one k-block are in flight while the other set stores its own), 8-15 epilogue (tcgen05.ld, running sum, bias / ReLU / mask,
+// store; two warps share a quarter of the TMEM lanes and take 64 columns each), 16 MMA issue and
+// TMEM allocation.  Every wait is bounded: one that runs out raises the CTA's abort flag, every role
 // falls through its loop, tensor memory is freed and the device flag word is set.
 #include "abs_gemm.cuh"
 #include "abs_pipeline.cuh"
@@ -25,12 +30,15 @@ namespace {
 constexpr int kTM = 128, kTN = 128;             // tile of C
 constexpr int kTK = 32;                         // k-block: 32 floats = one 128-byte swizzled row
 constexpr int kStagesT = 3;
-constexpr int kChunkKB = 4;                     // k-blocks per tensor-memory accumulator (128 values of k)
+constexpr int kChunkKB = 1;                     // k-blocks per tensor-memory accumulator (32 values of k)
 constexpr int kOperandBytes = kTM * 128;        // one 128 x 32 fp32 operand tile
 constexpr int kStageBytesT = 4 * kOperandBytes; // A_hi, A_lo, B_hi, B_lo
-constexpr int kLoaders = 128;
-constexpr int kThreadsT = 288;
-constexpr int kTmemCols = 256;                  // two accumulators of 128 columns
+constexpr int kLoaders = 128;                   // threads of one loader set
+constexpr int kLoaderSets = 2;
+constexpr int kEpiWarps = 8;
+constexpr int kMmaWarp = kLoaderSets * 4 + kEpiWarps;
+constexpr int kThreadsT = (kMmaWarp + 1) * 32;  // 544
+constexpr int kTmemCols = 512;                  // two sets of two accumulators (main, cross terms) of 128 columns
 constexpr size_t kSmemT = static_cast<size_t>(kStagesT) * kStageBytesT + 1024 + 256;
 
 struct TcParams {
@@ -64,21 +72,18 @@ __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint
 __device__ __forceinline__ void umma_commit_t(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// 32 consecutive accumulator columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32_t(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 16 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16_t(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%32];\n\t"
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
       "tcgen05.wait::ld.sync.aligned;"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr), "r"(taddr + 16u)
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
       : "memory");
 #pragma unroll
-  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+  for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
 }
 // Bounded wait that sleeps between polls, for the warps that wait long (they leave the issue slots
 // to the loaders and the MMA thread).
@@ -130,7 +135,8 @@ __device__ __forceinline__ float4 load4_guard(const float* p, long long left, bo
 
 // One operand tile [128 rows of the tile] x [32 values of k] of a k-block, into registers.
 //   KC (k contiguous):  element (row, k) at P[row * rs + k];   piece e -> row e / 8, k quad e % 8
-//   else (row contiguous): element (row, k) at P[k * ks + row]; piece e -> k = e % 32, row quad e / 32
+//   else (row contiguous): element (row, k) at P[k * ks + row]; piece e -> k = e / 32, row quad e % 32
+// Either way a warp instruction reads whole 128-byte lines.
 template <bool KC>
 __device__ __forceinline__ void fetch_operand(const float* P, long long rs_or_ks, long long row_base, long long n_rows,
                                               int k0, int K, bool vec, int t, float4 (&r)[8]) {
@@ -142,14 +148,20 @@ __device__ __forceinline__ void fetch_operand(const float* P, long long rs_or_ks
       const int k = k0 + 4 * (e & 7);
       r[i] = load4_guard(P + row * rs_or_ks + k, row < n_rows ? K - k : 0, vec);
     } else {
-      const int k = k0 + (e & 31);
-      const long long row = row_base + 4 * (e >> 5);
+      const int k = k0 + (e >> 5);
+      const long long row = row_base + 4 * (e & 31);
       r[i] = load4_guard(P + k * rs_or_ks + row, k < K ? n_rows - row : 0, vec);
     }
   }
 }
-// ... and from registers into the hi and lo tiles (K-major rows of 128 bytes; the 16-byte chunk c
-// of row r sits at chunk position c ^ (r % 8)).
+// ... and from registers into the hi and lo tiles, 16 bytes at a time, in the layout the tensor core
+// reads with the 128-byte swizzle:
+//   KC:   K-major.  Row r of the tile is 128 bytes (its 32 values of k); the 16-byte chunk c of row r
+//         sits at chunk position c ^ (r % 8); 8-row groups are 1024 bytes apart.
+//   else: MN-major, for which TF32 operands have one layout: the 128-byte swizzle with a 32-byte base.
+//         The tile is cut into blocks of [4 values of k] x [32 rows] (512 bytes): inside a block the 32
+//         rows of one k are 128 contiguous bytes, and the 32-byte piece p of k-line kr sits at piece
+//         position p ^ kr; the four row blocks of one k-quad are 512 bytes apart, the k-quads 2048.
 template <bool KC>
 __device__ __forceinline__ void stash_operand(uint32_t hi_tile, uint32_t lo_tile, int t, const float4 (&r)[8]) {
 #pragma unroll
@@ -157,22 +169,17 @@ __device__ __forceinline__ void stash_operand(uint32_t hi_tile, uint32_t lo_tile
     const int e = t + kLoaders * i;
     float4 hi, lo;
     split4(r[i], hi, lo);
+    uint32_t off;
     if (KC) {
       const uint32_t row = static_cast<uint32_t>(e >> 3), ch = static_cast<uint32_t>(e & 7);
-      const uint32_t off = row * 128u + ((ch ^ (row & 7u)) << 4);
-      sts128(hi_tile + off, hi);
-      sts128(lo_tile + off, lo);
+      off = row * 128u + ((ch ^ (row & 7u)) << 4);
     } else {
-      const uint32_t k = static_cast<uint32_t>(e & 31), row0 = 4u * static_cast<uint32_t>(e >> 5);
-      const float h[4] = {hi.x, hi.y, hi.z, hi.w}, l[4] = {lo.x, lo.y, lo.z, lo.w};
-#pragma unroll
-      for (uint32_t j = 0; j < 4; ++j) {
-        const uint32_t row = row0 + j;
-        const uint32_t off = row * 128u + (((k >> 2) ^ (row & 7u)) << 4) + (k & 3u) * 4u;
-        sts32(hi_tile + off, h[j]);
-        sts32(lo_tile + off, l[j]);
-      }
+      const uint32_t k = static_cast<uint32_t>(e >> 5), rq = static_cast<uint32_t>(e & 31);
+      const uint32_t kr = k & 3u, c16 = rq & 7u;
+      off = (k >> 2) * 2048u + (rq >> 3) * 512u + kr * 128u + (((c16 >> 1) ^ kr) << 5) + ((c16 & 1u) << 4);
     }
+    sts128(hi_tile + off, hi);
+    sts128(lo_tile + off, lo);
   }
 }
 
@@ -204,13 +211,13 @@ gemm_tc_kernel(const TcParams prm) {
     }
     for (int k = 0; k < 2; ++k) {
       mbar_init(accfull_u32 + 8u * k, 1);
-      mbar_init(accempty_u32 + 8u * k, 128);
+      mbar_init(accempty_u32 + 8u * k, kEpiWarps * 32);
     }
     mbar_init(done_u32, 1);
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 8) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"(static_cast<uint32_t>(kTmemCols))
                  : "memory");
@@ -224,42 +231,44 @@ gemm_tc_kernel(const TcParams prm) {
   const int n_kb = (g.K + kTK - 1) / kTK;
   const int n_chunks = (n_kb + kChunkKB - 1) / kChunkKB;
 
-  if (warp < 4) {
-    // ---- loaders ----------------------------------------------------------------------------
+  if (warp < kLoaderSets * 4) {
+    // ---- loaders: set `set` takes the k-blocks kb = set, set + 2, ... ---------------------------
+    const int set = warp >> 2, t = tid & (kLoaders - 1);
     const float* A = g.A + z * g.a_bs;
     const float* B = g.B + z * g.b_bs;
     const long long a_str = A_KC ? g.a_rs : g.a_cs, b_str = B_KC ? g.b_cs : g.b_rs;
-    const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (a_str & 3) == 0 &&
-                       (A_KC || (r0 & 3) == 0);
-    const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (b_str & 3) == 0 &&
-                       (B_KC || (c0 & 3) == 0);
-    int s = 0;
-    uint32_t pass = 0;
-    for (int kb = 0; kb < n_kb; ++kb) {
+    const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (a_str & 3) == 0;
+    const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (b_str & 3) == 0;
+    for (int kb = set; kb < n_kb; kb += kLoaderSets) {
       const int k0 = kb * kTK;
+      const int s = kb % kStagesT;
+      const uint32_t pass = static_cast<uint32_t>(kb / kStagesT);
       float4 ra[8], rb[8];
-      fetch_operand<A_KC>(A, a_str, r0, g.rows, k0, g.K, a_vec, tid, ra);   // the loads are in flight while
-      fetch_operand<B_KC>(B, b_str, c0, g.cols, k0, g.K, b_vec, tid, rb);   // the stage is waited for
+      fetch_operand<A_KC>(A, a_str, r0, g.rows, k0, g.K, a_vec, t, ra);     // the loads are in flight while
+      fetch_operand<B_KC>(B, b_str, c0, g.cols, k0, g.K, b_vec, t, rb);     // the stage is waited for
       if (pass > 0) mbar_wait(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles);
       const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * kStageBytesT;
-      stash_operand<A_KC>(stage, stage + kOperandBytes, tid, ra);
-      stash_operand<B_KC>(stage + 2 * kOperandBytes, stage + 3 * kOperandBytes, tid, rb);
+      stash_operand<A_KC>(stage, stage + kOperandBytes, t, ra);
+      stash_operand<B_KC>(stage + 2 * kOperandBytes, stage + 3 * kOperandBytes, t, rb);
       fence_async_smem_t();                        // these stores, before the tensor core reads them
       mbar_arrive(full_u32 + 8u * s);
-      if (++s == kStagesT) {
-        s = 0;
-        ++pass;
-      }
     }
-  } else if (warp == 8) {
+  } else if (warp == kMmaWarp) {
     // ---- MMA issue ----------------------------------------------------------------------------
-    // instruction descriptor: fp32 accumulate (bit 4), tf32 x tf32 (2 at bits 7 and 10), both K-major,
-    // N / 8 at bit 17, M / 16 at bit 24
-    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(kTN >> 3) << 17) |
-                           (static_cast<uint32_t>(kTM >> 4) << 24);
-    // operand descriptor, K-major with 128-byte swizzle: start address / 16, 8-row groups 1024 bytes
-    // apart (64 << 32), descriptor version 1 (bit 46), swizzle mode 2 (bits 61-63)
-    const uint64_t desc_hi = (64ull << 32) | (1ull << 46) | (2ull << 61) | (1ull << 16);
+    // instruction descriptor: fp32 accumulate (bit 4), tf32 x tf32 (2 at bits 7 and 10), operand
+    // majors (bit 15 / 16: 1 = the rows of the tile, not k, are contiguous in shared memory), N / 8 at
+    // bit 17, M / 16 at bit 24
+    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (A_KC ? 0u : (1u << 15)) | (B_KC ? 0u : (1u << 16)) |
+                           (static_cast<uint32_t>(kTN >> 3) << 17) | (static_cast<uint32_t>(kTM >> 4) << 24);
+    // operand descriptors (version 1 at bit 46, swizzle mode at bits 61-63), offsets in units of 16 bytes.
+    // K-major, 128-byte swizzle (mode 2): 8-row groups 1024 bytes apart (stride offset 64); a k-step of
+    // 8 values is 32 bytes further along the row.  MN-major, 128-byte swizzle with 32-byte base (mode 1):
+    // row blocks 512 bytes apart (leading offset 32), k-quads 2048 bytes apart (stride offset 128); a
+    // k-step of 8 values is two k-quads, 4096 bytes.
+    const uint64_t desc_k = (64ull << 32) | (1ull << 46) | (2ull << 61) | (1ull << 16);
+    const uint64_t desc_mn = (128ull << 32) | (1ull << 46) | (1ull << 61) | (32ull << 16);
+    const uint64_t desc_a = A_KC ? desc_k : desc_mn, desc_b = B_KC ? desc_k : desc_mn;
+    const uint32_t step_a = A_KC ? 2u : 256u, step_b = B_KC ? 2u : 256u;
     int s = 0;
     uint32_t pass = 0;
     for (int kb = 0; kb < n_kb; ++kb) {
@@ -269,20 +278,23 @@ gemm_tc_kernel(const TcParams prm) {
       mbar_wait(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles);
       fence_async_smem_t();
       tc_after();
-      const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(kTN);
+      const uint32_t d_main = tmem_base + buf * static_cast<uint32_t>(2 * kTN), d_cross = d_main + kTN;
       const uint32_t base = ((ring_u32 + static_cast<uint32_t>(s) * kStageBytesT) & 0x3ffffu) >> 4;
       const uint32_t op16 = kOperandBytes >> 4;
       const bool last_of_chunk = pos == kChunkKB - 1 || kb == n_kb - 1;
       if (elect_one_t()) {
 #pragma unroll
         for (int k = 0; k < kTK / 8; ++k) {                          // an instruction takes 8 values of k (32 bytes)
-          const uint64_t a_hi = desc_hi | static_cast<uint64_t>(base + 2u * k);
-          const uint64_t a_lo = desc_hi | static_cast<uint64_t>(base + op16 + 2u * k);
-          const uint64_t b_hi = desc_hi | static_cast<uint64_t>(base + 2u * op16 + 2u * k);
-          const uint64_t b_lo = desc_hi | static_cast<uint64_t>(base + 3u * op16 + 2u * k);
-          umma_tf32(d_tmem, a_lo, b_hi, idesc, (pos == 0 && k == 0) ? 0u : 1u);   // the small terms first
-          umma_tf32(d_tmem, a_hi, b_lo, idesc, 1u);
-          umma_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
+          const uint64_t a_hi = desc_a | static_cast<uint64_t>(base + step_a * k);
+          const uint64_t a_lo = desc_a | static_cast<uint64_t>(base + op16 + step_a * k);
+          const uint64_t b_hi = desc_b | static_cast<uint64_t>(base + 2u * op16 + step_b * k);
+          const uint64_t b_lo = desc_b | static_cast<uint64_t>(base + 3u * op16 + step_b * k);
+          // The cross terms are 2^-11 of the main term: in an accumulator of their own their additions
+          // cost nothing in accuracy, and the main accumulator takes one addition per 8 values of k.
+          const uint32_t first = (pos == 0 && k == 0) ? 0u : 1u;
+          umma_tf32(d_main, a_hi, b_hi, idesc, first);
+          umma_tf32(d_cross, a_lo, b_hi, idesc, first);
+          umma_tf32(d_cross, a_hi, b_lo, idesc, 1u);
         }
         umma_commit_t(empty_u32 + 8u * s);                           // the stage may be refilled
         if (last_of_chunk) umma_commit_t(accfull_u32 + 8u * buf);
@@ -298,39 +310,44 @@ gemm_tc_kernel(const TcParams prm) {
     volatile unsigned ignore = 0u;
     mbar_wait(done_u32, 0u, &ignore, prm.timeout_cycles);            // no MMA in flight when TMEM is freed
   } else {
-    // ---- epilogue: this thread owns row 32 (warp % 4) + lane of the tile -------------------------
-    const int q = warp & 3;
+    // ---- epilogue: this thread owns row 32 (warp % 4) + lane of the tile and 64 of its columns ----
+    constexpr int kCols = kTN / 2;
+    const int q = warp & 3, half = (warp - kLoaderSets * 4) >> 2;
     const int row = q * 32 + lane;
-    float acc[kTN];
+    const int cb = half * kCols;                                     // first column of this thread's share
+    float acc[kCols];
 #pragma unroll
-    for (int j = 0; j < kTN; ++j) acc[j] = 0.f;
+    for (int j = 0; j < kCols; ++j) acc[j] = 0.f;
     for (int chunk = 0; chunk < n_chunks; ++chunk) {
       const uint32_t buf = static_cast<uint32_t>(chunk) & 1u, use = static_cast<uint32_t>(chunk) >> 1;
       mbar_wait_sleep(accfull_u32 + 8u * buf, use & 1u, abort_flag, prm.timeout_cycles);
       tc_after();
-      const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(kTN) + (static_cast<uint32_t>(q * 32) << 16);
+      const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(2 * kTN) + static_cast<uint32_t>(cb) +
+                             (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll
-      for (int c32 = 0; c32 < kTN; c32 += 32) {
-        float v[32];
-        tmem_ld32_t(taddr + static_cast<uint32_t>(c32), v);
+      for (int c16 = 0; c16 < kCols; c16 += 16) {
+        float v[16], w[16];
+        tmem_ld16_t(taddr + static_cast<uint32_t>(c16), v);            // main terms
+        tmem_ld16_t(taddr + static_cast<uint32_t>(kTN + c16), w);      // cross terms
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[c32 + j] += v[j];           // rounded to nearest
+        for (int j = 0; j < 16; ++j) acc[c16 + j] += v[j] + w[j];    // rounded to nearest
       }
       tc_before();
       mbar_arrive(accempty_u32 + 8u * buf);
     }
     const long long r = r0 + row;
     if (r < g.rows) {
-      float* Crow = g.C + z * g.c_bs + r * g.c_rs + c0;
-      const float* bias = (g.mode == 1 || g.mode == 2) ? g.bias + z * g.bias_bs + c0 : nullptr;
-      const float* mrow = g.mode == 3 ? g.mask + z * g.mask_bs + r * g.mask_rs + c0 : nullptr;
+      const long long cfirst = c0 + cb;
+      float* Crow = g.C + z * g.c_bs + r * g.c_rs + cfirst;
+      const float* bias = (g.mode == 1 || g.mode == 2) ? g.bias + z * g.bias_bs + cfirst : nullptr;
+      const float* mrow = g.mode == 3 ? g.mask + z * g.mask_bs + r * g.mask_rs + cfirst : nullptr;
       const bool vec = (reinterpret_cast<uintptr_t>(Crow) & 15u) == 0;
 #pragma unroll
-      for (int j = 0; j < kTN; j += 4) {
+      for (int j = 0; j < kCols; j += 4) {
         float o[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const long long c = c0 + j + u;
+          const long long c = cfirst + j + u;
           float v = acc[j + u];
           if (c < g.cols) {
             if (g.mode == 0) v *= g.alpha;
@@ -340,19 +357,19 @@ gemm_tc_kernel(const TcParams prm) {
           }
           o[u] = v;
         }
-        if (vec && c0 + j + 3 < g.cols) {
+        if (vec && cfirst + j + 3 < g.cols) {
           *reinterpret_cast<float4*>(Crow + j) = make_float4(o[0], o[1], o[2], o[3]);
         } else {
 #pragma unroll
           for (int u = 0; u < 4; ++u)
-            if (c0 + j + u < g.cols) Crow[j + u] = o[u];
+            if (cfirst + j + u < g.cols) Crow[j + u] = o[u];
         }
       }
     }
   }
   tc_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == kMmaWarp) {
     tc_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"(static_cast<uint32_t>(kTmemCols))
@@ -377,14 +394,18 @@ bool launch_tc_variant(const TcParams& prm, dim3 grid, cudaStream_t st) {
 bool launch_gemm_tc(const GemmArgs& g, int batch, unsigned* flag, long long timeout_cycles, cudaStream_t st) {
   const bool a_kc = g.a_cs == 1, a_rc = g.a_rs == 1, b_kc = g.b_rs == 1, b_cc = g.b_cs == 1;
   if (!(a_kc || a_rc) || !(b_kc || b_cc)) return false;
-  if (g.rows < 96 || g.cols < 96 || g.K < 64) return false;     // a 128 x 128 tile must be mostly used
+  // a 128 x 128 tile of 32-value k-blocks must be worth it: one large side, and enough work overall
+  if ((g.rows < 96 && g.cols < 96) || g.K < 8 ||
+      static_cast<long long>(g.rows) * g.cols * g.K < (1ll << 21))
+    return false;
   const unsigned gx = static_cast<unsigned>((g.cols + kTN - 1) / kTN), gy = static_cast<unsigned>((g.rows + kTM - 1) / kTM);
   if (gy > 65535u || batch > 65535) return false;
   TcParams prm{g, flag, timeout_cycles};
   const dim3 grid(gx, gy, static_cast<unsigned>(batch));
+  // the three operand layouts the producer has (A row-contiguous with B k-contiguous does not occur)
   if (a_kc && b_kc) return launch_tc_variant<true, true>(prm, grid, st);
   if (a_kc) return launch_tc_variant<true, false>(prm, grid, st);
-  if (b_kc) return launch_tc_variant<false, true>(prm, grid, st);
+  if (b_kc) return false;
   return launch_tc_variant<false, false>(prm, grid, st);
 }
 
