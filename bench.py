@@ -430,6 +430,7 @@ PROFILE_CASES = {
     "stats_bf16_b256": dict(kind="stats", M=1, b=256, d=2_000_000, dtype="bf16"),
     "adamw": dict(kind="adamw", M=8, d=8_000_000),
     "logreg_fused": dict(kind="logreg_fused"),          # the 50 rounds of the logistic configuration, fused
+    "mlp_grads": dict(kind="mlp_grads", M=2, b=1024),   # forward/backward of the 784-1024-1024-10 MLP (tensor-core products)
     # full-size cases of the sweep, for timing only (not for multi-pass captures)
     "stats_f32_b64_d11m": dict(kind="stats", M=1, b=64, d=11_200_000, dtype="f32"),
     "stats_f32_b256_d11m": dict(kind="stats", M=1, b=256, d=11_200_000, dtype="f32"),
@@ -457,6 +458,20 @@ def run_profile_case(args):
     peak, _ = measured_peak()
     if case["kind"] == "logreg_fused":
         print(json.dumps(dict(case=args.case, **logreg_rounds_fused(torch, pkg, inputs, ctx))))
+        ctx.close()
+        return
+    if case["kind"] == "mlp_grads":
+        dims, M, b, n = (784, 1024, 1024, 10), case["M"], case["b"], 65536
+        inp, lab = inputs.gaussian_mixture(5, n, dim=dims[0], classes=dims[3], device="cuda")
+        X = inputs.mlp_init(6, dims, device="cuda").unsqueeze(0).repeat(M, 1).contiguous()
+        idx = inputs.batch_indices(11, (M, b), n, device="cuda")
+        scratch = ctx.mlp_scratch(M, b, dims)
+        Gb = torch.empty((M, ctx.mlp_param_count(dims)), device="cuda")
+        sec = time_steps(torch, lambda i: ctx.abs_mlp_grads(inp, lab, dims, idx, X, b, Gb, scratch), args.steps,
+                         args.warmup)
+        flops = 3 * 2.0 * M * b * (dims[0] * dims[1] + dims[1] * dims[2] + dims[2] * dims[3])   # forward, two backward products
+        print(json.dumps(dict(case=args.case, tune=args.tune, ms=sec * 1e3, TFLOPs=flops / sec / 1e12,
+                              note="fp32-equivalent flops of the matrix products; each runs as 3 TF32 products")))
         ctx.close()
         return
     if case["kind"] == "stats":

@@ -72,18 +72,25 @@ __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint
 __device__ __forceinline__ void umma_commit_t(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// 16 consecutive accumulator columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16_t(uint32_t taddr, float (&v)[16]) {
-  uint32_t r[16];
+// 16 consecutive columns of this thread's TMEM lane from each of two accumulators: both loads in
+// flight, one wait.
+__device__ __forceinline__ void tmem_ld16x2_t(uint32_t taddr0, uint32_t taddr1, float (&v)[16], float (&w)[16]) {
+  uint32_t r[32];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%32];\n\t"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];\n\t"
       "tcgen05.wait::ld.sync.aligned;"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr0), "r"(taddr1)
       : "memory");
 #pragma unroll
-  for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+  for (int j = 0; j < 16; ++j) {
+    v[j] = __uint_as_float(r[j]);
+    w[j] = __uint_as_float(r[16 + j]);
+  }
 }
 // Bounded wait that sleeps between polls, for the warps that wait long (they leave the issue slots
 // to the loaders and the MMA thread).
@@ -327,8 +334,7 @@ gemm_tc_kernel(const TcParams prm) {
 #pragma unroll
       for (int c16 = 0; c16 < kCols; c16 += 16) {
         float v[16], w[16];
-        tmem_ld16_t(taddr + static_cast<uint32_t>(c16), v);            // main terms
-        tmem_ld16_t(taddr + static_cast<uint32_t>(kTN + c16), w);      // cross terms
+        tmem_ld16x2_t(taddr + static_cast<uint32_t>(c16), taddr + static_cast<uint32_t>(kTN + c16), v, w);   // main, cross
 #pragma unroll
         for (int j = 0; j < 16; ++j) acc[c16 + j] += v[j] + w[j];    // rounded to nearest
       }
