@@ -81,9 +81,10 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_stage_kb" (upper bound on one tile buffer, 4..200 KiB),
  * "stats_timeout_cycles" (SM clock cycles a wait for a tile copy may last before
  * the record is flagged ABS_STATUS_TIMEOUT; default about two seconds),
- * "stats_fault_drop_loads" (fault injection for tests: the loaders of the tiled
- * and of the tcgen05 kernel issue no copies, and abs_logreg_rounds_fused sends no
- * partial gradients, so every wait runs out and the records come back flagged
+ * "stats_fault_drop_loads" (fault injection for tests: the loaders of the tiled,
+ * cluster and tcgen05 kernels issue no copies, abs_logreg_rounds_fused sends no
+ * partial gradients and the tensor-core products of the MLP producer fill no
+ * operand tile, so every wait runs out and the records come back flagged
  * ABS_STATUS_TIMEOUT; nothing traps or hangs),
  * "stats_cluster_rows" (target rows per CTA of the cluster kernel, 16..512),
  * "stats_no_cluster" (1 = do not split the rows of a batch over a thread-block

@@ -19,9 +19,11 @@ struct GemmArgs {
 };
 
 // Tensor-core route (tcgen05, 3 x TF32 split products, fp32 accumulation in TMEM folded into fp32
-// registers every 128 values of k).  Returns false when the shape is not worth a 128 x 128 tile or
+// registers every 32 values of k).  Returns false when the shape is not worth a 128 x 128 tile or
 // an operand has no contiguous index; the caller then uses the CUDA-core kernels.
 // `flag`: device word that receives 1 when a bounded wait ran out (the results are then not valid).
-bool launch_gemm_tc(const GemmArgs& g, int batch, unsigned* flag, long long timeout_cycles, cudaStream_t st);
+// `drop_loads`: fault injection for tests (no operand tile is ever filled, so every wait runs out).
+bool launch_gemm_tc(const GemmArgs& g, int batch, unsigned* flag, long long timeout_cycles, bool drop_loads,
+                    cudaStream_t st);
 
 }  // namespace absk

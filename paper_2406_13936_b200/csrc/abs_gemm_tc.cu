@@ -45,6 +45,7 @@ struct TcParams {
   GemmArgs g;
   unsigned* flag;
   long long timeout_cycles;
+  int drop_loads;       // fault injection for the bounded waits: the loaders fill nothing and never arrive
 };
 
 __device__ __forceinline__ void fence_async_smem_t() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -247,6 +248,7 @@ gemm_tc_kernel(const TcParams prm) {
     const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (a_str & 3) == 0;
     const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (b_str & 3) == 0;
     for (int kb = set; kb < n_kb; kb += kLoaderSets) {
+      if (prm.drop_loads) break;                   // test hook: the waits of the other roles must run out, not hang
       const int k0 = kb * kTK;
       const int s = kb % kStagesT;
       const uint32_t pass = static_cast<uint32_t>(kb / kStagesT);
@@ -397,7 +399,8 @@ bool launch_tc_variant(const TcParams& prm, dim3 grid, cudaStream_t st) {
 
 }  // namespace
 
-bool launch_gemm_tc(const GemmArgs& g, int batch, unsigned* flag, long long timeout_cycles, cudaStream_t st) {
+bool launch_gemm_tc(const GemmArgs& g, int batch, unsigned* flag, long long timeout_cycles, bool drop_loads,
+                    cudaStream_t st) {
   const bool a_kc = g.a_cs == 1, a_rc = g.a_rs == 1, b_kc = g.b_rs == 1, b_cc = g.b_cs == 1;
   if (!(a_kc || a_rc) || !(b_kc || b_cc)) return false;
   // a 128 x 128 tile of 32-value k-blocks must be worth it: one large side, and enough work overall
@@ -406,7 +409,7 @@ bool launch_gemm_tc(const GemmArgs& g, int batch, unsigned* flag, long long time
     return false;
   const unsigned gx = static_cast<unsigned>((g.cols + kTN - 1) / kTN), gy = static_cast<unsigned>((g.rows + kTM - 1) / kTM);
   if (gy > 65535u || batch > 65535) return false;
-  TcParams prm{g, flag, timeout_cycles};
+  TcParams prm{g, flag, timeout_cycles, drop_loads ? 1 : 0};
   const dim3 grid(gx, gy, static_cast<unsigned>(batch));
   // the three operand layouts the producer has (A row-contiguous with B k-contiguous does not occur)
   if (a_kc && b_kc) return launch_tc_variant<true, true>(prm, grid, st);

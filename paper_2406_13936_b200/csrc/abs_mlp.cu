@@ -278,7 +278,8 @@ void launch_gemm(abs_ctx* ctx, const GemmArgs& g, int batch, cudaStream_t st) {
   // raises the context's time-out word, which the statistics that follow report
   if (!ctx->tuning.mlp_no_tensor_cores &&
       launch_gemm_tc(g, batch, ctx->flags,
-                     ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles, st))
+                     ctx->tuning.stats_timeout_cycles > 0 ? ctx->tuning.stats_timeout_cycles : kDefaultTimeoutCycles,
+                     ctx->tuning.stats_fault_drop_loads != 0, st))
     return;
   // the large-tile kernel where a 128 x 128 tile is mostly used and both operands have a contiguous index
   const bool a_ok = g.a_cs == 1 || g.a_rs == 1, b_ok = g.b_rs == 1 || g.b_cs == 1;

@@ -360,6 +360,38 @@ def test_mlp_tensor_core_products_match_the_cuda_core_products(ctx, dims, M, b):
             assert t[key] == pytest.approx(c[key], rel=2e-5)
 
 
+def test_mlp_tensor_core_wait_that_runs_out_is_reported(ctx):
+    """Failure detection without a fault: with the operand loaders switched off (test hook) the tensor-core
+    products' waits give up after the shortened limit, tensor memory is freed, the launches end, and the
+    statistics that follow carry ABS_STATUS_TIMEOUT; the next ordinary pass on the same context is
+    correct again (the same records as a context that never timed out)."""
+    dims, M, b, n = (200, 257, 191, 10), 2, 130, 2000
+    inp, lab, X = mlp_problem(7, n, dims, M)
+    d = ctx.mlp_param_count(dims)
+    idx = inputs.batch_indices(8, (M, b), n, device="cuda")
+
+    def run():
+        scratch = ctx.mlp_scratch(M, b, dims)
+        Gb = torch.zeros((M, d), device="cuda")
+        ctx.abs_mlp_grads(inp, lab, dims, idx, X, b, Gb, scratch)
+        st = ctx.new_stats(M)
+        ctx.abs_mlp_fused_stats(dims, b, scratch, Gb, st)
+        torch.cuda.synchronize()
+        return pkg.stats_to_dicts(st)
+
+    good = run()
+    ctx.set_tuning("stats_timeout_cycles", 2_000_000)        # about a millisecond
+    ctx.set_tuning("stats_fault_drop_loads", 1)
+    try:
+        flagged = run()
+    finally:
+        ctx.set_tuning("stats_fault_drop_loads", 0)
+        ctx.set_tuning("stats_timeout_cycles", 0)
+    assert all(r["status"] & pkg.binding.STATUS_TIMEOUT for r in flagged)
+    assert all(r["status"] == 0 for r in good)
+    assert run() == good
+
+
 @pytest.mark.parametrize("dims,M,b", [((20, 33, 17, 7), 3, 9), ((70, 130, 65, 10), 2, 67),
                                       ((784, 1024, 1024, 10), 2, 40), ((784, 1024, 1024, 10), 1, 600)])
 def test_mlp_fused_statistics_match_materialised_gradients(ctx, dims, M, b):
