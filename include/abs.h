@@ -124,7 +124,7 @@ typedef struct {
 } abs_stats;          /* 56 bytes */
 
 /* Batch-size test statistics of M workers (Eq. def_var applied per worker,
- * Eq. approx_norm_local; Algorithm 1, "compute Var").
+ * Eq. approx_norm_local; Algorithm 1, variance step).
  *   G            [M][b][d] per-sample (or per-micro-batch) gradients, dtype fp32
  *                or bf16; element (m,i,j) at G[m*worker_stride + i*row_stride + j]
  *   M >= 1, b >= 2 (the variance divides by b-1), d >= 1,

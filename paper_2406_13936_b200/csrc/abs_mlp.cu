@@ -1,7 +1,7 @@
 // Producer for the MLP end-to-end problem: forward and backward pass of a three-layer ReLU
 // classifier with softmax cross-entropy for M workers at once, the batch gradients, and -- for
-// the batch-size test -- the per-sample gradients written out as rows (Algorithm 1, "compute
-// per-sample gradients"; they are outer products delta_l,i (x) h_{l-1},i).
+// the batch-size test -- the per-sample gradients written out as rows (Algorithm 1, per-sample
+// gradient step; they are outer products delta_l,i (x) h_{l-1},i).
 //
 // Parameter layout of one replica (flat, fp32): W1 [n1][n0], b1 [n1], W2 [n2][n1], b2 [n2],
 // W3 [n3][n2], b3 [n3], each W row-major [out][in].

@@ -6,8 +6,9 @@
 //   ReLU MLP              softmax cross-entropy; per-sample gradients are outer products
 //                         delta_l,i (x) h_{l-1},i, written out row by row when the test needs them
 //
-// These kernels feed the hot path; they are plain fp32 CUDA-core code (the parity bound on the
-// parameters, 1e-6, rules out reduced-precision tensor-core products).
+// These kernels feed the hot path.  The logistic producer is plain fp32 CUDA-core code; the MLP's
+// matrix products run on the tensor cores with operands split so that the result keeps fp32
+// accuracy (abs_gemm_tc.cu), which the parity bound on the parameters, 1e-6, needs.
 #include "abs_internal.cuh"
 
 namespace absk {
