@@ -409,9 +409,12 @@ bool cluster_geometry(const Tuning& t, size_t smem_optin, int es, long long b, i
 // copies were also tried: 40 % slower.
 int preferred_cluster_size(const Tuning& t, long long b) {
   const int want_rows = t.stats_cluster_rows > 0 ? static_cast<int>(t.stats_cluster_rows) : (b > 2048 ? 512 : 256);
-  int C = 2;
-  while (C < kMaxCluster && (b + C - 1) / C > want_rows) C *= 2;
-  return C;
+  // the fewest CTAs that leave each at most want_rows rows: any size from 2 to 8 (not only powers of
+  // two), because fuller tiles matter more than how evenly the clusters tile the GPU
+  long long C = (b + want_rows - 1) / want_rows;
+  if (C < 2) C = 2;
+  if (C > kMaxCluster) C = kMaxCluster;
+  return static_cast<int>(C);
 }
 
 // One launch (or one occupancy query) of the variant that fits the geometry.
@@ -550,7 +553,7 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
 // smaller clusters when the larger one cannot be scheduled.
 int launch_stats_cluster(abs_ctx* ctx, const StatsLaunch& a, int* P_out) {
   if (a.b <= 256 || a.b > kMaxFastRows || !tma_addressable(a)) return ABS_ERR_UNSUPPORTED;
-  for (int C = preferred_cluster_size(ctx->tuning, a.b); C >= 2; C /= 2) {
+  for (int C = preferred_cluster_size(ctx->tuning, a.b); C >= 2; --C) {
     const int rc = try_cluster_size(ctx, a, C, P_out);
     if (rc != ABS_ERR_UNSUPPORTED) return rc;
   }

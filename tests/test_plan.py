@@ -56,7 +56,7 @@ def check_plan(dtype, b, p):
     assert p["warps_per_box"] * p["boxes_per_stage"] == 8
     if p["route"] == 1:
         C = p["cluster_size"]
-        assert C in (2, 4, 8, 16) and p["rows_per_cta"] * C >= b and p["rows_per_cta"] <= 512
+        assert 2 <= C <= 8 and p["rows_per_cta"] * C >= b and p["rows_per_cta"] <= 512
         assert (C - 1) * p["rows_per_cta"] < b               # no CTA of the cluster is left without rows
         assert row_bytes >= 128
         if p["full"]:
