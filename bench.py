@@ -26,6 +26,7 @@ WORKLOAD = dict(name="stats sweep centre: G fp32 [M=1, b=256, d=11.2M], sigma=1,
                 M=1, b=256, d=11_200_000, sigma=1.0, seed=2)
 HP = dict(lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
 FALLBACK_HBM_GBS = 6650.0
+LEG_PAUSE_S = 0.5
 # DRAM bytes (read + write) of one abs_stats_tiled_kernel<float,16,keep,full> launch on the 1.024 GB case
 # of profiles/stats_tiled_f32_b256_d1m.txt; traffic grows in proportion to the columns processed.
 NCU_TRAFFIC_SMALL = dict(dram_bytes=1.024040e9 + 3.832e6, d=1_000_000)
@@ -235,7 +236,11 @@ def aggregate_over_ranks(seconds, units_per_rank, dist=None, device="cuda"):
 
 # --------------------------------------------------------------------------- GPU legs
 def time_steps(torch, fn, steps, warmup):
-    """CUDA-event timing of `steps` calls of fn(i) after `warmup` untimed ones; returns seconds per call."""
+    """CUDA-event timing of `steps` calls of fn(i) after `warmup` untimed ones; returns seconds per call.
+    Every leg starts from an idle GPU (a short pause): a leg measured right after a long one ran
+    10-35 % slower here."""
+    torch.cuda.synchronize()
+    time.sleep(LEG_PAUSE_S)
     for i in range(warmup):
         fn(i)
     torch.cuda.synchronize()

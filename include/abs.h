@@ -94,7 +94,8 @@ const char* abs_last_error(const abs_ctx* ctx);
  * "stats_no_secondary" (1 = the cluster kernel leaves the SMs idle that its
  * clusters cannot occupy instead of giving them a second launch of two-CTA
  * clusters), "stats_secondary_pct" (the speed of an SM of that second launch in
- * per cent of an SM of the first, which sets its share of the columns; 0 = 95),
+ * per cent of an SM of the first, which sets its share of the columns; 0 = 95, or 80 for rows
+ * more than 64 MB apart),
  * "stats_no_gram" (1 = do not use the tensor-core Gram kernels for bf16, b <= 256),
  * "stats_no_recheck" (1 = keep a Gram kernel's record even when its sums are
  * ill-conditioned, i.e. never recompute it with the tiled kernel),

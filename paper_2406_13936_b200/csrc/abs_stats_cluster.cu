@@ -504,7 +504,12 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
     // the first launch (measured: the two finish together at about 100, and every per cent beyond
     // that costs a per cent of the whole call, so the default stays a little below); at least 64
     // strips per cluster
-    const long long pct = ctx->tuning.stats_secondary_pct > 0 ? ctx->tuning.stats_secondary_pct : 95;
+    // (rows further apart than about 64 MB: a CTA of the second launch touches 512 of them per tile and
+    // misses the TLB more often than one of the first with its 256; measured at a 102 MB row stride the
+    // two finish together at 80)
+    const long long row_bytes = a.row_stride * es;
+    const long long pct = ctx->tuning.stats_secondary_pct > 0 ? ctx->tuning.stats_secondary_pct
+                                                               : (row_bytes > (64ll << 20) ? 80 : 95);
     const double w2 = static_cast<double>(n2 * C2) * pct / 100.0;
     cols_second = static_cast<long long>(static_cast<double>(a.d) * w2 / (static_cast<double>(n1 * C) + w2));
     if (n2 < 1 || cols_second < 64 * n2 * geo2.cols) n2 = 0;
