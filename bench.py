@@ -285,6 +285,16 @@ def extra_legs(torch, pkg, inputs, ctx, peak, steps, warmup):
     # the nine cells of the statistics sweep (behind the short legs above, before the long ones below)
     out["sweep"] = stats_sweep(torch, pkg, inputs, ctx, peak, steps, warmup)
     out["worst_cell"] = worst_cell(out["sweep"])
+    # the sweep's other two noise levels on its centre cell: the same bytes are read whatever sigma is
+    out["sweep_sigma"] = []
+    for sigma in (0.1, 10.0):
+        G = inputs.gaussian_rows(2, 1, 256, 11_200_000, sigma, device="cuda")
+        stats = ctx.new_stats(1)
+        sec = time_steps(torch, lambda i: ctx.abs_test_stats(G, stats), 10, 3)
+        gbs = G.numel() * 4 / sec / 1e9
+        out["sweep_sigma"].append(dict(b=256, d=11_200_000, sigma=sigma, ms=sec * 1e3, GBps=gbs, frac_of_peak=gbs / peak))
+        del G
+        torch.cuda.empty_cache()
     free = torch.cuda.mem_get_info()[0]
     # fused local AdamW + averaging: M=8 fp32 replicas of a GPT-2-small-sized model, H=16 steps per round
     M, d, H = 8, 124_439_808, 16
@@ -343,6 +353,10 @@ def extra_legs(torch, pkg, inputs, ctx, peak, steps, warmup):
         out["rounds_logreg_fused"] = logreg_rounds_fused(torch, pkg, inputs, ctx)
     except pkg.AbsError as e:      # e.g. a tool that refuses cooperative cluster launches
         out["rounds_logreg_fused"] = dict(unavailable=str(e))
+    try:
+        out["rounds_logreg_fused_every_step"] = logreg_rounds_fused(torch, pkg, inputs, ctx, every_step=True)
+    except pkg.AbsError as e:
+        out["rounds_logreg_fused_every_step"] = dict(unavailable=str(e))
     out["rounds_mlp"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp")
     out["rounds_mlp_fused_stats"] = end_to_end_rounds(torch, pkg, inputs, ctx, "mlp_fused")
     return out
@@ -389,30 +403,41 @@ def end_to_end_rounds(torch, pkg, inputs, ctx, which):
                 b_last=history[-1], rounds_until_cap=next((i for i, v in enumerate(history) if v >= b_max), None))
 
 
-def logreg_rounds_fused(torch, pkg, inputs, ctx):
+def logreg_rounds_fused(torch, pkg, inputs, ctx, every_step=False):
     """The logistic configuration with all 50 rounds in one cooperative launch (abs_logreg_rounds_fused:
     parameters in shared memory, batch size on the device, no per-sample gradient matrix), and with one
-    launch per round; CUDA-event time of the launches, after one untimed run."""
+    launch per round; CUDA-event time of the launches, after one untimed run.  every_step: Algorithm 1's
+    cadence (the test after every local step, one size per worker, sample counter on the device)."""
     n, d, M, H, lr, b0, b_max, rounds = 65536, 256, 4, 8, 0.1, 16, 1024, 50
     A, y = inputs.logreg_dataset(1, n, d, device="cuda")
     cfg = pkg.make_test_cfg("norm", b_max, eta=0.5)
     idx = inputs.batch_indices(11, (rounds, H, M, b_max), n, device="cuda")
-    stats = ctx.new_stats(rounds * M)
-    hist = torch.zeros(rounds + 1, dtype=torch.int64, device="cuda")
+    per = H if every_step else 1
+    stats = ctx.new_stats(rounds * per * M)
+    hist = torch.zeros((rounds + 1) if not every_step else (rounds * H * M), dtype=torch.int64, device="cuda")
     out = dict(rounds=rounds, M=M, H=H)
+    ctl = ctx.new_round_ctl() if every_step else None
+    opts = pkg.make_round_opts(test_every_step=True, per_worker=True, ctl=ctl) if every_step else None
     for mode in ("one_launch", "launch_per_round"):
         best = None
         for rep in range(4):
             X = torch.zeros((M, d), device="cuda")
-            b_dev = torch.tensor([b0], dtype=torch.int64, device="cuda")
+            b_dev = torch.full((M if every_step else 1,), b0, dtype=torch.int64, device="cuda")
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
             e0.record()
             if mode == "one_launch":
-                ctx.abs_logreg_rounds_fused(A, y, idx, X, H, lr, cfg, stats, b_dev, b_hist=hist)
+                if every_step:
+                    ctx.abs_logreg_rounds_fused_opts(A, y, idx, X, H, lr, cfg, opts, stats, b_dev, b_hist=hist)
+                else:
+                    ctx.abs_logreg_rounds_fused(A, y, idx, X, H, lr, cfg, stats, b_dev, b_hist=hist)
             else:
                 for k in range(rounds):
-                    ctx.abs_logreg_rounds_fused(A, y, idx[k:k + 1], X, H, lr, cfg, stats[k * M:(k + 1) * M], b_dev)
+                    if every_step:
+                        ctx.abs_logreg_rounds_fused_opts(A, y, idx[k:k + 1], X, H, lr, cfg, opts,
+                                                         stats[k * per * M:(k + 1) * per * M], b_dev)
+                    else:
+                        ctx.abs_logreg_rounds_fused(A, y, idx[k:k + 1], X, H, lr, cfg, stats[k * M:(k + 1) * M], b_dev)
             e1.record()
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1)
@@ -420,7 +445,10 @@ def logreg_rounds_fused(torch, pkg, inputs, ctx):
                 best = ms if best is None else min(best, ms)
         out[mode] = dict(rounds_per_s=rounds / (best * 1e-3), us_per_round=best * 1e3 / rounds)
     h = hist.tolist()
-    out.update(b_first=h[0], b_last=h[-1], rounds_until_cap=next((i for i, v in enumerate(h) if v >= b_max), None))
+    if every_step:
+        out.update(b_first=h[0], b_last=max(h), samples=int(ctl[0].item()))
+    else:
+        out.update(b_first=h[0], b_last=h[-1], rounds_until_cap=next((i for i, v in enumerate(h) if v >= b_max), None))
     return out
 
 

@@ -445,6 +445,8 @@ def _device_gib_free():
 FULL_WIDTH = [
     # (dtype, b, d, recipe, route)   the oracle gets the whole matrix: every column is independent
     (torch.float32, 64, 11_200_000, "gauss", 2),       # tiled kernel, a column of the sweep
+    (torch.float32, 64, 11_200_000, "gauss0.1", 2),    # the sweep's other noise levels: mean-dominated ...
+    (torch.float32, 256, 2_800_000, "gauss10", 2),     # ... and noise-dominated
     (torch.float32, 16, 25_600_000, "gauss", 2),       # tiled kernel, widest rows of the sweep
     (torch.float32, 320, 2_800_000, "gauss", 1),       # cluster kernel (2 CTAs x 160 rows)
     (torch.float32, 1100, 1_000_000, "gauss", 1),      # cluster kernel, last CTA short of rows
@@ -467,7 +469,8 @@ def test_full_width_independent_columns_against_the_oracle(ctx, dtype, b, d, rec
     if recipe == "student":
         G = inputs.student_t_rows(31, 1, b, d, device="cuda", dtype=dtype)
     else:
-        G = inputs.gaussian_rows(31 + b, 1, b, d, 1.0, device="cuda", dtype=dtype)
+        sigma = float(recipe[5:]) if len(recipe) > 5 else 1.0
+        G = inputs.gaussian_rows(31 + b, 1, b, d, sigma, device="cuda", dtype=dtype)
     recs, gbar = run_gpu(ctx, G)
     H = to_f64(G)[0]
     del G
