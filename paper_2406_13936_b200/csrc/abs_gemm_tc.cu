@@ -130,9 +130,15 @@ __device__ __forceinline__ void split4(const float4 a, float4& hi, float4& lo) {
   split_tf32(a.w, hi.w, lo.w);
 }
 
-// Four consecutive elements starting at p; elements at or past `left` read as zero.
+// Four consecutive elements starting at p; elements at or past `left` read as zero.  `vec`: p is
+// 16-byte aligned; else 8-byte alignment is tried (odd replicas of a parameter vector of odd
+// half-length are 8 bytes off).
 __device__ __forceinline__ float4 load4_guard(const float* p, long long left, bool vec) {
   if (left >= 4 && vec) return __ldg(reinterpret_cast<const float4*>(p));
+  if (left >= 4 && (reinterpret_cast<uintptr_t>(p) & 7u) == 0) {
+    const float2 a = __ldg(reinterpret_cast<const float2*>(p)), b = __ldg(reinterpret_cast<const float2*>(p) + 1);
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
   float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
   if (left > 0) v.x = __ldg(p);
   if (left > 1) v.y = __ldg(p + 1);
