@@ -177,17 +177,19 @@ abs_stats_finalize_kernel(double* ws, long long b, int P, unsigned* __restrict__
     const long long r = r0 + col;
     double e = 0.0;
     if (r < r_end) {
-      // eight loads are issued before the first sum needs one (a load per iteration would cost a
-      // round trip to L2 each); the sums are still taken in the order of p
-      int p = grp;
-      for (; p + 7 * tpr < P; p += 8 * tpr) {
-        double v[8];
+      // sixteen loads are issued before the first sum needs one (a load per iteration would cost a
+      // round trip to L2 each; so would a scalar tail, hence the predicated last batch: adding 0.0
+      // changes nothing); the sums are still taken in the order of p
+      for (int p0 = grp; p0 < P; p0 += 16 * tpr) {
+        double v[16];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = base[static_cast<size_t>(p + u * tpr) * rec + r];
+        for (int u = 0; u < 16; ++u) {
+          const int p = p0 + u * tpr;
+          v[u] = p < P ? base[static_cast<size_t>(p) * rec + r] : 0.0;
+        }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) e += v[u];
+        for (int u = 0; u < 16; ++u) e += v[u];
       }
-      for (; p < P; p += tpr) e += base[static_cast<size_t>(p) * rec + r];
     }
     esum[tid] = e;
     __syncthreads();
