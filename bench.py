@@ -416,11 +416,13 @@ def logreg_rounds_fused(torch, pkg, inputs, ctx, every_step=False):
     stats = ctx.new_stats(rounds * per * M)
     hist = torch.zeros((rounds + 1) if not every_step else (rounds * H * M), dtype=torch.int64, device="cuda")
     out = dict(rounds=rounds, M=M, H=H)
-    ctl = ctx.new_round_ctl() if every_step else None
-    opts = pkg.make_round_opts(test_every_step=True, per_worker=True, ctl=ctl) if every_step else None
+    ctl, opts = None, None
     for mode in ("one_launch", "launch_per_round"):
         best = None
         for rep in range(4):
+            if every_step:     # fresh counters for every run
+                ctl = ctx.new_round_ctl()
+                opts = pkg.make_round_opts(test_every_step=True, per_worker=True, ctl=ctl)
             X = torch.zeros((M, d), device="cuda")
             b_dev = torch.full((M if every_step else 1,), b0, dtype=torch.int64, device="cuda")
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
