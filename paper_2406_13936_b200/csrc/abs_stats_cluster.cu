@@ -492,11 +492,11 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
   ClusterGeom geo2;
   long long n2 = 0, cols_second = 0;
   const long long idle = ctx->sm_count - n1 * a.M * C;
-  // Only pairs are known to fit what four-CTA clusters leave over; clusters of four beside clusters
-  // of eight were tried (b = 2048) and mostly ran after the first launch instead of beside it:
-  // 6.7 -> 8.8 ms.
+  // Only pairs are known to fit what clusters of three or four leave over; clusters of four beside
+  // clusters of eight were tried (b = 2048) and mostly ran after the first launch instead of beside
+  // it: 6.7 -> 8.8 ms.
   const int C2 = 2;
-  if (C == 4 && !ctx->tuning.stats_no_secondary && ctx->tuning.stats_ctas_per_worker == 0 && idle >= C2 &&
+  if ((C == 3 || C == 4) && !ctx->tuning.stats_no_secondary && ctx->tuning.stats_ctas_per_worker == 0 && idle >= C2 &&
       n1 * a.M == (static_cast<long long>(max_clusters) / a.M) * a.M &&
       cluster_geometry(ctx->tuning, ctx->smem_optin, es, a.b, C2, &geo2)) {
     n2 = (idle / C2) / a.M;
@@ -504,12 +504,13 @@ int try_cluster_size(abs_ctx* ctx, const StatsLaunch& a, int C, int* P_out) {
     // the first launch (measured: the two finish together at about 100, and every per cent beyond
     // that costs a per cent of the whole call, so the default stays a little below); at least 64
     // strips per cluster
-    // (rows further apart than about 64 MB: a CTA of the second launch touches 512 of them per tile and
+    // (beside clusters of three the pairs were worth 60: b = 768, 6.09 -> 6.39 TB/s, and 95 lost; rows
+    // further apart than about 64 MB: a CTA of the second launch touches 512 of them per tile and
     // misses the TLB more often than one of the first with its 256; measured at a 102 MB row stride the
     // two finish together at 80)
     const long long row_bytes = a.row_stride * es;
     const long long pct = ctx->tuning.stats_secondary_pct > 0 ? ctx->tuning.stats_secondary_pct
-                                                               : (row_bytes > (64ll << 20) ? 80 : 95);
+                                                               : (C == 3 ? 60 : (row_bytes > (64ll << 20) ? 80 : 95));
     const double w2 = static_cast<double>(n2 * C2) * pct / 100.0;
     cols_second = static_cast<long long>(static_cast<double>(a.d) * w2 / (static_cast<double>(n1 * C) + w2));
     if (n2 < 1 || cols_second < 64 * n2 * geo2.cols) n2 = 0;
