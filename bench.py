@@ -387,15 +387,25 @@ def end_to_end_rounds(torch, pkg, inputs, ctx, which):
     Gb = torch.empty((M, d), device="cuda")
     stats = ctx.new_stats(M)
     b_dev = torch.tensor([b], dtype=torch.int64, device="cuda")
-    history = [b]
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for k in range(rounds):
+    def one_round(k, b):
         if which == "logreg":
             ctx.abs_logreg_round(A, y, idx[k], X, H, b, lr, cfg, G, Gb, stats, b_dev)
         else:
             ctx.abs_mlp_round(inp, lab, dims, idx[k], X, H, b, lr, cfg, scratch, G, stride, Gb, stats, b_dev)
-        b = int(b_dev.item())          # one 8-byte read-back per round
+        return int(b_dev.item())       # one 8-byte read-back per round
+
+    # three untimed rounds (module loading, first-call queries), then the run starts over from x_0, b_0
+    X0, b0 = X.clone(), b
+    for k in range(3):
+        b = one_round(k, b)
+    X.copy_(X0)
+    b = b0
+    b_dev.fill_(b0)
+    history = [b]
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for k in range(rounds):
+        b = one_round(k, b)
         history.append(b)
     torch.cuda.synchronize()
     sec = time.perf_counter() - t0

@@ -37,6 +37,28 @@ struct Tuning {
   long long stats_fault_drop_loads = 0;    // test hook: the tiled kernel's loader issues no copies
 };
 
+// What the launchers remember per kernel function, so that a call does not repeat host-side runtime
+// queries whose answers cannot change: the largest dynamic shared-memory size already granted
+// (cudaFuncSetAttribute costs about a microsecond per call) and, for cluster kernels, how many
+// clusters of a given size and shared-memory footprint can be resident at once
+// (cudaOccupancyMaxActiveClusters costs tens of microseconds).
+struct FnCache {
+  static constexpr int kSlots = 128;
+  const void* fn[kSlots] = {};
+  size_t smem_granted[kSlots] = {};
+  int cluster_size[kSlots] = {};
+  size_t cluster_smem[kSlots] = {};
+  int max_clusters[kSlots] = {};
+  int n = 0;
+  int slot(const void* f) {            // index of f's entry, created if there is room; -1 otherwise
+    for (int i = 0; i < n; ++i)
+      if (fn[i] == f) return i;
+    if (n == kSlots) return -1;
+    fn[n] = f;
+    return n++;
+  }
+};
+
 }  // namespace absk
 
 // The context: device, workspace for per-CTA partial sums, a device staging area
@@ -55,12 +77,24 @@ struct abs_ctx {
   void* staging_out = nullptr;     // device buffer for stats / gbar of *_host calls
   size_t staging_out_bytes = 0;
   absk::Tuning tuning;
+  absk::FnCache fn_cache;
   char err[512] = {0};
 };
 
 namespace absk {
 
 int set_error(abs_ctx* ctx, int code, const char* fmt, ...);
+
+// Grants `kernel` at least `smem` bytes of dynamic shared memory (once per context and size).
+template <typename K>
+inline cudaError_t ensure_dynamic_smem(abs_ctx* ctx, K kernel, size_t smem) {
+  const void* f = reinterpret_cast<const void*>(kernel);
+  const int i = ctx->fn_cache.slot(f);
+  if (i >= 0 && ctx->fn_cache.smem_granted[i] >= smem) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e == cudaSuccess && i >= 0) ctx->fn_cache.smem_granted[i] = smem;
+  return e;
+}
 
 #define ABS_CUDA_TRY(ctx, expr)                                                          \
   do {                                                                                   \

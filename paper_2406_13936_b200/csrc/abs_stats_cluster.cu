@@ -332,7 +332,7 @@ template <typename T, int RMAX, bool FULL>
 int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams prm, const StatsLaunch& a, int C,
                            size_t smem, const ClusterShare& share) {
   auto kern = abs_stats_cluster_kernel<T, RMAX, FULL>;
-  ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  ABS_CUDA_TRY(ctx, ensure_dynamic_smem(ctx, kern, smem));
   if (C > 8 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
     cudaGetLastError();
     return ABS_ERR_UNSUPPORTED;
@@ -351,6 +351,11 @@ int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams 
   cfg.attrs = attr;
   cfg.numAttrs = share.beside_previous ? 2 : 1;
   if (share.n_clusters == 0) {
+    const int slot = ctx->fn_cache.slot(reinterpret_cast<const void*>(kern));
+    if (slot >= 0 && ctx->fn_cache.cluster_size[slot] == C && ctx->fn_cache.cluster_smem[slot] == smem) {
+      *share.max_clusters_out = ctx->fn_cache.max_clusters[slot];     // asked before: the answer cannot change
+      return ABS_OK;
+    }
     cfg.gridDim = dim3(static_cast<unsigned>(C), 1, 1);
     cfg.numAttrs = 1;
     int max_clusters = 0;
@@ -360,6 +365,11 @@ int launch_cluster_variant(abs_ctx* ctx, const CUtensorMap& tmap, ClusterParams 
       set_error(ctx, ABS_ERR_UNSUPPORTED, "a cluster of %d CTAs cannot be scheduled (%s, %d clusters)", C,
                 cudaGetErrorString(occ), max_clusters);
       return ABS_ERR_UNSUPPORTED;
+    }
+    if (slot >= 0) {
+      ctx->fn_cache.cluster_size[slot] = C;
+      ctx->fn_cache.cluster_smem[slot] = smem;
+      ctx->fn_cache.max_clusters[slot] = max_clusters;
     }
     *share.max_clusters_out = max_clusters;
     return ABS_OK;

@@ -296,7 +296,7 @@ template <int NB, bool WANT_GBAR>
 int launch_gram_variant(abs_ctx* ctx, const CUtensorMap& tmap, const GramParams& prm, dim3 grid, size_t smem,
                         cudaStream_t stream) {
   auto kern = abs_stats_gram_kernel<NB, WANT_GBAR>;
-  ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  ABS_CUDA_TRY(ctx, ensure_dynamic_smem(ctx, kern, smem));
   kern<<<grid, kThreadsG, smem, stream>>>(tmap, prm);
   ABS_CUDA_TRY(ctx, cudaGetLastError());
   return ABS_OK;

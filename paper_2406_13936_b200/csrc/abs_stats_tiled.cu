@@ -408,7 +408,7 @@ template <typename T, int RMAX, bool KEEP, bool FULL>
 int launch_variant(abs_ctx* ctx, const CUtensorMap& tmap, const TiledParams& prm, dim3 grid, size_t smem,
                    cudaStream_t stream) {
   auto kern = abs_stats_tiled_kernel<T, RMAX, KEEP, FULL>;
-  ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  ABS_CUDA_TRY(ctx, ensure_dynamic_smem(ctx, kern, smem));
   kern<<<grid, kThreads, smem, stream>>>(tmap, prm);
   ABS_CUDA_TRY(ctx, cudaGetLastError());
   return ABS_OK;

@@ -565,7 +565,7 @@ bool umma_geometry(const Tuning& t, size_t smem_optin, long long b, UmmaGeom* g)
 template <int MB, bool WANT_GBAR>
 int launch_umma_variant(abs_ctx* ctx, const UmmaParams& prm, dim3 grid, size_t smem, cudaStream_t stream) {
   auto kern = abs_stats_umma_kernel<MB, WANT_GBAR>;
-  ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  ABS_CUDA_TRY(ctx, ensure_dynamic_smem(ctx, kern, smem));
   kern<<<grid, WANT_GBAR ? 416 : 288, smem, stream>>>(prm);
   ABS_CUDA_TRY(ctx, cudaGetLastError());
   return ABS_OK;
