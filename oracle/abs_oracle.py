@@ -482,3 +482,35 @@ def run_until_samples(X0, per_sample_grads, H, lr, b0, b_max, kind, n_samples, p
             b = b_next
         k += 1
     return X[0].copy(), k, B, history
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 2 as printed: the test on the workers' batch gradients
+# ----------------------------------------------------------------------------
+def local_round_worker_test(X, batch_grads, H, lr, b_cur, b_max, eta):
+    """One round of Alg. 2 ("actual implementation"): H local SGD steps per worker on batch
+    gradients only, model averaging, then the norm test from the WORKERS' batch gradients:
+        gbar = (1/M) sum_m g^m,
+        Var  = b * 1/(M-1) sum_m ||g^m - gbar||^2          (the estimator of Section 4.3),
+        T    = ceil( Var / (M eta^2 ||gbar||^2) )          (Eq. test_stat_actual),
+        b_next = max{T, b}  (capped at the maximum local batch size),
+    where g^m is worker m's batch gradient of the round's last local step (the gradients that
+    exist when the models are synchronised).  The sample counter grows by H M b.
+
+    X [M, d]; batch_grads(m, h, x) returns the batch gradient [d] of worker m at local step h.
+    Returns (X_next, b_next, T, stats of the M gradients as rows, samples).
+    """
+    X = np.array(X, dtype=np.float64)
+    M = X.shape[0]
+    if M < 2:
+        raise ValueError("the variance over workers needs M >= 2")
+    Gb = np.empty_like(X)
+    for h in range(H):
+        for m in range(M):
+            Gb[m] = np.asarray(batch_grads(m, h, X[m]), dtype=np.float64)
+        X = sgd_step(X, Gb, lr)
+    X = replica_average(X)
+    stats = batch_test_stats(Gb)                      # rows = workers: var_norm = 1/(M-1) sum ||g^m - gbar||^2
+    T = batch_test_statistic(stats, "norm", eta=eta, row_weight=float(b_cur), divisor=float(M))
+    b_next = min(b_max, max(b_cur, T))
+    return X, b_next, T, stats, samples_of_round(H, M, b_cur)

@@ -497,3 +497,23 @@ def test_sample_counter_and_stop_rule():
                                               per_step=True, shared=False, eta=0.5)
         assert K == K_exp and hist[0] == [2, 2] and (B == 9 if K == 1 else B > 9)
     assert hist[1] == [3, 2]                               # the second round starts from the sizes the first ended with
+
+
+def test_worker_gradient_round_by_hand():
+    # Alg. 2 on f(x; xi) = 0.5 (x - xi)^2 with two workers, one dimension, H = 2, lr = 1/2, b = 4, eta = 1/2.
+    # Batch gradients are x - (mean of the worker's batch), here given directly as x - c[m][h]:
+    #   worker 1: c = 1 then 2:  x: 3 -> 3 - (3-1)/2 = 2 -> g = 2 - 2 = 0,  x stays 2
+    #   worker 2: c = 5 then 6:  x: 3 -> 3 - (3-5)/2 = 4 -> g = 4 - 6 = -2, x = 4 + 1 = 5
+    # average (2 + 5) / 2 = 3.5; gbar = -1, ||gbar||^2 = 1; 1/(M-1) sum (g - gbar)^2 = 1 + 1 = 2;
+    # Var = b * 2 = 8; T = ceil(8 / (2 * (1/4) * 1)) = 16; B += H M b = 16.
+    c = [[1.0, 2.0], [5.0, 6.0]]
+    X, b_next, T, stats, samples = orc.local_round_worker_test(
+        np.array([[3.0], [3.0]]), lambda m, h, x: x - c[m][h], 2, 0.5, 4, 1000, 0.5)
+    np.testing.assert_allclose(X, [[3.5], [3.5]], rtol=1e-15)
+    assert stats["gbar_sq"] == pytest.approx(1.0, rel=1e-15) and stats["var_norm"] == pytest.approx(2.0, rel=1e-15)
+    assert (T, b_next, samples) == (16, 16, 16)
+    # capped, and never smaller than the current size
+    assert orc.local_round_worker_test(np.array([[3.0], [3.0]]), lambda m, h, x: x - c[m][h], 2, 0.5, 4, 10, 0.5)[1] == 10
+    assert orc.local_round_worker_test(np.array([[3.0], [3.0]]), lambda m, h, x: x - c[m][h], 2, 0.5, 40, 100, 0.5)[1] == 40
+    # the estimator: for batch gradients that are means of b i.i.d. samples, b * Var_m(g^m) estimates the
+    # per-sample variance (Section 4.3); checked in expectation elsewhere (test_worker_gradient_estimator_...)
