@@ -514,6 +514,9 @@ def test_worker_gradient_round_by_hand():
     assert (T, b_next, samples) == (16, 16, 16)
     # capped, and never smaller than the current size
     assert orc.local_round_worker_test(np.array([[3.0], [3.0]]), lambda m, h, x: x - c[m][h], 2, 0.5, 4, 10, 0.5)[1] == 10
-    assert orc.local_round_worker_test(np.array([[3.0], [3.0]]), lambda m, h, x: x - c[m][h], 2, 0.5, 40, 100, 0.5)[1] == 40
+    # gradients that nearly agree (g^1 = 1, g^2 = 1.2): ratio b (g1-g2)^2 / (eta^2 (g1+g2)^2) = 40 * 0.04 / 1.21, T = 2 < b
+    c2 = [[1.0, 1.0], [5.0, 2.8]]
+    _, b_next, T, _, _ = orc.local_round_worker_test(np.array([[3.0], [3.0]]), lambda m, h, x: x - c2[m][h], 2, 0.5, 40, 100, 0.5)
+    assert (T, b_next) == (2, 40)
     # the estimator: for batch gradients that are means of b i.i.d. samples, b * Var_m(g^m) estimates the
     # per-sample variance (Section 4.3); checked in expectation elsewhere (test_worker_gradient_estimator_...)
