@@ -230,7 +230,16 @@ int abs_test_stats_noalloc(const void* G, abs_dtype dtype, int M, long long b, l
 /* Message of the last failing abs_test_stats_noalloc call on this thread. */
 const char* abs_noalloc_last_error(void);
 
-typedef enum { ABS_TEST_NORM = 0, ABS_TEST_AUG_INNER_PRODUCT = 1 } abs_test_kind;
+typedef enum {
+  ABS_TEST_NORM = 0,               /* norm test on the rows of G (Eq. approx_norm_local)               */
+  ABS_TEST_AUG_INNER_PRODUCT = 1,  /* augmented inner-product test on the rows of G                    */
+  ABS_TEST_NORM_WORKERS = 2        /* Algorithm 2 ("actual implementation"): the norm test on the M
+                                      workers' BATCH gradients (Eq. test_stat_actual).  For
+                                      abs_next_batch it is the norm test (the caller sets row_weight =
+                                      local batch size and divisor = M); the per-round drivers
+                                      abs_logreg_round / abs_mlp_round form the statistics themselves
+                                      from the batch gradients of the round's last local step          */
+} abs_test_kind;
 
 typedef struct {
   int kind;             /* abs_test_kind                                              */
@@ -376,6 +385,10 @@ int abs_logreg_grads(abs_ctx* ctx, const float* A, const float* y, long long n, 
  *   *b_dev);  G_scratch [M][b][d], Gb_scratch [M][d], stats [M], T_out [M] or NULL;
  *   b_dev device int64: holds b on entry and the next batch size afterwards.
  *   ctl device counter block or NULL: B += H M b (Algorithm 2's counter), k += 1.
+ * cfg->kind == ABS_TEST_NORM_WORKERS runs Algorithm 2 as printed: no per-sample test; after
+ * the averaging the M batch gradients of the last local step (rows of Gb_scratch) give
+ * Var = b/(M-1) sum_m ||g^m - gbar||^2 and T = ceil(Var / (M eta^2 ||gbar||^2)); needs M >= 2;
+ * stats[0] receives that record (rows = M), T_out[0] the T, the other entries are unspecified.
  * Only enqueues; read b_dev (and ctl) back before sizing the next round.          */
 int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, long long n, long long d,
                      const int* idx, long long idx_stride, float* X, int M, int H, long long b,

@@ -13,7 +13,7 @@ import torch
 from . import build as _build
 
 ABS_F32, ABS_BF16 = 0, 1
-ABS_TEST_NORM, ABS_TEST_AUG_INNER_PRODUCT = 0, 1
+ABS_TEST_NORM, ABS_TEST_AUG_INNER_PRODUCT, ABS_TEST_NORM_WORKERS = 0, 1, 2
 STATUS_NONFINITE, STATUS_ZERO_MEAN, STATUS_TIMEOUT, STATUS_NORM_ONLY = 1, 2, 4, 8
 STATS_RECORD_BYTES = 56
 
@@ -487,7 +487,7 @@ def stats_to_dicts(stats):
 
 
 def make_test_cfg(kind, b_max, eta=0.0, theta=0.0, nu=0.0, row_weight=1.0, divisor=1.0):
-    code = {"norm": ABS_TEST_NORM, "aug_ip": ABS_TEST_AUG_INNER_PRODUCT}[kind]
+    code = {"norm": ABS_TEST_NORM, "aug_ip": ABS_TEST_AUG_INNER_PRODUCT, "norm_workers": ABS_TEST_NORM_WORKERS}[kind]
     return TestCfg(code, 0, float(eta), float(theta), float(nu), int(b_max), float(row_weight), float(divisor))
 
 

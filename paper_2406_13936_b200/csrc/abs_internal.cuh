@@ -149,11 +149,12 @@ __device__ __forceinline__ long long ceil_saturating(double x) {
 // scale * (variance / (constant^2 * N [* N])).  A record that cannot be used gives 0.
 __device__ __forceinline__ long long test_size_from_record(const abs_stats& s, const abs_test_cfg& cfg) {
   const bool usable = (s.status & (ABS_STATUS_NONFINITE | ABS_STATUS_TIMEOUT)) == 0u &&
-                      (cfg.kind == ABS_TEST_NORM || (s.status & ABS_STATUS_NORM_ONLY) == 0u);
+                      (cfg.kind != ABS_TEST_AUG_INNER_PRODUCT || (s.status & ABS_STATUS_NORM_ONLY) == 0u);
   if (!usable) return 0;
   const double scale = cfg.row_weight / cfg.divisor;
   const double N = s.gbar_sq;
-  if (cfg.kind == ABS_TEST_NORM) return ceil_saturating(scale * safe_ratio(s.var_norm, cfg.eta * cfg.eta * N));
+  if (cfg.kind != ABS_TEST_AUG_INNER_PRODUCT)      // the norm test, on per-sample rows or on workers' batch gradients
+    return ceil_saturating(scale * safe_ratio(s.var_norm, cfg.eta * cfg.eta * N));
   const long long t_ip = ceil_saturating(scale * safe_ratio(s.var_ip, cfg.theta * cfg.theta * N * N));
   const long long t_orth = ceil_saturating(scale * safe_ratio(s.var_orth, cfg.nu * cfg.nu * N));
   return t_ip > t_orth ? t_ip : t_orth;
@@ -229,6 +230,10 @@ int launch_stats_generic(abs_ctx* ctx, const StatsLaunch& a, int* P_out);
 int launch_stats_finalize(abs_ctx* ctx, const StatsLaunch& a, int P, const Recheck& rk = Recheck());
 // True when launch_stats_tiled would take the call (shape, alignment, workspace).
 bool stats_tiled_feasible(abs_ctx* ctx, const StatsLaunch& a);
+
+// Round end of Algorithm 2 (abs_rounds.cu), shared by the per-round drivers.
+int worker_gradient_test(abs_ctx* ctx, const float* Gb, int M, long long d, long long b, const abs_test_cfg* cfg,
+                         abs_stats* stats, long long* T_out, long long* b_dev, void* stream);
 
 // Host-side planning shared by the launchers and abs_plan_stats; ABS_OK or ABS_ERR_UNSUPPORTED.
 int plan_stats_gram(const Tuning& t, size_t smem_optin, abs_dtype dtype, long long b, abs_stats_plan* out);

@@ -668,6 +668,9 @@ extern "C" int abs_logreg_rounds_fused_opts(abs_ctx* ctx, const float* A, const 
     return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
   if (n < 1 || d < 1 || M < 1 || H < 1 || rounds < 1)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "need n, d, M, H, rounds >= 1");
+  if (cfg->kind == ABS_TEST_NORM_WORKERS)
+    return set_error(ctx, ABS_ERR_UNSUPPORTED, "the fused rounds run the per-sample tests; use abs_logreg_round for the test "
+                                               "on the workers' batch gradients");
   if (cfg->kind != ABS_TEST_NORM && cfg->kind != ABS_TEST_AUG_INNER_PRODUCT)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "unknown test kind %d", cfg->kind);
   if (cfg->b_max < 2 || !(cfg->row_weight > 0.0) || !(cfg->divisor > 0.0))

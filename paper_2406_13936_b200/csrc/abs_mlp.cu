@@ -741,7 +741,9 @@ extern "C" int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* label
     rc = abs_mlp_grads(ctx, inputs, labels, n, dims, idx_h, idx_stride, X, M, b, Gb_scratch, scratch, scratch_bytes,
                        stream);
     if (rc != ABS_OK) return rc;
-    if (h == H - 1 && G_scratch == nullptr) {
+    if (h == H - 1 && cfg->kind == ABS_TEST_NORM_WORKERS) {
+      // Algorithm 2: no per-sample statistics at all; the batch gradients are tested after the step
+    } else if (h == H - 1 && G_scratch == nullptr) {
       rc = abs_mlp_fused_stats(ctx, dims, b, M, scratch, scratch_bytes, Gb_scratch, stats, stream);
       if (rc != ABS_OK) return rc;
     } else if (h == H - 1) {
@@ -760,5 +762,7 @@ extern "C" int abs_mlp_round(abs_ctx* ctx, const float* inputs, const int* label
     rc = abs_round_count(ctx, ctl, b_dev, 1, static_cast<long long>(H) * M, 1, stream);
     if (rc != ABS_OK) return rc;
   }
+  if (cfg->kind == ABS_TEST_NORM_WORKERS)
+    return worker_gradient_test(ctx, Gb_scratch, M, d, b, cfg, stats, T_out, b_dev, stream);
   return abs_next_batch(ctx, stats, M, cfg, b_dev, T_out, b_dev, stream);
 }

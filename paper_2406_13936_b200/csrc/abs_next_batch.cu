@@ -45,11 +45,11 @@ extern "C" int abs_next_batch(abs_ctx* ctx, const abs_stats* stats, int M, const
   if (stats == nullptr || cfg == nullptr || b_cur == nullptr || b_next == nullptr)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
   if (M < 1 || M > kThreads) return set_error(ctx, ABS_ERR_INVALID_ARG, "M must be in 1..%d, got %d", kThreads, M);
-  if (cfg->kind != ABS_TEST_NORM && cfg->kind != ABS_TEST_AUG_INNER_PRODUCT)
+  if (cfg->kind != ABS_TEST_NORM && cfg->kind != ABS_TEST_AUG_INNER_PRODUCT && cfg->kind != ABS_TEST_NORM_WORKERS)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "unknown test kind %d", cfg->kind);
   if (cfg->b_max < 1 || !(cfg->row_weight > 0.0) || !(cfg->divisor > 0.0))
     return set_error(ctx, ABS_ERR_INVALID_ARG, "need b_max >= 1, row_weight > 0, divisor > 0");
-  if (cfg->kind == ABS_TEST_NORM ? !(cfg->eta > 0.0) : !(cfg->theta > 0.0 && cfg->nu > 0.0))
+  if (cfg->kind != ABS_TEST_AUG_INNER_PRODUCT ? !(cfg->eta > 0.0) : !(cfg->theta > 0.0 && cfg->nu > 0.0))
     return set_error(ctx, ABS_ERR_INVALID_ARG, "test constants must be positive");
   int prev = -1;
   ABS_CUDA_TRY(ctx, cudaGetDevice(&prev));

@@ -100,5 +100,7 @@ extern "C" int abs_logreg_round(abs_ctx* ctx, const float* A, const float* y, lo
     const int rc = abs_round_count(ctx, ctl, b_dev, 1, static_cast<long long>(H) * M, 1, stream);
     if (rc != ABS_OK) return rc;
   }
+  if (cfg->kind == ABS_TEST_NORM_WORKERS)
+    return worker_gradient_test(ctx, Gb_scratch, M, d, b, cfg, stats, T_out, b_dev, stream);
   return abs_next_batch(ctx, stats, M, cfg, b_dev, T_out, b_dev, stream);
 }

@@ -46,6 +46,8 @@ int round_per_step(abs_ctx* ctx, float* X, int M, int H, long long d, long long*
                    const abs_test_cfg* cfg, const abs_round_opts* opts, float* Gb, abs_stats* stats, long long* T_out,
                    long long* b_dev, cudaStream_t st, Produce produce) {
   if (H < 1 || M < 1) return set_error(ctx, ABS_ERR_INVALID_ARG, "need H >= 1 and M >= 1");
+  if (cfg->kind == ABS_TEST_NORM_WORKERS)
+    return set_error(ctx, ABS_ERR_UNSUPPORTED, "the test on the workers' batch gradients runs once per round (Algorithm 2)");
   const bool per_worker = opts != nullptr && opts->per_worker != 0;
   const double* eta_m = opts != nullptr ? opts->eta_m : nullptr;
   abs_round_ctl* ctl = opts != nullptr ? opts->ctl : nullptr;
@@ -88,6 +90,20 @@ int round_per_step(abs_ctx* ctx, float* X, int M, int H, long long d, long long*
 }  // namespace absk
 
 using namespace absk;
+
+// The end of a round under Algorithm 2 as printed: statistics of the M workers' batch gradients
+// (rows of Gb [M][d]) into stats[0], T and the size update with row_weight = b and divisor = M.
+int absk::worker_gradient_test(abs_ctx* ctx, const float* Gb, int M, long long d, long long b, const abs_test_cfg* cfg,
+                               abs_stats* stats, long long* T_out, long long* b_dev, void* stream) {
+  if (M < 2) return set_error(ctx, ABS_ERR_INVALID_ARG, "the variance over the workers needs M >= 2");
+  int rc = abs_test_stats(ctx, Gb, ABS_F32, 1, M, d, d, static_cast<long long>(M) * d, nullptr, stats, stream);
+  if (rc != ABS_OK) return rc;
+  abs_test_cfg c = *cfg;
+  c.kind = ABS_TEST_NORM;
+  c.row_weight = static_cast<double>(b);     // a row is the mean of b samples (Section 4.3)
+  c.divisor = static_cast<double>(M);        // Eq. test_stat_actual
+  return abs_next_batch(ctx, stats, 1, &c, b_dev, T_out, b_dev, stream);
+}
 
 extern "C" int abs_round_count(abs_ctx* ctx, abs_round_ctl* ctl, const long long* sizes, int n, long long times,
                                long long add_rounds, void* stream) {

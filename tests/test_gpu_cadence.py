@@ -347,3 +347,85 @@ def test_per_round_drivers_count_samples(ctx):
         B += H * M * b
         b = int(b_dev.item())
         assert ctl.tolist()[:2] == [B, k + 1]
+
+
+# ------------------------------------------------------------------ Algorithm 2 as printed
+@pytest.mark.parametrize("problem", ["logreg", "mlp"])
+def test_rounds_with_the_test_on_the_workers_batch_gradients(ctx, problem):
+    """Algorithm 2 ("actual implementation"): no per-sample statistics; after the averaging the M batch
+    gradients of the round's last local step give Var = b/(M-1) sum ||g^m - gbar||^2 and
+    T = ceil(Var / (M eta^2 ||gbar||^2)).  Teacher-forced rounds against the oracle; B counts H M b."""
+    M, H, eta, rounds = 4, 3, 0.5, 6
+    if problem == "logreg":
+        n, d, lr, b, b_max = 8192, 64, 0.1, 8, 4096
+        A, y = inputs.logreg_dataset(9, n, d, device="cuda")
+        X = torch.zeros((M, d), device="cuda")
+        G = torch.empty((M, b_max, d), device="cuda")
+        An, yn = f64(A), f64(y)
+        tol_stats = 1e-5
+    else:
+        dims, n, lr, b, b_max = (64, 48, 32, 10), 4096, 0.05, 8, 2048
+        inp, lab = inputs.gaussian_mixture(5, n, dim=dims[0], classes=dims[3], device="cuda")
+        X = inputs.mlp_init(6, dims, device="cuda").unsqueeze(0).repeat(M, 1).contiguous()
+        d = ctx.mlp_param_count(dims)
+        scratch = ctx.mlp_scratch(M, b_max, dims)
+        inp_n, lab_n = f64(inp), lab.cpu().numpy()
+        tol_stats = 2e-4                        # fp32 forward/backward against the fp64 oracle
+    idx = inputs.batch_indices(28, (rounds, H, M, b_max), n, device="cuda")
+    In = idx.cpu().numpy()
+    Gb = torch.empty((M, d), device="cuda")
+    stats = ctx.new_stats(M)
+    T_out = torch.zeros(M, dtype=torch.int64, device="cuda")
+    b_dev = torch.tensor([b], dtype=torch.int64, device="cuda")
+    ctl = ctx.new_round_ctl()
+    cfg = pkg.make_test_cfg("norm_workers", b_max, eta=eta)
+    B, grew = 0, False
+    for k in range(rounds):
+        X0 = f64(X)
+        if problem == "logreg":
+            ctx.abs_logreg_round(A, y, idx[k], X, H, b, lr, cfg, G, Gb, stats, b_dev, T_out=T_out, ctl=ctl)
+
+            def batch_grads(m, h, x, k=k, b=b):
+                rows = In[k, h, m, :b]
+                return orc.batch_mean(orc.logreg_per_sample_grads(An[rows], yn[rows], x))
+        else:
+            ctx.abs_mlp_round(inp, lab, dims, idx[k], X, H, b, lr, cfg, scratch, None, 0, Gb, stats, b_dev,
+                              T_out=T_out, ctl=ctl)
+
+            def batch_grads(m, h, x, k=k, b=b):
+                rows = In[k, h, m, :b]
+                return orc.batch_mean(orc.mlp_per_sample_grads(inp_n[rows], lab_n[rows], x, dims))
+        torch.cuda.synchronize()
+        Xr, b_ref, T_ref, st_ref, samples = orc.local_round_worker_test(X0, batch_grads, H, lr, b, b_max, eta)
+        params_close(X, Xr)
+        rec = pkg.stats_to_dicts(stats)[0]
+        assert rec["rows"] == M and rec["status"] == 0
+        for key in ("gbar_sq", "var_norm"):
+            assert rec[key] == pytest.approx(st_ref[key], rel=tol_stats)
+        ratio = b / M * st_ref["var_norm"] / (eta * eta * st_ref["gbar_sq"])
+        if near_integer(ratio, max(tol_stats, 1e-5)):
+            assert abs(T_out[0].item() - T_ref) <= 1
+        else:
+            assert T_out[0].item() == T_ref
+        B += samples
+        assert ctl.tolist()[:2] == [B, k + 1]
+        b_new = int(b_dev.item())
+        if T_out[0].item() == T_ref:
+            assert b_new == b_ref
+        grew = grew or b_new > b
+        assert b <= b_new <= b_max
+        b = b_new
+    assert grew
+
+
+def test_workers_test_is_refused_where_it_does_not_apply(ctx):
+    cfg = pkg.make_test_cfg("norm_workers", 64, eta=0.5)
+    A, y = inputs.logreg_dataset(9, 256, 32, device="cuda")
+    idx = inputs.batch_indices(28, (1, 1, 2, 64), 256, device="cuda")
+    X = torch.zeros((2, 32), device="cuda")
+    with pytest.raises(pkg.AbsError):                      # the fused rounds run the per-sample tests
+        ctx.abs_logreg_rounds_fused(A, y, idx, X, 1, 0.1, cfg, ctx.new_stats(2), torch.tensor([4], dtype=torch.int64, device="cuda"))
+    X1 = torch.zeros((1, 32), device="cuda")              # one worker has no variance over workers
+    with pytest.raises(pkg.AbsError):
+        ctx.abs_logreg_round(A, y, idx[0, :, :1], X1, 1, 4, 0.1, cfg, torch.empty((1, 64, 32), device="cuda"),
+                             torch.empty((1, 32), device="cuda"), ctx.new_stats(1), torch.tensor([4], dtype=torch.int64, device="cuda"))
