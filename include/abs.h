@@ -449,6 +449,11 @@ int abs_logreg_rounds_fused(abs_ctx* ctx, const float* A, const float* y, long l
  *   test_every_step:       stats, T_out, b_hist [rounds][H][M]: record, T and the size of
  *                          every local step (Algorithm 1); one cluster-wide barrier per step
  *                          more, and a grid-wide one per step when the size is shared
+ *   cfg->kind == ABS_TEST_NORM_WORKERS (with or without opts; not with test_every_step or
+ *                          per_worker; M >= 2): Algorithm 2 as printed -- no per-sample
+ *                          statistics, the norm test on the M batch gradients of the round's
+ *                          last local step after the averaging; per round stats[.][0] holds that
+ *                          record (rows = M, flagged ABS_STATUS_NORM_ONLY) and T_out[.][0] the T
  *   opts->ctl              B and k are read at the start and written back at the end; no
  *                          round starts once B >= n_stop (entries of rounds that did not
  *                          run are left untouched); X holds x_{K,0} of the last round run.  */

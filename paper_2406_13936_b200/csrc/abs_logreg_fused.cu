@@ -79,6 +79,9 @@ struct FusedParams {
   int sizes_per_worker;   // b_dev / b_hist hold one value per worker
   const double* eta_m;    // [M] norm-test constants per worker, or NULL
   abs_round_ctl* ctl;     // sample counter and stop rule, or NULL
+  int workers_test;       // Algorithm 2 as printed: no per-sample statistics; the norm test on the workers'
+                          // batch gradients of the round's last local step, after the averaging
+  float* Gpre;            // [2][M][d]  those batch gradients (alternating by round like Xpre)
 };
 
 __device__ __forceinline__ void st_cluster_f64(uint32_t addr, double v) {
@@ -191,7 +194,8 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
     for (int h = 0; h < prm.H; ++h) {
       const long long gstep = static_cast<long long>(r) * prm.H + h;
       const bool last = h == prm.H - 1;
-      const bool test_now = EVERY || last;                          // statistics on this step's gradients
+      const bool workers = !EVERY && prm.workers_test != 0;         // Algorithm 2: the test is on batch gradients
+      const bool test_now = EVERY || (last && !workers);            // per-sample statistics on this step's gradients
       const int* idx_m = prm.idx + (gstep * M + m) * prm.idx_stride;
       float4* part4 = inbox4 + (gstep & 1) * static_cast<long long>(P) * DV;
       if (EVERY && h > 0) {
@@ -347,8 +351,19 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
         }
         __syncthreads();
       }
-      if (!test_now) continue;
+      if (!test_now && !(last && workers)) continue;
 
+      if (last && workers) {
+        // ---- Algorithm 2: the step is taken; publish the parameters and the batch gradient -----------
+        float4* Gpre4 = reinterpret_cast<float4*>(prm.Gpre);
+        if (p == 0) {
+          for (int j = tid; j < DV; j += NT) {
+            __stcg(Xpre4 + (static_cast<long long>(r & 1) * M + m) * DV + j, x4[j]);
+            __stcg(Gpre4 + (static_cast<long long>(r & 1) * M + m) * DV + j, g4[j]);
+          }
+          if (tid == 0 && prm.ctl != nullptr) __stcg(prm.Sx + static_cast<long long>(r & 1) * M + m, used);
+        }
+      } else {
       // ---- phase C: statistics of the last local step's per-sample gradients -----------------
       if (warp == 0) {
         const float* g = reinterpret_cast<const float*>(g4);
@@ -535,6 +550,7 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
           if (p == 0) __stcg(Xpre4 + (static_cast<long long>(r & 1) * M + m) * DV + j, xv);
         }
       }
+      }   // per-sample statistics
       if (tid == 0 && abort_s != 0u) atomicOr(prm.flag, 1u);
       grid.sync();
       const bool timed_out = __ldcg(prm.flag) != 0u;
@@ -544,7 +560,57 @@ __global__ void __launch_bounds__(NW * 32, 1) logreg_rounds_kernel(const FusedPa
       // they are spread over the threads and issued together: the records by one warp per worker
       // (lane q reads the sums of CTA q; the shuffle tree adds them in a fixed order), the
       // parameters by thread groups that split the workers and are added in group order.
-      if (!EVERY) {
+      if (workers) {
+        // The rows are the M workers' batch gradients (Eq. test_stat_actual): gbar = mean_m g^m,
+        // V = sum_m ||g^m - gbar||^2, N = ||gbar||^2, by every CTA from the same numbers in the same order.
+        const float4* Gpre4 = reinterpret_cast<const float4*>(prm.Gpre) + static_cast<long long>(r & 1) * M * DV;
+        const float inv_M = 1.0f / static_cast<float>(M);
+        double v_loc = 0.0, n_loc = 0.0;
+        for (int jj = tid; jj < DV; jj += NT) {
+          float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int w = 0; w < M; ++w) {
+            const float4 v = __ldcg(Gpre4 + static_cast<long long>(w) * DV + jj);
+            mean.x += v.x; mean.y += v.y; mean.z += v.z; mean.w += v.w;
+          }
+          mean.x *= inv_M; mean.y *= inv_M; mean.z *= inv_M; mean.w *= inv_M;
+          float vs = 0.f;
+          for (int w = 0; w < M; ++w) {
+            const float4 v = __ldcg(Gpre4 + static_cast<long long>(w) * DV + jj);
+            const float dx = v.x - mean.x, dy = v.y - mean.y, dz = v.z - mean.z, dw = v.w - mean.w;
+            vs = fmaf(dx, dx, vs); vs = fmaf(dy, dy, vs); vs = fmaf(dz, dz, vs); vs = fmaf(dw, dw, vs);
+          }
+          v_loc += static_cast<double>(vs);
+          n_loc += static_cast<double>(fmaf(mean.x, mean.x, fmaf(mean.y, mean.y, fmaf(mean.z, mean.z, mean.w * mean.w))));
+        }
+        v_loc = warp_sum_dd(v_loc);
+        n_loc = warp_sum_dd(n_loc);
+        if (lane == 0) {
+          red[warp][0] = v_loc;
+          red[warp][1] = n_loc;
+        }
+        __syncthreads();
+        if (tid == 0) {
+          double V = 0.0, N = 0.0;
+          for (int w = 0; w < NW; ++w) {
+            V += red[w][0];
+            N += red[w][1];
+          }
+          abs_stats rec = record_from_sums(V, N, 0.0, 0.0, M, timed_out);
+          rec.status |= ABS_STATUS_NORM_ONLY;            // the per-worker inner products are not formed
+          abs_test_cfg c = prm.cfg;
+          c.kind = ABS_TEST_NORM;
+          c.row_weight = static_cast<double>(b);          // a row is the mean of b samples (Section 4.3)
+          c.divisor = static_cast<double>(M);             // Eq. test_stat_actual
+          const long long T = test_size_from_record(rec, c);
+          for (int w = 0; w < M; ++w) T_s[w] = T;
+          if (blockIdx.x == 0) {
+            prm.stats[static_cast<long long>(r) * M] = rec;
+            if (prm.T_out != nullptr) prm.T_out[static_cast<long long>(r) * M] = T;
+            if (prm.b_hist != nullptr && prm.sizes_per_worker)
+              for (int w = 0; w < M; ++w) prm.b_hist[static_cast<long long>(r) * M + w] = b;
+          }
+        }
+      } else if (!EVERY) {
         for (int w = warp; w < M; w += NW) {
           double a0 = 0.0, a1 = 0.0, a2 = 0.0, nn = 0.0;
           if (lane < P) {
@@ -668,14 +734,15 @@ extern "C" int abs_logreg_rounds_fused_opts(abs_ctx* ctx, const float* A, const 
     return set_error(ctx, ABS_ERR_INVALID_ARG, "null pointer argument");
   if (n < 1 || d < 1 || M < 1 || H < 1 || rounds < 1)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "need n, d, M, H, rounds >= 1");
-  if (cfg->kind == ABS_TEST_NORM_WORKERS)
-    return set_error(ctx, ABS_ERR_UNSUPPORTED, "the fused rounds run the per-sample tests; use abs_logreg_round for the test "
-                                               "on the workers' batch gradients");
-  if (cfg->kind != ABS_TEST_NORM && cfg->kind != ABS_TEST_AUG_INNER_PRODUCT)
+  const bool workers_test = cfg->kind == ABS_TEST_NORM_WORKERS;
+  if (workers_test && (M < 2 || (opts != nullptr && (opts->test_every_step != 0 || opts->per_worker != 0))))
+    return set_error(ctx, ABS_ERR_INVALID_ARG, "the test on the workers' batch gradients (Algorithm 2) needs M >= 2, runs once "
+                                               "per round and gives all workers one size");
+  if (cfg->kind != ABS_TEST_NORM && cfg->kind != ABS_TEST_AUG_INNER_PRODUCT && !workers_test)
     return set_error(ctx, ABS_ERR_INVALID_ARG, "unknown test kind %d", cfg->kind);
   if (cfg->b_max < 2 || !(cfg->row_weight > 0.0) || !(cfg->divisor > 0.0))
     return set_error(ctx, ABS_ERR_INVALID_ARG, "need b_max >= 2, row_weight > 0, divisor > 0");
-  if (cfg->kind == ABS_TEST_NORM ? !(cfg->eta > 0.0 || (opts != nullptr && opts->eta_m != nullptr))
+  if (cfg->kind != ABS_TEST_AUG_INNER_PRODUCT ? !(cfg->eta > 0.0 || (opts != nullptr && opts->eta_m != nullptr))
                                  : !(cfg->theta > 0.0 && cfg->nu > 0.0))
     return set_error(ctx, ABS_ERR_INVALID_ARG, "test constants must be positive");
   if (idx_stride < cfg->b_max)
@@ -738,9 +805,9 @@ extern "C" int abs_logreg_rounds_fused_opts(abs_ctx* ctx, const float* A, const 
   const size_t S_bytes = 2 * static_cast<size_t>(M) * P * 4 * sizeof(double);       // two copies each,
   const size_t xpre_bytes = 2 * static_cast<size_t>(M) * d * sizeof(float);          // alternating by round
   const size_t cnt_bytes = 2 * static_cast<size_t>(M) * sizeof(long long);
-  if (S_bytes + xpre_bytes + 2 * cnt_bytes > ctx->workspace_bytes)
+  if (S_bytes + 2 * xpre_bytes + 2 * cnt_bytes > ctx->workspace_bytes)      // Xpre and Gpre have the same size
     return set_error(ctx, ABS_ERR_WORKSPACE, "workspace of %zu bytes is too small (%zu needed)", ctx->workspace_bytes,
-                     S_bytes + xpre_bytes + 2 * cnt_bytes);
+                     S_bytes + 2 * xpre_bytes + 2 * cnt_bytes);
   unsigned char* ws = static_cast<unsigned char*>(ctx->workspace);
 
   FusedParams prm;
@@ -762,6 +829,8 @@ extern "C" int abs_logreg_rounds_fused_opts(abs_ctx* ctx, const float* A, const 
   prm.sizes_per_worker = opts != nullptr ? 1 : 0;
   prm.eta_m = opts != nullptr ? opts->eta_m : nullptr;
   prm.ctl = opts != nullptr ? opts->ctl : nullptr;
+  prm.workers_test = workers_test ? 1 : 0;
+  prm.Gpre = reinterpret_cast<float*>(ws + S_bytes + 2 * cnt_bytes + xpre_bytes);
   ABS_CUDA_TRY(ctx, cudaLaunchKernelEx(&lc, kernel, prm));
   return ABS_OK;
 }

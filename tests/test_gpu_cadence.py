@@ -418,14 +418,84 @@ def test_rounds_with_the_test_on_the_workers_batch_gradients(ctx, problem):
     assert grew
 
 
+def test_fused_rounds_with_the_test_on_the_workers_batch_gradients(ctx):
+    """Algorithm 2 inside the one-launch rounds: teacher-forced against the oracle round by round, and
+    many rounds in one launch equal to a launch per round, with the counter on the device."""
+    n, d, M, H, lr, eta, b0, b_max, rounds = 8192, 64, 4, 3, 0.1, 0.5, 8, 4096, 10
+    A, y = inputs.logreg_dataset(9, n, d, device="cuda")
+    idx = inputs.batch_indices(28, (rounds, H, M, b_max), n, device="cuda")
+    An, yn, In = f64(A), f64(y), idx.cpu().numpy()
+    cfg = pkg.make_test_cfg("norm_workers", b_max, eta=eta)
+    X = torch.zeros((M, d), device="cuda")
+    stats = ctx.new_stats(rounds * M)
+    T_out = torch.zeros((rounds, M), dtype=torch.int64, device="cuda")
+    b_dev = torch.tensor([b0], dtype=torch.int64, device="cuda")
+    b, sizes = b0, [b0]
+    for k in range(rounds):
+        X0 = f64(X)
+        ctx.abs_logreg_rounds_fused(A, y, idx[k:k + 1], X, H, lr, cfg, stats[k * M:(k + 1) * M], b_dev, T_out=T_out[k:k + 1])
+        torch.cuda.synchronize()
+
+        def batch_grads(m, h, x, k=k, b=b):
+            rows = In[k, h, m, :b]
+            return orc.batch_mean(orc.logreg_per_sample_grads(An[rows], yn[rows], x))
+        Xr, b_ref, T_ref, st_ref, _ = orc.local_round_worker_test(X0, batch_grads, H, lr, b, b_max, eta)
+        params_close(X, Xr)
+        rec = pkg.stats_to_dicts(stats[k * M:k * M + 1])[0]
+        assert rec["rows"] == M and rec["status"] == pkg.binding.STATUS_NORM_ONLY
+        for key in ("gbar_sq", "var_norm"):
+            assert rec[key] == pytest.approx(st_ref[key], rel=1e-5)
+        ratio = b / M * st_ref["var_norm"] / (eta * eta * st_ref["gbar_sq"])
+        if near_integer(ratio):
+            assert abs(T_out[k, 0].item() - T_ref) <= 1
+        else:
+            assert T_out[k, 0].item() == T_ref
+        b_new = int(b_dev.item())
+        if T_out[k, 0].item() == T_ref:
+            assert b_new == b_ref
+        b = b_new
+        sizes.append(b)
+    assert sizes[-1] > sizes[0]
+    # all rounds in one launch, with the counters: the same parameters and decisions, B = H M sum_k b_k
+    X1 = torch.zeros((M, d), device="cuda")
+    stats1 = ctx.new_stats(rounds * M)
+    T1 = torch.zeros((rounds, M), dtype=torch.int64, device="cuda")
+    b1 = torch.full((M,), b0, dtype=torch.int64, device="cuda")
+    ctl = ctx.new_round_ctl()
+    ctx.abs_logreg_rounds_fused_opts(A, y, idx, X1, H, lr, cfg, pkg.make_round_opts(ctl=ctl), stats1, b1, T_out=T1)
+    torch.cuda.synchronize()
+    assert torch.equal(X1, X) and torch.equal(T1[:, 0], T_out[:, 0]) and b1.tolist() == [sizes[-1]] * M
+    assert ctl.tolist()[:2] == [H * M * sum(sizes[:-1]), rounds]
+    # the unfused driver forms the same statistics with the library's statistics kernels
+    X3 = torch.zeros((M, d), device="cuda")
+    G = torch.empty((M, b_max, d), device="cuda")
+    Gb = torch.empty((M, d), device="cuda")
+    st3 = ctx.new_stats(M)
+    b3 = torch.tensor([b0], dtype=torch.int64, device="cuda")
+    b = b0
+    for k in range(rounds):
+        ctx.abs_logreg_round(A, y, idx[k], X3, H, b, lr, cfg, G, Gb, st3, b3)
+        b = int(b3.item())
+        if b != sizes[k + 1]:
+            assert abs(b - sizes[k + 1]) <= 1          # a ratio on a rounding boundary forks the runs
+            break
+    else:
+        params_close(X3, f64(X), tol=1e-5)
+
+
 def test_workers_test_is_refused_where_it_does_not_apply(ctx):
     cfg = pkg.make_test_cfg("norm_workers", 64, eta=0.5)
     A, y = inputs.logreg_dataset(9, 256, 32, device="cuda")
     idx = inputs.batch_indices(28, (1, 1, 2, 64), 256, device="cuda")
     X = torch.zeros((2, 32), device="cuda")
-    with pytest.raises(pkg.AbsError):                      # the fused rounds run the per-sample tests
-        ctx.abs_logreg_rounds_fused(A, y, idx, X, 1, 0.1, cfg, ctx.new_stats(2), torch.tensor([4], dtype=torch.int64, device="cuda"))
+    b_dev = torch.tensor([4, 4], dtype=torch.int64, device="cuda")
+    for opts in (pkg.make_round_opts(test_every_step=True), pkg.make_round_opts(per_worker=True)):
+        with pytest.raises(pkg.AbsError):                  # Algorithm 2 tests once per round, one size for all
+            ctx.abs_logreg_rounds_fused_opts(A, y, idx, X, 1, 0.1, cfg, opts, ctx.new_stats(2), b_dev)
     X1 = torch.zeros((1, 32), device="cuda")              # one worker has no variance over workers
     with pytest.raises(pkg.AbsError):
         ctx.abs_logreg_round(A, y, idx[0, :, :1], X1, 1, 4, 0.1, cfg, torch.empty((1, 64, 32), device="cuda"),
                              torch.empty((1, 32), device="cuda"), ctx.new_stats(1), torch.tensor([4], dtype=torch.int64, device="cuda"))
+    idx1 = inputs.batch_indices(28, (1, 1, 1, 64), 256, device="cuda")
+    with pytest.raises(pkg.AbsError):
+        ctx.abs_logreg_rounds_fused(A, y, idx1, X1, 1, 0.1, cfg, ctx.new_stats(1), b_dev[:1])
