@@ -253,18 +253,25 @@ gemm_tc_kernel(const TcParams prm) {
     const long long a_str = A_KC ? g.a_rs : g.a_cs, b_str = B_KC ? g.b_cs : g.b_rs;
     const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (a_str & 3) == 0;
     const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (b_str & 3) == 0;
+    // Software pipeline: the loads of a set's next k-block are issued between the stores of this
+    // one (A's after A is stored, B's after B), so they are in flight while the other operand is
+    // split and stored and while the stage is waited for; the registers are the same 16 vectors.
+    float4 ra[8], rb[8];
+    if (set < n_kb && !prm.drop_loads) {
+      fetch_operand<A_KC>(A, a_str, r0, g.rows, set * kTK, g.K, a_vec, t, ra);
+      fetch_operand<B_KC>(B, b_str, c0, g.cols, set * kTK, g.K, b_vec, t, rb);
+    }
     for (int kb = set; kb < n_kb; kb += kLoaderSets) {
       if (prm.drop_loads) break;                   // test hook: the waits of the other roles must run out, not hang
-      const int k0 = kb * kTK;
+      const int k_next = (kb + kLoaderSets) * kTK;                          // past K: reads nothing, gives zeros
       const int s = kb % kStagesT;
       const uint32_t pass = static_cast<uint32_t>(kb / kStagesT);
-      float4 ra[8], rb[8];
-      fetch_operand<A_KC>(A, a_str, r0, g.rows, k0, g.K, a_vec, t, ra);     // the loads are in flight while
-      fetch_operand<B_KC>(B, b_str, c0, g.cols, k0, g.K, b_vec, t, rb);     // the stage is waited for
       if (pass > 0) mbar_wait(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles);
       const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * kStageBytesT;
       stash_operand<A_KC>(stage, stage + kOperandBytes, t, ra);
+      fetch_operand<A_KC>(A, a_str, r0, g.rows, k_next, g.K, a_vec, t, ra);
       stash_operand<B_KC>(stage + 2 * kOperandBytes, stage + 3 * kOperandBytes, t, rb);
+      fetch_operand<B_KC>(B, b_str, c0, g.cols, k_next, g.K, b_vec, t, rb);
       fence_async_smem_t();                        // these stores, before the tensor core reads them
       mbar_arrive(full_u32 + 8u * s);
     }
