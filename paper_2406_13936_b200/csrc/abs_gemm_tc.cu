@@ -356,35 +356,67 @@ gemm_tc_kernel(const TcParams prm) {
       tc_before();
       mbar_arrive(accempty_u32 + 8u * buf);
     }
-    const long long r = r0 + row;
-    if (r < g.rows) {
-      const long long cfirst = c0 + cb;
-      float* Crow = g.C + z * g.c_bs + r * g.c_rs + cfirst;
-      const float* bias = (g.mode == 1 || g.mode == 2) ? g.bias + z * g.bias_bs + cfirst : nullptr;
-      const float* mrow = g.mode == 3 ? g.mask + z * g.mask_bs + r * g.mask_rs + cfirst : nullptr;
-      const bool vec = (reinterpret_cast<uintptr_t>(Crow) & 15u) == 0;
+    // The thread owns a row of the tile, so stores straight from its registers would touch 32 lines
+    // per warp instruction.  The tile goes through shared memory instead (the ring is free: the last
+    // accumulator was complete, so every product has read its operands): row r at r * 512 bytes, its
+    // 16-byte chunk c at position c ^ (r % 32), which keeps both the row-per-thread stores and the
+    // row-per-warp loads free of bank conflicts.  Then a warp instruction moves 512 contiguous bytes
+    // of one row of C (and of the mask).
 #pragma unroll
-      for (int j = 0; j < kCols; j += 4) {
-        float o[4];
+    for (int j = 0; j < kCols; j += 4) {
+      const uint32_t c = static_cast<uint32_t>((cb + j) >> 2);
+      sts128(ring_u32 + static_cast<uint32_t>(row) * 512u + ((c ^ static_cast<uint32_t>(row & 31)) << 4),
+             make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]));
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");   // the epilogue warps only
+    const int ew = warp - kLoaderSets * 4;
+    const long long c = c0 + 4 * lane;                               // this lane's four columns
+    float4 bias4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (g.mode == 1 || g.mode == 2) {
+      const float* bias = g.bias + z * g.bias_bs + c;
+      if (c < g.cols) bias4.x = bias[0];
+      if (c + 1 < g.cols) bias4.y = bias[1];
+      if (c + 2 < g.cols) bias4.z = bias[2];
+      if (c + 3 < g.cols) bias4.w = bias[3];
+    }
+    constexpr int kRowsPerWarp = kTM / kEpiWarps;
+    for (int rr = 0; rr < kRowsPerWarp; ++rr) {
+      const int trow = ew * kRowsPerWarp + rr;
+      const long long r = r0 + trow;
+      if (r >= g.rows || c >= g.cols) break;
+      const uint4 u = lds128(ring_u32 + static_cast<uint32_t>(trow) * 512u +
+                             ((static_cast<uint32_t>(lane) ^ static_cast<uint32_t>(trow & 31)) << 4));
+      float o[4] = {__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w)};
+      const bool full = c + 3 < g.cols;
+      if (g.mode == 0) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const long long c = cfirst + j + u;
-          float v = acc[j + u];
-          if (c < g.cols) {
-            if (g.mode == 0) v *= g.alpha;
-            else if (g.mode == 1) v = fmaxf(v + bias[j + u], 0.f);
-            else if (g.mode == 2) v = v + bias[j + u];
-            else v = mrow[j + u] > 0.f ? v : 0.f;
-          }
-          o[u] = v;
-        }
-        if (vec && cfirst + j + 3 < g.cols) {
-          *reinterpret_cast<float4*>(Crow + j) = make_float4(o[0], o[1], o[2], o[3]);
+        for (int q4 = 0; q4 < 4; ++q4) o[q4] *= g.alpha;
+      } else if (g.mode == 1) {
+        o[0] = fmaxf(o[0] + bias4.x, 0.f); o[1] = fmaxf(o[1] + bias4.y, 0.f);
+        o[2] = fmaxf(o[2] + bias4.z, 0.f); o[3] = fmaxf(o[3] + bias4.w, 0.f);
+      } else if (g.mode == 2) {
+        o[0] += bias4.x; o[1] += bias4.y; o[2] += bias4.z; o[3] += bias4.w;
+      } else {
+        const float* mrow = g.mask + z * g.mask_bs + r * g.mask_rs + c;
+        float mk[4] = {0.f, 0.f, 0.f, 0.f};
+        if (full && (reinterpret_cast<uintptr_t>(mrow) & 15u) == 0) {
+          const float4 m4 = __ldg(reinterpret_cast<const float4*>(mrow));
+          mk[0] = m4.x; mk[1] = m4.y; mk[2] = m4.z; mk[3] = m4.w;
         } else {
 #pragma unroll
-          for (int u = 0; u < 4; ++u)
-            if (cfirst + j + u < g.cols) Crow[j + u] = o[u];
+          for (int q4 = 0; q4 < 4; ++q4)
+            if (c + q4 < g.cols) mk[q4] = __ldg(mrow + q4);
         }
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) o[q4] = mk[q4] > 0.f ? o[q4] : 0.f;
+      }
+      float* Crow = g.C + z * g.c_bs + r * g.c_rs + c;
+      if (full && (reinterpret_cast<uintptr_t>(Crow) & 15u) == 0) {
+        *reinterpret_cast<float4*>(Crow) = make_float4(o[0], o[1], o[2], o[3]);
+      } else {
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4)
+          if (c + q4 < g.cols) Crow[q4] = o[q4];
       }
     }
   }
