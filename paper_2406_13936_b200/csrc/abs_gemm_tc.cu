@@ -5,22 +5,31 @@
 // therefore split in the loaders into hi = the value rounded to 11 bits and lo = the exact
 // remainder, and one product a b becomes three tensor-core products a_hi b_hi + a_hi b_lo + a_lo b_hi
 // (what is dropped is below 2^-22 |a b|).  The tensor core accumulates in fp32 in tensor memory
-// without rounding to nearest, so a long sum would drift: an accumulator only ever takes 32 values
-// of k, the cross terms (2^-11 of the main term) have an accumulator of their own so that the main
-// one sees four additions, and both are then added, rounded to nearest, to a running fp32 sum in
-// the registers of the epilogue warps.  Two accumulator pairs alternate so that this overlaps the
-// next k-block's products.  Measured against fp64 on the first layer of the MLP (K = 784, values up
-// to 11): rms error 4.4e-7 with all three products in one accumulator of 32 values of k, 1e-5 (max)
-// with 128 values; the CUDA-core kernels (fp32 slices folded into fp64) have 1.3e-7.
+// without rounding to nearest, so a long sum would drift: a main accumulator only ever takes 32
+// values of k (four additions) and is then added, rounded to nearest, to a running fp32 sum in the
+// registers of the epilogue warps; three of them rotate so that this overlaps the products of the
+// next two k-blocks.  The cross terms (2^-11 of the main term) have one accumulator of their own for
+// the whole of K, read once at the end: what their additions lose stays below 1e-8 of the result.
+// Measured against fp64 on the first layer of the MLP (K = 784, values up to 11): rms error 4.4e-7
+// with all three products in one accumulator of 32 values of k, 1e-5 (max) with 128 values; the
+// CUDA-core kernels (fp32 slices folded into fp64) have 1.3e-7.
 //
 // CTA = one 128 x 128 tile of C.  Warp roles: 0-7 loaders in two sets that take alternate k-blocks
 // (global -> registers -> split -> shared memory with the 128-byte swizzle: K-major when k is the
 // operand's contiguous index in global memory, MN-major when the tile's rows are, so every global
-// load and every shared-memory store moves whole 16-byte pieces and nothing is transposed; a
-// set's loads of one k-block are in flight while the other set stores its own), 8-15 epilogue (tcgen05.ld, running sum, bias / ReLU / mask,
-// store; two warps share a quarter of the TMEM lanes and take 64 columns each), 16 MMA issue and
-// TMEM allocation.  Every wait is bounded: one that runs out raises the CTA's abort flag, every role
-// falls through its loop, tensor memory is freed and the device flag word is set.
+// load and every shared-memory store moves whole 16-byte pieces and nothing is transposed; a set
+// issues the loads of its next k-block right after it has handed over the current one, so they are
+// in flight while the other set works and while the stage is waited for), 8-15 epilogue
+// (tcgen05.ld, running sum; two warps share a quarter of the TMEM lanes and take 64 columns each;
+// at the end the tile goes through shared memory so that a warp stores whole rows of C), 16 MMA
+// issue and TMEM allocation.  Every wait is bounded: one that runs out raises the CTA's abort flag,
+// every role falls through its loop, tensor memory is freed and the device flag word is set.
+//
+// Where the time goes (M = 8 workers, b = 4096, the 784-1024-1024-10 network; per k-block of a
+// CTA, measured by leaving parts out): products alone about 870 clocks, the loads 880, split and
+// stores 540, the hand-overs between the roles 500, and they overlap only partly (about 2000 per
+// k-block in all); a hand-over from the tensor core to a loader and back costs about a
+// microsecond, which is what three stages of 64 KiB barely cover.
 #include "abs_gemm.cuh"
 #include "abs_pipeline.cuh"
 
@@ -30,7 +39,7 @@ namespace {
 constexpr int kTM = 128, kTN = 128;             // tile of C
 constexpr int kTK = 32;                         // k-block: 32 floats = one 128-byte swizzled row
 constexpr int kStagesT = 3;
-constexpr int kChunkKB = 1;                     // k-blocks per tensor-memory accumulator (32 values of k)
+constexpr uint32_t kAccBufs = 3;                // main accumulators in tensor memory, one k-block (32 values of k) each
 constexpr int kOperandBytes = kTM * 128;        // one 128 x 32 fp32 operand tile
 constexpr int kStageBytesT = 4 * kOperandBytes; // A_hi, A_lo, B_hi, B_lo
 constexpr int kLoaders = 128;                   // threads of one loader set
@@ -38,7 +47,7 @@ constexpr int kLoaderSets = 2;
 constexpr int kEpiWarps = 8;
 constexpr int kMmaWarp = kLoaderSets * 4 + kEpiWarps;
 constexpr int kThreadsT = (kMmaWarp + 1) * 32;  // 544
-constexpr int kTmemCols = 512;                  // two sets of two accumulators (main, cross terms) of 128 columns
+constexpr int kTmemCols = 512;                  // three main accumulators and one for the cross terms, 128 columns each
 constexpr size_t kSmemT = static_cast<size_t>(kStagesT) * kStageBytesT + 1024 + 256;
 
 struct TcParams {
@@ -209,21 +218,21 @@ gemm_tc_kernel(const TcParams prm) {
   const uint32_t raw_u32 = smem_u32(smem_dyn);
   const uint32_t ring_u32 = (raw_u32 + 1023u) & ~1023u;            // the swizzle is a function of the address
   unsigned char* tail = smem_dyn + (ring_u32 - raw_u32) + static_cast<size_t>(kStagesT) * kStageBytesT;
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);   // full[3] empty[3] accfull[2] accempty[2] done
-  volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + 12);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);   // full[3] empty[3] accfull[3] accempty[3] done
+  volatile unsigned* abort_flag = reinterpret_cast<volatile unsigned*>(bars + 14);
   unsigned* tmem_slot = const_cast<unsigned*>(abort_flag) + 1;
   const uint32_t full_u32 = smem_u32(bars);
   const uint32_t empty_u32 = full_u32 + 8u * kStagesT;
   const uint32_t accfull_u32 = empty_u32 + 8u * kStagesT;
-  const uint32_t accempty_u32 = accfull_u32 + 16u;
-  const uint32_t done_u32 = accempty_u32 + 16u;
+  const uint32_t accempty_u32 = accfull_u32 + 8u * kAccBufs;
+  const uint32_t done_u32 = accempty_u32 + 8u * kAccBufs;
 
   if (tid == 0) {
     for (int s = 0; s < kStagesT; ++s) {
       mbar_init(full_u32 + 8u * s, kLoaders);
       mbar_init(empty_u32 + 8u * s, 1);
     }
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < kAccBufs; ++k) {
       mbar_init(accfull_u32 + 8u * k, 1);
       mbar_init(accempty_u32 + 8u * k, kEpiWarps * 32);
     }
@@ -243,7 +252,6 @@ gemm_tc_kernel(const TcParams prm) {
   const uint32_t tmem_base = *tmem_slot;
 
   const int n_kb = (g.K + kTK - 1) / kTK;
-  const int n_chunks = (n_kb + kChunkKB - 1) / kChunkKB;
 
   if (warp < kLoaderSets * 4) {
     // ---- loaders: set `set` takes the k-blocks kb = set, set + 2, ... ---------------------------
@@ -253,9 +261,9 @@ gemm_tc_kernel(const TcParams prm) {
     const long long a_str = A_KC ? g.a_rs : g.a_cs, b_str = B_KC ? g.b_cs : g.b_rs;
     const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (a_str & 3) == 0;
     const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (b_str & 3) == 0;
-    // Software pipeline: the loads of a set's next k-block are issued between the stores of this
-    // one (A's after A is stored, B's after B), so they are in flight while the other operand is
-    // split and stored and while the stage is waited for; the registers are the same 16 vectors.
+    // Software pipeline: the loads of a set's next k-block are issued as soon as this one is handed
+    // over (after the arrive: a fence or an arrive placed after them would wait for them), into the
+    // same 16 vector registers; they are in flight while the other set works and the stage is waited for.
     float4 ra[8], rb[8];
     if (set < n_kb && !prm.drop_loads) {
       fetch_operand<A_KC>(A, a_str, r0, g.rows, set * kTK, g.K, a_vec, t, ra);
@@ -269,11 +277,11 @@ gemm_tc_kernel(const TcParams prm) {
       if (pass > 0) mbar_wait(empty_u32 + 8u * s, (pass - 1) & 1u, abort_flag, prm.timeout_cycles);
       const uint32_t stage = ring_u32 + static_cast<uint32_t>(s) * kStageBytesT;
       stash_operand<A_KC>(stage, stage + kOperandBytes, t, ra);
-      fetch_operand<A_KC>(A, a_str, r0, g.rows, k_next, g.K, a_vec, t, ra);
       stash_operand<B_KC>(stage + 2 * kOperandBytes, stage + 3 * kOperandBytes, t, rb);
-      fetch_operand<B_KC>(B, b_str, c0, g.cols, k_next, g.K, b_vec, t, rb);
       fence_async_smem_t();                        // these stores, before the tensor core reads them
       mbar_arrive(full_u32 + 8u * s);
+      fetch_operand<A_KC>(A, a_str, r0, g.rows, k_next, g.K, a_vec, t, ra);
+      fetch_operand<B_KC>(B, b_str, c0, g.cols, k_next, g.K, b_vec, t, rb);
     }
   } else if (warp == kMmaWarp) {
     // ---- MMA issue ----------------------------------------------------------------------------
@@ -294,16 +302,14 @@ gemm_tc_kernel(const TcParams prm) {
     int s = 0;
     uint32_t pass = 0;
     for (int kb = 0; kb < n_kb; ++kb) {
-      const int chunk = kb / kChunkKB, pos = kb - chunk * kChunkKB;
-      const uint32_t buf = static_cast<uint32_t>(chunk) & 1u, use = static_cast<uint32_t>(chunk) >> 1;
-      if (pos == 0 && use > 0) mbar_wait(accempty_u32 + 8u * buf, (use - 1) & 1u, abort_flag, prm.timeout_cycles);
+      const uint32_t buf = static_cast<uint32_t>(kb) % kAccBufs, use = static_cast<uint32_t>(kb) / kAccBufs;
+      if (use > 0) mbar_wait(accempty_u32 + 8u * buf, (use - 1) & 1u, abort_flag, prm.timeout_cycles);
       mbar_wait(full_u32 + 8u * s, pass & 1u, abort_flag, prm.timeout_cycles);
       fence_async_smem_t();
       tc_after();
-      const uint32_t d_main = tmem_base + buf * static_cast<uint32_t>(2 * kTN), d_cross = d_main + kTN;
+      const uint32_t d_main = tmem_base + buf * static_cast<uint32_t>(kTN), d_cross = tmem_base + kAccBufs * kTN;
       const uint32_t base = ((ring_u32 + static_cast<uint32_t>(s) * kStageBytesT) & 0x3ffffu) >> 4;
       const uint32_t op16 = kOperandBytes >> 4;
-      const bool last_of_chunk = pos == kChunkKB - 1 || kb == n_kb - 1;
       if (elect_one_t()) {
 #pragma unroll
         for (int k = 0; k < kTK / 8; ++k) {                          // an instruction takes 8 values of k (32 bytes)
@@ -311,15 +317,15 @@ gemm_tc_kernel(const TcParams prm) {
           const uint64_t a_lo = desc_a | static_cast<uint64_t>(base + op16 + step_a * k);
           const uint64_t b_hi = desc_b | static_cast<uint64_t>(base + 2u * op16 + step_b * k);
           const uint64_t b_lo = desc_b | static_cast<uint64_t>(base + 3u * op16 + step_b * k);
-          // The cross terms are 2^-11 of the main term: in an accumulator of their own their additions
-          // cost nothing in accuracy, and the main accumulator takes one addition per 8 values of k.
-          const uint32_t first = (pos == 0 && k == 0) ? 0u : 1u;
-          umma_tf32(d_main, a_hi, b_hi, idesc, first);
-          umma_tf32(d_cross, a_lo, b_hi, idesc, first);
+          // The cross terms are 2^-11 of the main term: they have an accumulator of their own for the
+          // whole of K (what their additions lose is below 1e-8 of the result), and a main accumulator
+          // takes one addition per 8 values of k, four in all.
+          umma_tf32(d_main, a_hi, b_hi, idesc, k == 0 ? 0u : 1u);
+          umma_tf32(d_cross, a_lo, b_hi, idesc, (kb == 0 && k == 0) ? 0u : 1u);
           umma_tf32(d_cross, a_hi, b_lo, idesc, 1u);
         }
         umma_commit_t(empty_u32 + 8u * s);                           // the stage may be refilled
-        if (last_of_chunk) umma_commit_t(accfull_u32 + 8u * buf);
+        umma_commit_t(accfull_u32 + 8u * buf);
       }
       __syncwarp();
       if (++s == kStagesT) {
@@ -340,21 +346,37 @@ gemm_tc_kernel(const TcParams prm) {
     float acc[kCols];
 #pragma unroll
     for (int j = 0; j < kCols; ++j) acc[j] = 0.f;
-    for (int chunk = 0; chunk < n_chunks; ++chunk) {
-      const uint32_t buf = static_cast<uint32_t>(chunk) & 1u, use = static_cast<uint32_t>(chunk) >> 1;
+    const uint32_t t_row = tmem_base + static_cast<uint32_t>(cb) + (static_cast<uint32_t>(q * 32) << 16);
+    for (int kb = 0; kb < n_kb; ++kb) {
+      const uint32_t buf = static_cast<uint32_t>(kb) % kAccBufs, use = static_cast<uint32_t>(kb) / kAccBufs;
       mbar_wait_sleep(accfull_u32 + 8u * buf, use & 1u, abort_flag, prm.timeout_cycles);
       tc_after();
-      const uint32_t taddr = tmem_base + buf * static_cast<uint32_t>(2 * kTN) + static_cast<uint32_t>(cb) +
-                             (static_cast<uint32_t>(q * 32) << 16);
+      const uint32_t taddr = t_row + buf * static_cast<uint32_t>(kTN);
 #pragma unroll
-      for (int c16 = 0; c16 < kCols; c16 += 16) {
+      for (int c32 = 0; c32 < kCols; c32 += 32) {
         float v[16], w[16];
-        tmem_ld16x2_t(taddr + static_cast<uint32_t>(c16), taddr + static_cast<uint32_t>(kTN + c16), v, w);   // main, cross
+        tmem_ld16x2_t(taddr + static_cast<uint32_t>(c32), taddr + static_cast<uint32_t>(c32 + 16), v, w);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) acc[c16 + j] += v[j] + w[j];    // rounded to nearest
+        for (int j = 0; j < 16; ++j) {
+          acc[c32 + j] += v[j];                                      // rounded to nearest
+          acc[c32 + 16 + j] += w[j];
+        }
       }
       tc_before();
       mbar_arrive(accempty_u32 + 8u * buf);
+    }
+    if (n_kb > 0) {                                                  // the cross terms of the whole product
+#pragma unroll
+      for (int c32 = 0; c32 < kCols; c32 += 32) {
+        float v[16], w[16];
+        tmem_ld16x2_t(t_row + kAccBufs * kTN + static_cast<uint32_t>(c32),
+                      t_row + kAccBufs * kTN + static_cast<uint32_t>(c32 + 16), v, w);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          acc[c32 + j] += v[j];
+          acc[c32 + 16 + j] += w[j];
+        }
+      }
     }
     // The thread owns a row of the tile, so stores straight from its registers would touch 32 lines
     // per warp instruction.  The tile goes through shared memory instead (the ring is free: the last
