@@ -262,7 +262,7 @@ gemm_tc_kernel(const TcParams prm) {
     const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (a_str & 3) == 0;
     const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (b_str & 3) == 0;
     // Software pipeline: the loads of a set's next k-block are issued as soon as this one is handed
-    // over (after the arrive: a fence or an arrive placed after them would wait for them), into the
+    // over (after the arrive, so that neither the fence nor the arrive has loads ahead of it), into the
     // same 16 vector registers; they are in flight while the other set works and the stage is waited for.
     float4 ra[8], rb[8];
     if (set < n_kb && !prm.drop_loads) {
