@@ -327,7 +327,7 @@ def test_mlp_batch_and_per_sample_gradients(ctx, dims, M, b):
                                       ((300, 400, 500, 12), 2, 1000)])
 def test_mlp_tensor_core_products_match_the_cuda_core_products(ctx, dims, M, b):
     """The same forward/backward pass twice: matrix products on the tensor cores (fp32 operands split
-    into two TF32 parts, three products each, 128-value chunks added in fp32) and on the CUDA cores
+    into two TF32 parts, three products each, 32-value chunks added in fp32) and on the CUDA cores
     (fp32 products folded into fp64).  Batch gradients, activations and deltas agree to a few fp32
     ulps of the largest entry."""
     n = 4000
