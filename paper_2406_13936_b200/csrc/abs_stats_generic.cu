@@ -15,6 +15,7 @@ namespace {
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kStrip = 256;
+constexpr int kChain = 16;            // rows a thread adds up in fp32 before the sum moves on
 
 __device__ __forceinline__ float load_elt(const float* p) { return __ldg(p); }
 __device__ __forceinline__ float load_elt(const __nv_bfloat16* p) {
@@ -56,17 +57,31 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
   for (long long it = p; it < n_strips; it += P) {
     const long long j0 = it * kStrip;
     // sweep A: column sums, rows split over the warps
-    float cs[kStrip / 32];
+    // (no fp32 sum takes more than kChain terms in a row: a thread's rows are summed in groups, and
+    // the groups' sums are added to a second accumulator, so that thousands of rows of one sign or
+    // one large entry among tiny ones do not wear the low bits away)
+    float cs[kStrip / 32], cg[kStrip / 32];
 #pragma unroll
-    for (int c = 0; c < kStrip / 32; ++c) cs[c] = 0.f;
+    for (int c = 0; c < kStrip / 32; ++c) cs[c] = cg[c] = 0.f;
+    int chain = 0;
     for (long long r = warp; r < b; r += kWarps) {
       const T* row = Gm + r * row_stride + j0;
 #pragma unroll
       for (int c = 0; c < kStrip / 32; ++c) {
         const long long col = j0 + c * 32 + lane;
-        if (col < d) cs[c] += load_elt(row + c * 32 + lane);
+        if (col < d) cg[c] += load_elt(row + c * 32 + lane);
+      }
+      if (++chain == kChain) {
+        chain = 0;
+#pragma unroll
+        for (int c = 0; c < kStrip / 32; ++c) {
+          cs[c] += cg[c];
+          cg[c] = 0.f;
+        }
       }
     }
+#pragma unroll
+    for (int c = 0; c < kStrip / 32; ++c) cs[c] += cg[c];
 #pragma unroll
     for (int c = 0; c < kStrip / 32; ++c) colpart[warp][c * 32 + lane] = cs[c];
     __syncthreads();
@@ -87,6 +102,7 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
 #pragma unroll
     for (int c = 0; c < kStrip / 32; ++c) gl[c] = gbar_s[c * 32 + lane];
     float vl = 0.f;
+    chain = 0;
     for (long long r = warp; r < b; r += kWarps) {
       const T* row = Gm + r * row_stride + j0;
       float el = 0.f;
@@ -102,6 +118,11 @@ abs_stats_generic_kernel(const T* __restrict__ G, long long b, long long d, long
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) el += __shfl_xor_sync(0xffffffffu, el, off);
       if (lane == 0) e_acc[r] += static_cast<double>(el);
+      if (++chain == kChain) {
+        chain = 0;
+        vacc += static_cast<double>(vl);
+        vl = 0.f;
+      }
     }
     vacc += static_cast<double>(vl);
     __syncthreads();

@@ -280,6 +280,29 @@ def test_degenerate_inputs(ctx):
     assert run_gpu(ctx, nan, want_gbar=False)[0][0]["status"] & orc.STATUS_NONFINITE
 
 
+@pytest.mark.parametrize("b,d,pad", [(4096, 255, 0), (4096, 256, 0), (3000, 65, 1), (3000, 64, 0), (1500, 257, 3), (700, 1000, 0)])
+def test_long_columns_do_not_wear_the_low_bits_away(ctx, b, d, pad):
+    """Thousands of rows whose terms all round the same way: one entry of 3 among zeros (every later
+    term of the centred sum of squares is below half an ulp of the running sum), and identical rows
+    (a mean that is off by the rounding of a long fp32 sum shows up as variance).  Both the aligned
+    route and the alignment-free kernel must keep their fp32 chains short."""
+    base = torch.zeros((1, b, d))
+    base[0, 5, d // 2] = 3.0
+    G = make_G(0, 1, b, d, torch.float32, pad=pad)
+    G.copy_(base.to("cuda"))
+    rec = run_gpu(ctx, G, want_gbar=False)[0][0]
+    ref = orc.batch_test_stats(base[0].double().numpy())
+    assert rec["sum_sq"] == pytest.approx(9.0, rel=1e-5)
+    assert rec["var_norm"] == pytest.approx(ref["var_norm"], rel=1e-5)
+    assert rec["gbar_sq"] == pytest.approx(ref["gbar_sq"], rel=1e-5)
+    row = torch.randn(d, generator=torch.Generator().manual_seed(1))
+    G.copy_(row.repeat(b, 1).unsqueeze(0).to("cuda"))
+    rec = run_gpu(ctx, G, want_gbar=False)[0][0]
+    assert rec["status"] == 0
+    assert rec["gbar_sq"] == pytest.approx(float(row.double().pow(2).sum()), rel=1e-5)
+    assert rec["var_norm"] <= 1e-11 * rec["gbar_sq"]
+
+
 def test_invalid_arguments_are_rejected_before_any_launch(ctx):
     G = torch.ones((1, 1, 16), device="cuda")
     with pytest.raises(pkg.AbsError, match="b must be >= 2"):
