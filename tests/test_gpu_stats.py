@@ -303,6 +303,63 @@ def test_long_columns_do_not_wear_the_low_bits_away(ctx, b, d, pad):
     assert rec["var_norm"] <= 1e-11 * rec["gbar_sq"]
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_randomised_shapes_strides_and_recipes_against_the_oracle(ctx, seed):
+    """Seeded random cases: M, b (around every tile and cluster boundary), d, row padding and base offset
+    (aligned and not), both types, with or without gbar, five input recipes; every record is compared
+    with the oracle.  (Single-column cases are left out: with d = 1 and a mean far below the noise,
+    N itself is ill-conditioned in fp32.)"""
+    import random
+    rng = random.Random(seed)
+    for case in range(60):
+        dtype = rng.choice([torch.float32, torch.bfloat16])
+        M = rng.choice([1, 1, 2, 3, 8])
+        b = rng.choice([2, 3, 5, 8, 9, 16, 17, 32, 33, 40, 41, 64, 65, 128, 129, 136, 192, 256, 257, 300, 512, 513,
+                        1000, 1024, 1025, 1500, 2048, 2049, 3000, 4096, rng.randint(2, 4096)])
+        dmax = max(2, 400_000 // (M * b))
+        d = min(dmax, rng.choice([2, 3, 7, 8, 63, 64, 65, 255, 256, 257, 1000, 4099, rng.randint(2, dmax)]))
+        align = 4 if dtype == torch.float32 else 8
+        pad = rng.choice([0, 0, align, 3 * align, 1, 3, 5])
+        offset = rng.choice([0, 0, align, 1, 2, 3])
+        recipe = rng.choice(["noise", "noise", "mean", "t", "onehot"])
+        g = torch.Generator("cpu").manual_seed(1000 * seed + case)
+        if recipe == "noise":
+            base = torch.randn((1, 1, d), generator=g) / math.sqrt(d) + rng.choice([0.1, 1.0, 10.0]) * torch.randn((M, b, d), generator=g)
+        elif recipe == "mean":
+            base = torch.randn((1, 1, d), generator=g) + rng.choice([1e-3, 1e-2, 0.1]) * torch.randn((M, b, d), generator=g)
+        elif recipe == "t":
+            chi = torch.randn((3, M, b, d), generator=g).pow(2).sum(0) / 3
+            base = 1e-3 * torch.randn((M, b, d), generator=g) / chi.sqrt() + 1e-4
+        else:
+            base = torch.zeros((M, b, d))
+            base[:, rng.randrange(b), rng.randrange(d)] = 3.0
+        base = base.to(dtype)
+        buf = torch.zeros(M * b * (d + pad) + offset + 64, device="cuda", dtype=dtype)
+        G = buf[offset:offset + M * b * (d + pad)].view(M, b, d + pad)[:, :, :d]
+        G.copy_(base.to("cuda"))
+        want_gbar = rng.random() < 0.5
+        recs, gbar = run_gpu(ctx, G, want_gbar=want_gbar)
+        tol = 1e-5 if dtype == torch.float32 else 1e-3
+        what = (seed, case, dtype, M, b, d, pad, offset, recipe)
+        for m in range(M):
+            G64 = base[m].to(torch.float64).numpy()
+            ref = orc.batch_test_stats(G64)
+            rec = recs[m]
+            assert rec["rows"] == b and rec["status"] == ref["status"], what
+            assert rec["gbar_sq"] == pytest.approx(ref["gbar_sq"], rel=tol), what
+            assert rec["var_norm"] == pytest.approx(ref["var_norm"], rel=tol), what
+            assert rec["sum_sq"] == pytest.approx(ref["sum_sq"], rel=tol), what
+            N = ref["gbar_sq"]
+            # V_ip enters the test as V_ip / N^2 beside V_orth / N: where it is far below N V_norm its own
+            # digits do not matter, the bound is then relative to that scale
+            assert abs(rec["var_ip"] - ref["var_ip"]) <= max(tol * ref["var_ip"], tol * 1e-3 * N * ref["var_norm"]), what
+            orth_decides = ref["var_orth"] * N >= ref["var_ip"]
+            assert abs(rec["var_orth"] - ref["var_orth"]) <= tol * (ref["var_orth"] if orth_decides else ref["var_norm"]), what
+            if want_gbar:
+                err = np.abs(gbar[m].double().cpu().numpy() - G64.mean(axis=0)).max()
+                assert err <= 2e-6 * np.abs(G64).max(), what
+
+
 def test_invalid_arguments_are_rejected_before_any_launch(ctx):
     G = torch.ones((1, 1, 16), device="cuda")
     with pytest.raises(pkg.AbsError, match="b must be >= 2"):
