@@ -103,11 +103,13 @@ __device__ __forceinline__ float dot4(const float4 a, const float4 b, float acc)
   acc = fmaf(a.z, b.z, acc);
   return fmaf(a.w, b.w, acc);
 }
-// numerically stable logistic function minus the label
+// sigmoid(z) - label.  For the labels 1 and 0 nothing is subtracted (sigmoid(z) - 1 = -sigmoid(-z)),
+// so a well-fitted sample, whose residual is tiny, keeps its relative accuracy.
 __device__ __forceinline__ float residual(float z, float label) {
   const float ez = expf(-fabsf(z));
-  const float p = z >= 0.f ? 1.f / (1.f + ez) : ez / (1.f + ez);
-  return p - label;
+  const float big = 1.f / (1.f + ez), small = ez * big;          // sigmoid(|z|), sigmoid(-|z|)
+  const float p = z >= 0.f ? big : small, q = z >= 0.f ? small : big;   // sigmoid(z), sigmoid(-z)
+  return label == 1.f ? -q : (label == 0.f ? p : p - label);
 }
 
 __device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }

@@ -328,8 +328,12 @@ __global__ void softmax_delta_kernel(float* __restrict__ scratch, long long per_
     z[c] = e;
     sum += e;
   }
+  // the label's own entry is softmax - 1 = -(sum of the other classes) / sum: nothing is subtracted from
+  // a probability near 1, so a well-fitted sample keeps the relative accuracy of its (tiny) delta
   const int label = labels[clamp_sample(idx[m * idx_stride + i], n)];
-  for (int c = 0; c < n3; ++c) z[c] = z[c] / sum - (c == label ? 1.f : 0.f);
+  float others = 0.f;
+  for (int c = 0; c < n3; ++c) others += c == label ? 0.f : z[c];
+  for (int c = 0; c < n3; ++c) z[c] = c == label ? -others / sum : z[c] / sum;
 }
 
 // db[o] = (1/b) sum_i D[i][o].  A CTA covers 32 output units of one worker: warp w sums the rows

@@ -45,10 +45,13 @@ logreg_grads_kernel(const float* __restrict__ A, const float* __restrict__ y, lo
   for (long long j = lane; j < d; j += 32) z = fmaf(a[j], x[j], z);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
-  // numerically stable logistic function
+  // sigmoid(z) - label; for the labels 1 and 0 nothing is subtracted (sigmoid(z) - 1 = -sigmoid(-z)),
+  // so a well-fitted sample, whose residual is tiny, keeps its relative accuracy
   const float ez = expf(-fabsf(z));
-  const float p = z >= 0.f ? 1.f / (1.f + ez) : ez / (1.f + ez);
-  const float r = p - y[row];
+  const float big = 1.f / (1.f + ez), small = ez * big;          // sigmoid(|z|), sigmoid(-|z|)
+  const float p = z >= 0.f ? big : small, q = z >= 0.f ? small : big;
+  const float label = y[row];
+  const float r = label == 1.f ? -q : (label == 0.f ? p : p - label);
   float* g = G + (static_cast<long long>(m) * b + i) * d;
   for (long long j = lane; j < d; j += 32) g[j] = r * a[j];
 }

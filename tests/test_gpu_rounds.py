@@ -56,6 +56,63 @@ def test_logreg_per_sample_gradients(ctx):
         assert np.abs(got - ref).max() <= 2e-6 * np.abs(ref).max()
 
 
+def test_gradients_of_well_fitted_samples_keep_their_relative_accuracy(ctx):
+    """A sample the model fits has a residual far below 1: sigmoid(z) - 1 and softmax - 1 must not be
+    formed by subtracting from a rounded probability.  Rows are compared one by one, each relative to
+    its own norm."""
+    # logistic: x along the direction that produced the labels, no flips, |z| of about 5 to 20 (beyond 35 the
+    # oracle's own fp64 difference sigmoid(z) - 1 runs out of digits)
+    n, d, M, b = 400, 64, 2, 50
+    A, y = inputs.logreg_dataset(4, n, d, flip=0.0, device="cuda")
+    An, yn = f64(A), f64(y)
+    w = np.linalg.lstsq(An, 2.0 * yn - 1.0, rcond=None)[0]
+    X = torch.tensor(np.stack([8.0 * w, 20.0 * w]), dtype=torch.float32, device="cuda")
+    idx = inputs.batch_indices(5, (M, b), n, device="cuda")
+    G = torch.empty((M, b, d), device="cuda")
+    ctx.abs_logreg_grads(A, y, idx, X, b, G)
+    Xn, In = f64(X), idx.cpu().numpy()
+    tiny = 0
+    for m in range(M):
+        ref = orc.logreg_per_sample_grads(An[In[m]], yn[In[m]], Xn[m])
+        got = f64(G[m])
+        for i in range(b):
+            scale = np.linalg.norm(ref[i])
+            tiny += scale < 1e-3 * np.linalg.norm(An[In[m, i]])
+            assert np.linalg.norm(got[i] - ref[i]) <= 5e-5 * scale + 1e-12 * np.linalg.norm(An[In[m, i]])
+    assert tiny >= b                                  # the case is what it claims: many residuals below 1e-3
+    # softmax: a small network whose last layer is scaled up, labels = the predicted class
+    dims, M, b, n = (6, 5, 4, 3), 2, 16, 60
+    inp, _, X = mlp_problem(8, n, dims, M)
+    X = X * 1.0
+    dW3 = dims[3] * dims[2]
+    off3 = ctx.mlp_param_count(dims) - dW3 - dims[3]
+    X[:, off3:off3 + dW3] *= 12.0     # (1 - p below 1e-9 would exhaust the oracle's own fp64 difference)
+    layers = orc.mlp_unpack(f64(X[0]), dims)
+    h = f64(inp)
+    for l, (W, bias) in enumerate(layers):
+        h = h @ W.T + bias
+        if l < len(layers) - 1:
+            h = np.maximum(h, 0.0)
+    lab = torch.tensor(h.argmax(axis=1), dtype=torch.int32, device="cuda")
+    X[1] = X[0]
+    idx = inputs.batch_indices(9, (M, b), n, device="cuda")
+    scratch = ctx.mlp_scratch(M, b, dims)
+    d = ctx.mlp_param_count(dims)
+    Gb = torch.empty((M, d), device="cuda")
+    ctx.abs_mlp_grads(inp, lab, dims, idx, X, b, Gb, scratch)
+    Gs = torch.zeros((b, (d + 3) // 4 * 4), device="cuda")
+    ctx.abs_mlp_per_sample(dims, b, 0, scratch, Gs)
+    rows = idx.cpu().numpy()[0, :b]
+    ref = orc.mlp_per_sample_grads(f64(inp)[rows], lab.cpu().numpy()[rows], f64(X[0]), dims)
+    got = f64(Gs[:, :d])
+    small = 0
+    for i in range(b):
+        scale = np.linalg.norm(ref[i])
+        small += scale < 1e-3
+        assert np.linalg.norm(got[i] - ref[i]) <= 1e-3 * scale + 1e-9
+    assert small >= 3
+
+
 def logistic_loss(A, y, x):
     z = A @ x
     return float(np.mean(np.logaddexp(0.0, z) - y * z))
