@@ -85,14 +85,23 @@ namespace absk {
 
 int set_error(abs_ctx* ctx, int code, const char* fmt, ...);
 
-// Grants `kernel` at least `smem` bytes of dynamic shared memory (once per context and size).
+// Grants `kernel` at least `smem` bytes of dynamic shared memory (once per context).  The limit is a
+// property of the kernel in the process, not of the context, and setting it again lowers it: so what
+// is asked for is always the device's opt-in maximum, the same from every context and from the
+// context-free entry point, and nobody's later, smaller need can take away what another remembers
+// to have been granted.
 template <typename K>
 inline cudaError_t ensure_dynamic_smem(abs_ctx* ctx, K kernel, size_t smem) {
   const void* f = reinterpret_cast<const void*>(kernel);
   const int i = ctx->fn_cache.slot(f);
   if (i >= 0 && ctx->fn_cache.smem_granted[i] >= smem) return cudaSuccess;
-  const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  if (e == cudaSuccess && i >= 0) ctx->fn_cache.smem_granted[i] = smem;
+  cudaFuncAttributes fa;
+  cudaError_t e = cudaFuncGetAttributes(&fa, f);               // its static shared memory counts against the maximum
+  if (e != cudaSuccess) return e;
+  const size_t room = ctx->smem_optin > fa.sharedSizeBytes ? ctx->smem_optin - fa.sharedSizeBytes : 0;
+  const size_t grant = room > smem ? room : smem;
+  e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(grant));
+  if (e == cudaSuccess && i >= 0) ctx->fn_cache.smem_granted[i] = grant;
   return e;
 }
 

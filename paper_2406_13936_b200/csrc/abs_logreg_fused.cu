@@ -786,8 +786,10 @@ extern "C" int abs_logreg_rounds_fused_opts(abs_ctx* ctx, const float* A, const 
   for (int cand = kMaxCtasPerWorker; cand >= 1 && P == 0; cand >>= 1) {
     const size_t smem = smem_fixed + 2ull * cand * d * sizeof(float);
     if (smem + 2048 > ctx->smem_optin) continue;      // 2 KiB for the static shared variables
+    // (always the most this kernel can have, so that calls from other contexts or threads never lower it)
     ABS_CUDA_TRY(ctx, cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel),
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(ctx->smem_optin - 2048)));
     lc.dynamicSmemBytes = smem;
     attrs[0].val.clusterDim.x = static_cast<unsigned>(cand);
     attrs[0].val.clusterDim.y = 1;

@@ -360,6 +360,32 @@ def test_randomised_shapes_strides_and_recipes_against_the_oracle(ctx, seed):
                 assert err <= 2e-6 * np.abs(G64).max(), what
 
 
+def test_contexts_and_the_context_free_call_do_not_shrink_each_other_s_kernels(ctx):
+    """The shared-memory size a kernel may be launched with is a property of the kernel in the process,
+    not of a context.  Different batch sizes run the same kernel with different tile buffers: a second
+    context, or the context-free entry point, that needs a smaller one must not leave the first context
+    (which remembers what it was granted) unable to launch the larger one."""
+    other = pkg.Context(0)
+    try:
+        # (33, 257): without a context 257 rows go to the tiled kernel too, with the shape 33 rows use
+        for b_big, b_small in ((33, 257), (60, 33), (15, 9), (250, 130), (1000, 600), (4000, 2100)):
+            big = make_G(50 + b_big, 1, b_big, 20000, torch.float32)
+            small = make_G(60 + b_small, 1, b_small, 20000, torch.float32)
+            ref = run_gpu(ctx, big)[0][0]
+            st = ctx.new_stats(1)
+            other.abs_test_stats(small, st)
+            if b_small <= 2048:
+                pkg.abs_test_stats_noalloc(small, st)
+            torch.cuda.synchronize()
+            again = run_gpu(ctx, big)[0][0]
+            assert again == ref
+            other.abs_test_stats(big, st)
+            torch.cuda.synchronize()
+            assert pkg.stats_to_dicts(st)[0] == ref
+    finally:
+        other.close()
+
+
 def test_invalid_arguments_are_rejected_before_any_launch(ctx):
     G = torch.ones((1, 1, 16), device="cuda")
     with pytest.raises(pkg.AbsError, match="b must be >= 2"):
